@@ -1,0 +1,213 @@
+"""Seeded synthetic workloads: meshes, global arrays and (source type, target type) pairs.
+
+This module only *describes* inputs.  It holds none of the method's arithmetic (no base
+offsets, no tiling, no plan): it names meshes and distributed types and fills global arrays.
+It imports nothing else from this package, so test infrastructure can use it without loading
+the CUDA library.
+
+Notation (Section 2.2 of the paper, "Distributed array types"): a distributed type gives, per
+array dimension, the ordered list of mesh axes that partition it, listed minor-to-major (the
+first listed axis varies fastest).  Axes are named here by their index into ``mesh_shape``.
+A virtual device id is the row-major index of its coordinates over ``mesh_shape`` (last mesh
+axis fastest).
+
+The paper's evaluation samples 1000 problems with 3 mesh axes, arrays of up to 6 dimensions
+and 64 MB-800 MB of global data, each mesh axis either replicated or partitioning one
+dimension (Section 8, "Evaluation").  Those problems are not published; the workloads below
+stand in for them with the same structure.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Sequence, Tuple
+
+import numpy as np
+
+AxesPerDim = Tuple[Tuple[int, ...], ...]
+
+
+@dataclass(frozen=True)
+class DistType:
+    """A distributed array type: global shape plus, per dimension, its mesh axes (minor first)."""
+
+    global_shape: Tuple[int, ...]
+    axes: AxesPerDim
+
+    def __post_init__(self):
+        if len(self.global_shape) != len(self.axes):
+            raise ValueError("one axis list per dimension is required")
+
+    @property
+    def rank(self) -> int:
+        return len(self.global_shape)
+
+    def notation(self, mesh_shape: Sequence[int], names: Sequence[str] | None = None) -> str:
+        """Render as the paper writes types, e.g. ``[2{x}8, 2048, 2048{y}4096]``."""
+        names = list(names) if names is not None else [f"a{i}" for i in range(len(mesh_shape))]
+        parts = []
+        for s, ax in zip(self.global_shape, self.axes):
+            if not ax:
+                parts.append(str(s))
+                continue
+            k = 1
+            for a in ax:
+                k *= mesh_shape[a]
+            tile = s // k if s % k == 0 else f"{s}/{k}"
+            parts.append(f"{tile}{{{','.join(names[a] for a in ax)}}}{s}")
+        return "[" + ", ".join(parts) + "]"
+
+
+def dist_type(global_shape: Sequence[int], axes: Sequence[Sequence[int]]) -> DistType:
+    return DistType(tuple(int(s) for s in global_shape), tuple(tuple(int(a) for a in ax) for ax in axes))
+
+
+@dataclass(frozen=True)
+class Workload:
+    """One redistribution problem: mesh, element size, source and target type, fill recipe."""
+
+    name: str
+    mesh_shape: Tuple[int, ...]
+    axis_names: Tuple[str, ...]
+    elem_bytes: int
+    src: DistType
+    dst: DistType
+    fill: str          # "linear_u32" or "random_bits"
+    seed: int
+    note: str = ""
+
+    @property
+    def n_devices(self) -> int:
+        n = 1
+        for k in self.mesh_shape:
+            n *= k
+        return n
+
+    @property
+    def global_elems(self) -> int:
+        n = 1
+        for s in self.src.global_shape:
+            n *= s
+        return n
+
+    def reversed(self) -> "Workload":
+        return Workload(self.name + "_back", self.mesh_shape, self.axis_names, self.elem_bytes,
+                        self.dst, self.src, self.fill, self.seed, self.note)
+
+    def scaled(self, global_shape: Sequence[int], name_suffix: str = "_small") -> "Workload":
+        """Same mesh and axis placement on a different global shape (for parity-sized cases)."""
+        gs = tuple(int(s) for s in global_shape)
+        return Workload(self.name + name_suffix, self.mesh_shape, self.axis_names, self.elem_bytes,
+                        DistType(gs, self.src.axes), DistType(gs, self.dst.axes), self.fill, self.seed,
+                        self.note)
+
+
+def global_array_bytes(shape: Sequence[int], elem_bytes: int, fill: str, seed: int) -> np.ndarray:
+    """The logical global array as raw bytes, shape ``(*shape, elem_bytes)``, dtype uint8.
+
+    ``linear_u32``: element value is its global row-major linear index (4-byte little endian).
+    ``random_bits``: every bit drawn from ``numpy.random.default_rng(seed)``; bf16/f32 arrays
+    are filled this way so the patterns include NaNs and denormals (comparison is bytewise).
+    """
+    shape = tuple(int(s) for s in shape)
+    n = 1
+    for s in shape:
+        n *= s
+    if fill == "linear_u32":
+        if elem_bytes != 4:
+            raise ValueError("linear_u32 fill needs 4-byte elements")
+        g = np.arange(n, dtype="<u4").view(np.uint8)
+    elif fill == "random_bits":
+        rng = np.random.default_rng(seed)
+        g = rng.integers(0, 256, size=n * elem_bytes, dtype=np.uint8)
+    else:
+        raise ValueError(f"unknown fill {fill!r}")
+    return g.reshape(shape + (elem_bytes,))
+
+
+# ----------------------------------------------------------------------------------------------
+# The five benchmark configurations (full size).  Axis lists are minor-to-major.
+# ----------------------------------------------------------------------------------------------
+
+def config1() -> Workload:
+    """uint32 [256,256], value = global linear index, mesh (x:2, y:2); {d0:x,d1:y} -> {d0:y,d1:x}."""
+    gs = (256, 256)
+    return Workload("c1", (2, 2), ("x", "y"), 4, dist_type(gs, [[0], [1]]), dist_type(gs, [[1], [0]]),
+                    "linear_u32", 2112010751, "swap across dimensions")
+
+
+def config2() -> Workload:
+    """bf16 [8,2048,4096], mesh (x:4, y:2); {d0:x,d2:y} -> {d1:(x,y)} (x minor)."""
+    gs = (8, 2048, 4096)
+    return Workload("c2", (4, 2), ("x", "y"), 2, dist_type(gs, [[0], [], [1]]), dist_type(gs, [[], [0, 1], []]),
+                    "random_bits", 2112010752, "activation reshard")
+
+
+def config3(which: str) -> Workload:
+    """bf16 [16384,16384], mesh (a:8): 'a' row->col, 'b' replicated->row, 'c' col->replicated."""
+    gs = (16384, 16384)
+    rows, cols, repl = dist_type(gs, [[0], []]), dist_type(gs, [[], [0]]), dist_type(gs, [[], []])
+    src, dst = {"a": (rows, cols), "b": (repl, rows), "c": (cols, repl)}[which]
+    return Workload("c3" + which, (8,), ("a",), 2, src, dst, "random_bits", 2112010753, "weight reshard")
+
+
+def config5(which: str) -> Workload:
+    """bf16 [32768,32768], mesh (x:4,y:4,z:4): 'a' {d0:(x,y),d1:z}->{d0:(y,x),d1:z}; 'b' ->{d0:z,d1:(y,x)}."""
+    gs = (32768, 32768)
+    src = dist_type(gs, [[0, 1], [2]])
+    dst = {"a": dist_type(gs, [[1, 0], [2]]), "b": dist_type(gs, [[2], [1, 0]])}[which]
+    return Workload("c5" + which, (4, 4, 4), ("x", "y", "z"), 2, src, dst, "random_bits", 2112010755,
+                    "permutation heavy")
+
+
+CONFIG4_MESH = (2, 4, 2)
+CONFIG4_SHAPE = (64, 128, 256, 512)
+CONFIG4_PAIR_SEED = 2112010764
+CONFIG4_FILL_SEED = 2112010754
+
+
+def _draw_type(rng: np.random.Generator, mesh_shape: Sequence[int], global_shape: Sequence[int]) -> DistType:
+    """Each mesh axis independently: replicated or partitions one uniformly chosen dimension;
+    the axis list of every dimension is then shuffled (ordered subsets, multi-axis dims allowed)."""
+    rank = len(global_shape)
+    per_dim: List[List[int]] = [[] for _ in range(rank)]
+    for a in range(len(mesh_shape)):
+        choice = int(rng.integers(0, rank + 1))      # rank == replicated
+        if choice < rank:
+            per_dim[choice].append(a)
+    out = []
+    for k in range(rank):
+        ax = per_dim[k]
+        if len(ax) > 1:
+            ax = [ax[i] for i in rng.permutation(len(ax))]
+        out.append(ax)
+    return dist_type(global_shape, out)
+
+
+def random_pairs(n_pairs: int, mesh_shape: Sequence[int], global_shape: Sequence[int], seed: int,
+                 elem_bytes: int = 4, fill_seed: int = 0, name: str = "rand") -> List[Workload]:
+    """Seeded random (source, target) pairs in the shape of the paper's sampled problems."""
+    rng = np.random.default_rng(seed)
+    names = tuple("xyzuvw"[: len(mesh_shape)])
+    out = []
+    for i in range(n_pairs):
+        src = _draw_type(rng, mesh_shape, global_shape)
+        dst = _draw_type(rng, mesh_shape, global_shape)
+        out.append(Workload(f"{name}{i:03d}", tuple(mesh_shape), names, elem_bytes, src, dst,
+                            "random_bits", fill_seed, "random sweep"))
+    return out
+
+
+def config4(n_pairs: int = 100, global_shape: Sequence[int] = CONFIG4_SHAPE) -> List[Workload]:
+    """f32 [64,128,256,512], mesh (x:2,y:4,z:2): 100 seeded random (src, dst) pairs."""
+    return random_pairs(n_pairs, CONFIG4_MESH, global_shape, CONFIG4_PAIR_SEED, 4, CONFIG4_FILL_SEED, "c4_")
+
+
+def bench_workloads() -> Dict[str, Workload]:
+    """Named single problems of the benchmark configurations at full size."""
+    c1, c2 = config1(), config2()
+    w = {"c1": c1, "c1_back": c1.reversed(), "c2": c2, "c2_back": c2.reversed()}
+    for k in "abc":
+        w["c3" + k] = config3(k)
+    for k in "ab":
+        w["c5" + k] = config5(k)
+    return w
