@@ -1,0 +1,222 @@
+/*
+ * redist -- array redistribution over a logical device mesh, executed on one NVIDIA B200.
+ *
+ * The method is the one of "Memory-efficient array redistribution through portable collective
+ * communication" (arXiv 2112.01075): a multi-dimensional array is partitioned over a logical mesh
+ * under a source distributed type and must reach a target distributed type through a sequence of
+ * the collectives allgather, alltoall, dynslice and allpermute.  Here the N mesh devices are
+ * *virtual*: every device's tile is its own buffer in the memory of one GPU, and each collective
+ * step (or a fused run of adjacent steps) is one CUDA kernel that moves the tiles of all virtual
+ * devices at once.
+ *
+ * Conventions
+ *   - A distributed type lists, per array dimension, the mesh axes that partition it, ordered
+ *     minor-to-major: the first listed axis varies fastest (Section 2.2, "Distributed array
+ *     types").  Tile size = global size / product of the listed axis sizes; it must divide
+ *     (rule wf-dim).  Axes a type does not list replicate the data.
+ *   - Virtual device id = row-major index of the device's mesh coordinates over mesh_shape
+ *     (last mesh axis fastest).  The paper leaves this numbering to the runtime (Section 2.2).
+ *   - A tile is dense, row-major, last dimension contiguous, without padding.
+ *   - All functions return a redist_status; nothing throws, aborts or prints across this
+ *     boundary.  Output arguments are untouched on failure.
+ *   - "host" / "device" on a pointer argument says which memory it must point to.
+ */
+#ifndef REDIST_H_
+#define REDIST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum redist_status {
+    REDIST_OK = 0,
+    REDIST_EINVAL = 1,       /* null pointer, bad rank / element size / flag / index                   */
+    REDIST_EILLFORMED = 2,   /* rules wf-dim / wf-type: unknown axis, axis listed twice                */
+    REDIST_ENOTDIV = 3,      /* tile size * product of axis sizes != global size (wf-dim)             */
+    REDIST_EGLOBAL = 4,      /* source and target describe different global arrays (Section 2.5)      */
+    REDIST_ESCRATCH = 5,     /* scratch buffer missing or smaller than redist_plan_scratch_bytes      */
+    REDIST_EOVERLAP = 6,     /* destination / scratch ranges overlap each other or a source           */
+    REDIST_EALIGN = 7,       /* a buffer is not aligned to redist_plan_alignment bytes                */
+    REDIST_ENOMEM = 8,       /* host allocation failed                                                */
+    REDIST_ECUDA = 9,        /* a CUDA call or kernel launch reported an error                        */
+    REDIST_EUNSUPPORTED = 10,/* beyond a built-in limit (devices, rank, sizes); see redist_limits     */
+    REDIST_EINTERNAL = 11    /* the synthesized plan failed its own end-state check (a bug)           */
+} redist_status;
+
+/*
+ * A distributed type.  rank dimensions; global_shape[rank]; the axes of dimension k are
+ * axes[axes_off[k] .. axes_off[k+1]) as indices into mesh_shape, minor-to-major.  All arrays are
+ * host memory, read during the call only.
+ */
+typedef struct redist_type {
+    int32_t rank;
+    const int64_t *global_shape;
+    const int32_t *axes_off;     /* rank + 1 entries, axes_off[0] == 0 */
+    const int32_t *axes;         /* axes_off[rank] entries             */
+} redist_type;
+
+typedef struct redist_plan_s redist_plan_t;   /* opaque, host memory, immutable once created */
+
+/* plan flags: exactly one execution mode, optionally or-ed with REDIST_NO_OVERPARTITION */
+enum {
+    REDIST_FUSE_ADJACENT = 0,    /* default: adjacent steps of the sequence run as one kernel wherever
+                                    the fused copy keeps contiguous runs of at least 64 bytes         */
+    REDIST_FUSE_NONE = 1,        /* one kernel per collective of the sequence; intermediates ping-pong
+                                    between two scratch slots per virtual device                      */
+    REDIST_FUSE_ALL = 2,         /* the whole sequence as a single kernel, no scratch                  */
+    REDIST_NAIVE = 3,            /* comparison baseline only: gather the whole global array, then
+                                    slice (the "easy" redistribution, Section 4.3)                    */
+    REDIST_MODE_MASK = 3,
+    REDIST_NO_OVERPARTITION = 16 /* forbid dynslice steps that partition the array over more mesh
+                                    axes than the target type uses (over-partitioning, Section 7.2)  */
+};
+
+enum { REDIST_MAX_RANK = 8, REDIST_MAX_MESH_AXES = 16, REDIST_MAX_DEVICES = 1024 };
+
+typedef enum redist_step_kind {
+    REDIST_STEP_DYNSLICE = 0,
+    REDIST_STEP_ALLTOALL = 1,
+    REDIST_STEP_ALLGATHER = 2,
+    REDIST_STEP_ALLPERMUTE = 3,
+    REDIST_STEP_COPY = 4          /* only for an empty sequence (equal types): tiles are copied    */
+} redist_step_kind;
+
+/* One collective of the synthesized sequence (Sections 6 and 7). */
+typedef struct redist_step_info {
+    int32_t kind;                              /* redist_step_kind                                    */
+    int32_t dim_i;                             /* dimension the axes leave (or are sliced into); -1   */
+    int32_t dim_j;                             /* alltoall: dimension the axes move to; else -1       */
+    int64_t factor;                            /* n = product of the sizes of the axes acted on       */
+    int64_t local_before[REDIST_MAX_RANK];     /* localtype before the step                           */
+    int64_t local_after[REDIST_MAX_RANK];      /* localtype after the step                            */
+    int64_t cost;                              /* cost model of the paper, in elements per device     */
+    int64_t localsize_after;                   /* elements per device after the step (for the height) */
+} redist_step_info;
+
+/* One kernel launch of the executor. */
+typedef struct redist_launch_info {
+    int32_t first_step, n_steps;   /* the collectives this launch covers                               */
+    int32_t kernel;                /* 0 dynslice, 1 alltoall, 2 allgather, 3 allpermute, 4 copy,
+                                      5 fused sequence, 6 naive gather, 7 naive slice                  */
+    int32_t vector_bytes;          /* bytes per global memory access                                   */
+    int64_t run_bytes;             /* shortest contiguous run                                          */
+    int64_t bytes_read;            /* HBM bytes the launch reads (every source element once)          */
+    int64_t bytes_written;         /* HBM bytes the launch writes                                      */
+    int64_t n_items;               /* work items (thread-block sized pieces)                           */
+    int32_t fanout;                /* destination replicas stored per element read                     */
+    int32_t reserved;
+} redist_launch_info;
+
+/*
+ * redist_plan -- synthesize the sequence of collectives from src to dst (host only, no CUDA call).
+ *
+ * Follows Section 7: decompose the mesh into prime-sized axes (Principle 1, Section 3), search the
+ * graph of weak types (nodes: local types with localsize <= max(localsize src, localsize dst);
+ * edges: multi-axes dynslice / alltoall / allgather weighted by the cost model) for a shortest
+ * path, lower it to device-map collectives (Lowering Theorem, Section 6.1), and append at most one
+ * allpermute, placed before any trailing allgathers (Section 7.3).
+ *
+ *   n_mesh_axes, mesh_shape[n_mesh_axes]   host; the logical mesh, sizes >= 1
+ *   src, dst                               host; distributed types over that mesh
+ *   elem_bytes                             1, 2, 4, 8 or 16; elements are copied, never interpreted
+ *   flags                                  see above
+ *   out                                    host; receives the plan, owned by the caller until
+ *                                          redist_plan_destroy
+ * Errors: EINVAL, EILLFORMED, ENOTDIV, EGLOBAL, EUNSUPPORTED, ENOMEM, EINTERNAL.
+ */
+redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *src,
+                          const redist_type *dst, int32_t elem_bytes, uint32_t flags, redist_plan_t **out);
+
+void redist_plan_destroy(redist_plan_t *plan);
+
+/*
+ * redist_execute -- run the plan on the GPU (asynchronous on `stream`).
+ *
+ * Executes the collectives of the plan (typing rules T-AllGather, T-DynSlice, T-AllToAll and
+ * T-Permute; low-level forms of Section 6) as strided copy kernels over all virtual devices.  The
+ * result on every device is the tile its target type prescribes; data values never change.
+ *
+ *   src_shards[N]   host array of DEVICE pointers; src_shards[d] holds localsize(src)*elem_bytes
+ *                   bytes.  Devices that replicate a tile must hold identical bytes (not checked);
+ *                   source pointers may alias each other.  Read only.
+ *   dst_shards[N]   host array of DEVICE pointers; dst_shards[d] receives localsize(dst)*elem_bytes
+ *                   bytes.  Every destination is written completely.
+ *   scratch         DEVICE pointer to at least redist_plan_scratch_bytes(plan) bytes, or NULL when
+ *                   that is 0.  Contents are undefined afterwards.
+ *   cuda_stream     a cudaStream_t (NULL = default stream) on the current device
+ * Ownership: all buffers and the stream belong to the caller.  The call allocates nothing, copies
+ * no table to the device (tables travel as kernel parameters) and does not synchronize.  A plan
+ * may be executed from several host threads at once on different streams and buffers.
+ * Errors: EINVAL, ESCRATCH, EALIGN (pointers must be multiples of redist_plan_alignment),
+ * EOVERLAP (destination and scratch ranges must be disjoint from each other and from every
+ * source; checked on the host), ECUDA (launch error; see redist_last_cuda_error).
+ */
+redist_status redist_execute(const redist_plan_t *plan, const void *const *src_shards,
+                             void *const *dst_shards, void *scratch, size_t scratch_bytes,
+                             void *cuda_stream);
+
+/*
+ * redist_execute_host -- the same redistribution for tiles that live in HOST memory.
+ *
+ * Copies every source tile to dev_src (one cudaMemcpyAsync per tile), runs redist_execute on the
+ * staged tiles and copies every result tile back, all on `stream`; returns without synchronizing.
+ *
+ *   src_host[N], dst_host[N]   host arrays of HOST pointers (pinned memory gives true async copies)
+ *   dev_src, dev_dst           DEVICE staging buffers of at least redist_plan_staging_bytes(plan, 0)
+ *                              and (plan, 1) bytes: N tiles, each rounded up to 256 bytes
+ *   scratch                    as for redist_execute
+ * Errors: as redist_execute, plus ESCRATCH for staging buffers that are too small.
+ */
+redist_status redist_execute_host(const redist_plan_t *plan, const void *const *src_host,
+                                  void *const *dst_host, void *dev_src, size_t dev_src_bytes,
+                                  void *dev_dst, size_t dev_dst_bytes, void *scratch,
+                                  size_t scratch_bytes, void *cuda_stream);
+
+/* ---- queries (host only) -------------------------------------------------------------------- */
+
+int32_t redist_plan_num_devices(const redist_plan_t *plan);               /* N                        */
+int32_t redist_plan_rank(const redist_plan_t *plan);
+int64_t redist_plan_local_elems(const redist_plan_t *plan, int32_t which); /* 0: source, 1: target    */
+size_t  redist_plan_scratch_bytes(const redist_plan_t *plan);             /* total to pass to execute */
+size_t  redist_plan_scratch_bytes_per_device(const redist_plan_t *plan);  /* the per-virtual-device
+                                               share; for REDIST_NAIVE the size of the global array,
+                                               which the literal method would hold on every device   */
+size_t  redist_plan_staging_bytes(const redist_plan_t *plan, int32_t which);
+int32_t redist_plan_alignment(const redist_plan_t *plan);                 /* required pointer alignment */
+int64_t redist_plan_height(const redist_plan_t *plan);   /* max localsize over the sequence (elements);
+                                               the memory bound of Section 4.3 says
+                                               height <= max(localsize src, localsize dst)            */
+int64_t redist_plan_cost(const redist_plan_t *plan);     /* summed cost of the sequence (elements)    */
+int32_t redist_plan_num_steps(const redist_plan_t *plan);    /* collectives in the sequence           */
+int32_t redist_plan_num_launches(const redist_plan_t *plan); /* kernels redist_execute launches       */
+redist_status redist_plan_step_info(const redist_plan_t *plan, int32_t step, redist_step_info *out);
+redist_status redist_plan_launch_info(const redist_plan_t *plan, int32_t launch, redist_launch_info *out);
+
+/*
+ * redist_plan_describe -- the typed sequence and the launch descriptors as JSON (prime mesh, every
+ * step with the axes acted on, the type and the device map after it, costs, and per launch the copy
+ * descriptor the kernel receives).  Writes at most cap bytes including the terminating NUL and
+ * returns the length the full text needs (excluding the NUL); call with cap = 0 to size a buffer.
+ */
+size_t redist_plan_describe(const redist_plan_t *plan, char *buf, size_t cap);
+
+/*
+ * redist_base_offsets -- base offset map T[[type]] (figure "Semantics for distributed dimensions
+ * and types", part (a)): out_offsets[d*rank + k] is the lowest global index in dimension k of the
+ * tile held by virtual device d; out_tile[rank] is the local tile shape.  Host only.
+ */
+redist_status redist_base_offsets(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *type,
+                                  int64_t *out_tile, int64_t *out_offsets);
+
+const char *redist_status_string(redist_status status);
+
+/* The last CUDA error code (cudaError_t as int) seen by the calling thread inside this library. */
+int32_t redist_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REDIST_H_ */

@@ -1,0 +1,138 @@
+// JSON description of a plan: the typed sequence with its device maps, and the launch descriptors.
+#include <sstream>
+
+#include "plan.hpp"
+
+namespace redist {
+
+namespace {
+
+template <class T>
+void arr(std::ostringstream &o, const std::vector<T> &v)
+{
+    o << "[";
+    for (size_t i = 0; i < v.size(); ++i) o << (i ? "," : "") << (long long)v[i];
+    o << "]";
+}
+
+template <class T>
+void arr2(std::ostringstream &o, const std::vector<std::vector<T>> &v)
+{
+    o << "[";
+    for (size_t i = 0; i < v.size(); ++i) {
+        if (i) o << ",";
+        arr(o, v[i]);
+    }
+    o << "]";
+}
+
+void state(std::ostringstream &o, const char *name, const ConcreteState &s)
+{
+    o << "\"" << name << "_axes\":";
+    arr2(o, s.ax);
+    o << ",\"" << name << "_coords\":";
+    arr2(o, s.lc);
+}
+
+void fd(std::ostringstream &o, const FastDiv *f, uint32_t n)
+{
+    o << "[";
+    for (uint32_t i = 0; i < n; ++i) o << (i ? "," : "") << f[i].d;
+    o << "]";
+}
+
+template <class T>
+void raw(std::ostringstream &o, const T *v, uint32_t n)
+{
+    o << "[";
+    for (uint32_t i = 0; i < n; ++i) o << (i ? "," : "") << (long long)v[i];
+    o << "]";
+}
+
+const char *kKind[] = {"dynslice", "alltoall", "allgather", "allpermute", "copy"};
+const char *kKernel[] = {"dynslice", "alltoall", "allgather", "allpermute", "copy", "fused", "naive_gather", "naive_slice"};
+const char *kBuf[] = {"src", "dst", "scratch0", "scratch1", "global"};
+
+}  // namespace
+
+void describe(Plan &p)
+{
+    std::ostringstream o;
+    o << "{\"mesh_shape\":";
+    arr(o, p.mesh_shape);
+    o << ",\"global_shape\":";
+    arr(o, p.global_shape);
+    o << ",\"elem_bytes\":" << p.elem_bytes << ",\"n_devices\":" << p.n_devices << ",\"flags\":" << p.flags;
+    o << ",\"primes\":[";
+    for (size_t a = 0; a < p.primes.size(); ++a)
+        o << (a ? "," : "") << "{\"parent\":" << p.primes[a].parent << ",\"size\":" << p.primes[a].size
+          << ",\"stride\":" << p.primes[a].parent_stride << "}";
+    o << "],\"src_axes\":";
+    arr2(o, p.src_pax);
+    o << ",\"dst_axes\":";
+    arr2(o, p.dst_pax);
+    o << ",\"initial_coords\":";
+    arr2(o, p.initial.lc);
+    o << ",\"local_src\":" << p.local_src << ",\"local_dst\":" << p.local_dst << ",\"height\":" << p.height
+      << ",\"cost\":" << p.cost << ",\"slot_bytes\":" << p.slot_bytes << ",\"scratch_bytes\":" << p.scratch_bytes
+      << ",\"scratch_per_device\":" << p.scratch_per_device << ",\"alignment\":" << p.alignment;
+    o << ",\"steps\":[";
+    for (size_t s = 0; s < p.steps.size(); ++s) {
+        const Step &st = p.steps[s];
+        o << (s ? "," : "") << "{\"kind\":\"" << kKind[st.kind] << "\",\"i\":" << st.dim_i << ",\"j\":" << st.dim_j
+          << ",\"factor\":" << st.factor << ",\"acting\":";
+        arr(o, st.acting);
+        o << ",";
+        state(o, "pre", st.pre);
+        o << ",";
+        state(o, "post", st.post);
+        o << ",\"source_of\":";
+        arr(o, st.source_of);
+        o << ",\"local_before\":";
+        arr(o, st.local_before);
+        o << ",\"local_after\":";
+        arr(o, st.local_after);
+        o << ",\"cost\":" << st.cost << "}";
+    }
+    o << "],\"launches\":[";
+    for (size_t l = 0; l < p.launches.size(); ++l) {
+        const Launch &L = p.launches[l];
+        const CopyGeometry &G = L.geo;
+        o << (l ? "," : "") << "{\"first_step\":" << L.first_step << ",\"n_steps\":" << L.n_steps << ",\"kernel\":\""
+          << kKernel[L.kernel] << "\",\"from\":\"" << kBuf[L.from] << "\",\"to\":\"" << kBuf[L.to] << "\""
+          << ",\"run_bytes\":" << L.run_bytes << ",\"bytes_read\":" << L.bytes_read << ",\"bytes_written\":"
+          << L.bytes_written << ",\"src_tile_bytes\":" << L.src_tile_bytes << ",\"dst_tile_bytes\":"
+          << L.dst_tile_bytes << ",\"geometry\":{\"fanout\":" << G.fanout << ",\"vec_bytes\":" << G.vec_bytes
+          << ",\"lanes\":" << G.lanes << ",\"rows_per_pass\":" << G.rows_per_pass << ",\"rows\":" << G.rows
+          << ",\"rows_per_item\":" << G.rows_per_item << ",\"items_per_box\":" << G.items_per_box.d
+          << ",\"n_items\":" << G.n_items << ",\"unit_n\":";
+        fd(o, G.unit_n, G.n_unit);
+        o << ",\"unit_m1\":";
+        fd(o, G.unit_m1, G.n_unit);
+        o << ",\"unit_m2\":";
+        fd(o, G.unit_m2, G.n_unit);
+        o << ",\"unit_ts1\":";
+        raw(o, G.unit_ts1, G.n_unit);
+        o << ",\"unit_ts2\":";
+        raw(o, G.unit_ts2, G.n_unit);
+        o << ",\"unit_b1\":";
+        raw(o, G.unit_b1, G.n_unit);
+        o << ",\"unit_b2\":";
+        raw(o, G.unit_b2, G.n_unit);
+        o << ",\"row_n\":";
+        fd(o, G.row_n, G.n_row);
+        o << ",\"row_b1\":";
+        raw(o, G.row_b1, G.n_row);
+        o << ",\"row_b2\":";
+        raw(o, G.row_b2, G.n_row);
+        o << "},\"src_holder\":";
+        arr(o, L.src_holder);
+        o << ",\"dst_devs\":";
+        arr(o, L.dst_devs);
+        o << "}";
+    }
+    o << "]}";
+    p.json = o.str();
+}
+
+}  // namespace redist

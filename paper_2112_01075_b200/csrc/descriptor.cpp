@@ -1,0 +1,284 @@
+// From two layouts of the same global array to the copy descriptor a kernel receives, and from a
+// synthesized sequence to the list of kernel launches (one per collective, or one per fused run
+// of adjacent collectives -- merging of adjacent operations, Section 7.1, taken one step further:
+// on one GPU any run of steps composes into a single strided copy).
+#include <algorithm>
+#include <numeric>
+
+#include "plan.hpp"
+
+namespace redist {
+
+namespace {
+
+FastDiv make_div(uint32_t d)
+{
+    FastDiv f{d, 0, 0};
+    if (d > 1) {
+        uint32_t lg = 0;
+        while ((1ull << lg) < d) ++lg;                 // ceil(log2 d)
+        const uint32_t pw = 31 + lg;
+        f.mul = uint32_t(((1ull << pw) + d - 1) / d);  // ceil(2^pw / d) < 2^32 because d > 2^(lg-1)
+        f.shr = pw - 32;
+    }
+    return f;
+}
+
+i64 round_up(i64 v, i64 a) { return (v + a - 1) / a * a; }
+
+struct RowDigit {
+    i64 n, b1, b2;
+};
+
+}  // namespace
+
+redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch &out)
+{
+    const int r = p.rank;
+    const i64 e = p.elem_bytes;
+    std::vector<i64> g(r), m1(r), m2(r), nq(r), es1(r), es2(r), ts1(r), ts2(r);
+    for (int k = r - 1; k >= 0; --k) {
+        g[k] = std::gcd(a.tile[k], b.tile[k]);
+        m1[k] = a.tile[k] / g[k];
+        m2[k] = b.tile[k] / g[k];
+        nq[k] = p.global_shape[k] / g[k];
+        es1[k] = k == r - 1 ? 1 : es1[k + 1] * a.tile[k + 1];
+        es2[k] = k == r - 1 ? 1 : es2[k + 1] * b.tile[k + 1];
+        ts1[k] = k == r - 1 ? 1 : ts1[k + 1] * a.ntiles[k + 1];
+        ts2[k] = k == r - 1 ? 1 : ts2[k + 1] * b.ntiles[k + 1];
+    }
+    int kp = -1;   // last dimension whose tile size differs between the two layouts
+    for (int k = 0; k < r; ++k)
+        if (a.tile[k] != b.tile[k]) kp = k;
+    i64 run_elems = 1;
+    for (int k = std::max(kp, 0); k < r; ++k) run_elems *= (k == kp ? g[k] : a.tile[k]);
+    if (kp < 0) {
+        run_elems = 1;
+        for (int k = 0; k < r; ++k) run_elems *= a.tile[k];
+    }
+    i64 run_bytes = run_elems * e;
+
+    CopyGeometry &G = out.geo;
+    G = CopyGeometry();
+    // unit digits, outer to inner
+    i64 n_boxes = 1;
+    uint32_t nu = 0;
+    for (int k = 0; k < r; ++k) {
+        if (nq[k] == 1) continue;
+        if (nq[k] >= (1ll << 31) || ts1[k] >= (1ll << 31) || ts2[k] >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+        G.unit_n[nu] = make_div(uint32_t(nq[k]));
+        G.unit_m1[nu] = make_div(uint32_t(m1[k]));
+        G.unit_m2[nu] = make_div(uint32_t(m2[k]));
+        G.unit_ts1[nu] = uint32_t(ts1[k]);
+        G.unit_ts2[nu] = uint32_t(ts2[k]);
+        G.unit_b1[nu] = g[k] * es1[k] * e;
+        G.unit_b2[nu] = g[k] * es2[k] * e;
+        n_boxes *= nq[k];
+        if (n_boxes >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+        ++nu;
+    }
+    G.n_unit = nu;
+    // row digits inside a box: the dimensions before kp, merged where both sides stay contiguous
+    std::vector<RowDigit> rows;
+    for (int k = 0; k < kp; ++k) {
+        if (g[k] == 1) continue;
+        RowDigit d{g[k], es1[k] * e, es2[k] * e};
+        rows.push_back(d);
+    }
+    for (size_t q = rows.size(); q-- > 1;) {
+        RowDigit &o = rows[q - 1], &in = rows[q];
+        if (o.b1 == in.n * in.b1 && o.b2 == in.n * in.b2) {
+            in.n *= o.n;
+            rows.erase(rows.begin() + (q - 1));
+        }
+    }
+    // vector width: the largest power of two dividing every byte quantity that forms an address
+    i64 align = 16;
+    auto fit = [&](i64 v) {
+        while (align > 1 && v % align) align >>= 1;
+    };
+    fit(run_bytes);
+    for (uint32_t u = 0; u < nu; ++u) {
+        if (G.unit_m1[u].d > 1) fit(G.unit_b1[u]);
+        if (G.unit_m2[u].d > 1) fit(G.unit_b2[u]);
+    }
+    for (const RowDigit &d : rows) {
+        fit(d.b1);
+        fit(d.b2);
+    }
+    const i64 vec = align;
+    i64 run_vecs = run_bytes / vec;
+    i64 lanes = run_vecs;
+    if (run_vecs > kBlockThreads) {
+        lanes = 1;
+        for (i64 c = kBlockThreads; c >= 1; --c)
+            if (run_vecs % c == 0) {
+                lanes = c;
+                break;
+            }
+        rows.push_back(RowDigit{run_vecs / lanes, lanes * vec, lanes * vec});
+    }
+    if (rows.size() > size_t(kMaxRowDigits)) return REDIST_EUNSUPPORTED;
+    i64 n_rows = 1;
+    for (size_t q = 0; q < rows.size(); ++q) {
+        if (rows[q].n >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+        G.row_n[q] = make_div(uint32_t(rows[q].n));
+        G.row_b1[q] = rows[q].b1;
+        G.row_b2[q] = rows[q].b2;
+        n_rows *= rows[q].n;
+        if (n_rows >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+    }
+    G.n_row = uint32_t(rows.size());
+    G.vec_bytes = uint32_t(vec);
+    G.lanes = uint32_t(lanes);
+    G.lanes_div = make_div(uint32_t(lanes));
+    G.rows_per_pass = uint32_t(kBlockThreads / lanes);
+    G.rows = uint32_t(n_rows);
+    // a work item: about 32 KiB, a whole number of passes
+    const i64 kItemBytes = 32 * 1024;
+    i64 rpi = std::max<i64>(G.rows_per_pass, kItemBytes / (lanes * vec) / G.rows_per_pass * G.rows_per_pass);
+    rpi = std::min<i64>(rpi, round_up(n_rows, G.rows_per_pass));
+    G.rows_per_item = uint32_t(rpi);
+    const i64 ipb = (n_rows + rpi - 1) / rpi;
+    G.items_per_box = make_div(uint32_t(ipb));
+    if (n_boxes * ipb >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+    G.n_items = uint32_t(n_boxes * ipb);
+
+    // tables
+    i64 nt1 = 1, nt2 = 1;
+    for (int k = 0; k < r; ++k) {
+        nt1 *= a.ntiles[k];
+        nt2 *= b.ntiles[k];
+    }
+    const int N = p.n_devices;
+    out.src_holder.assign(size_t(nt1), -1);
+    if (!a.shared_global) {
+        for (int d = N - 1; d >= 0; --d) out.src_holder[a.tile_of[d]] = d;   // lowest id holding the tile
+        for (int32_t h : out.src_holder)
+            if (h < 0) return REDIST_EINTERNAL;
+    }
+    if (b.shared_global) {
+        G.fanout = 1;
+        out.dst_devs.assign(1, -1);
+    } else {
+        if (N % nt2) return REDIST_EINTERNAL;
+        const i64 R = N / nt2;
+        G.fanout = uint32_t(R);
+        out.dst_devs.assign(size_t(nt2 * R), -1);
+        std::vector<int> fill(size_t(nt2), 0);
+        for (int d = 0; d < N; ++d) {
+            int32_t t = b.tile_of[d];
+            if (fill[t] >= R) return REDIST_EINTERNAL;
+            out.dst_devs[size_t(t) * R + fill[t]++] = d;
+        }
+    }
+    i64 gsize = 1, l1 = 1, l2 = 1;
+    for (int k = 0; k < r; ++k) {
+        gsize *= p.global_shape[k];
+        l1 *= a.tile[k];
+        l2 *= b.tile[k];
+    }
+    out.run_bytes = run_bytes;
+    out.src_tile_bytes = l1 * e;
+    out.dst_tile_bytes = l2 * e;
+    out.bytes_read = gsize * e;
+    out.bytes_written = b.shared_global ? gsize * e : i64(N) * l2 * e;
+    return REDIST_OK;
+}
+
+redist_status build_launches(Plan &p)
+{
+    const int mode = int(p.flags & REDIST_MODE_MASK);
+    const int n = int(p.steps.size());
+    const i64 e = p.elem_bytes;
+    std::vector<Layout> lay;
+    lay.push_back(layout_of(p, p.initial));
+    for (const Step &s : p.steps) lay.push_back(layout_of(p, s.post));
+    p.launches.clear();
+    p.slot_bytes = 0;
+    i64 gsize = 1;
+    for (i64 s : p.global_shape) gsize *= s;
+
+    auto add = [&](int s0, int s1, int kernel) -> redist_status {
+        Launch L;
+        L.first_step = s0;
+        L.n_steps = s1 - s0;
+        L.kernel = kernel;
+        redist_status rc = build_copy(p, lay[s0], lay[s1], L);
+        if (rc != REDIST_OK) return rc;
+        p.launches.push_back(L);
+        return REDIST_OK;
+    };
+
+    if (mode == REDIST_NAIVE) {
+        Layout glob;
+        glob.tile = p.global_shape;
+        glob.ntiles.assign(p.rank, 1);
+        glob.tile_of.assign(p.n_devices, 0);
+        glob.shared_global = true;
+        Launch a, b;
+        a.first_step = 0; a.n_steps = n; a.kernel = 6;
+        b.first_step = 0; b.n_steps = n; b.kernel = 7;
+        redist_status rc = build_copy(p, lay.front(), glob, a);
+        if (rc == REDIST_OK) rc = build_copy(p, glob, lay.back(), b);
+        if (rc != REDIST_OK) return rc;
+        a.from = BUF_SRC; a.to = BUF_GLOBAL;
+        b.from = BUF_GLOBAL; b.to = BUF_DST;
+        p.launches = {a, b};
+        p.scratch_bytes = round_up(gsize * e, 256);
+        p.scratch_per_device = gsize * e;
+    } else {
+        std::vector<std::pair<int, int>> segs;
+        if (n == 0 || mode == REDIST_FUSE_ALL) {
+            segs.push_back({0, n});
+        } else if (mode == REDIST_FUSE_NONE) {
+            for (int s = 0; s < n; ++s) segs.push_back({s, s + 1});
+        } else {
+            // fuse adjacent steps while the fused copy keeps runs of 64 bytes, or at least as long
+            // as the shortest run of the steps it replaces
+            int s = 0;
+            while (s < n) {
+                int t = s + 1;
+                Launch probe;
+                redist_status rc = build_copy(p, lay[s], lay[t], probe);
+                if (rc != REDIST_OK) return rc;
+                i64 min_run = probe.run_bytes;
+                while (t < n) {
+                    Launch one, fused;
+                    rc = build_copy(p, lay[t], lay[t + 1], one);
+                    if (rc == REDIST_OK) rc = build_copy(p, lay[s], lay[t + 1], fused);
+                    if (rc != REDIST_OK) return rc;
+                    i64 mr = std::min(min_run, one.run_bytes);
+                    if (fused.run_bytes < 64 && fused.run_bytes < mr) break;
+                    min_run = mr;
+                    ++t;
+                }
+                segs.push_back({s, t});
+                s = t;
+            }
+        }
+        for (auto &sg : segs) {
+            int kernel = 5;
+            if (sg.second - sg.first == 0) kernel = REDIST_STEP_COPY;
+            if (sg.second - sg.first == 1) kernel = p.steps[sg.first].kind;
+            redist_status rc = add(sg.first, sg.second, kernel);
+            if (rc != REDIST_OK) return rc;
+        }
+        const int nl = int(p.launches.size());
+        i64 slot = 0;
+        for (int q = 0; q + 1 < nl; ++q) slot = std::max(slot, p.launches[q].dst_tile_bytes);
+        p.slot_bytes = round_up(slot, 256);
+        const int nslots = nl <= 1 ? 0 : (nl == 2 ? 1 : 2);
+        for (int q = 0; q < nl; ++q) {
+            p.launches[q].from = q == 0 ? BUF_SRC : ((q - 1) % 2 ? BUF_SCRATCH1 : BUF_SCRATCH0);
+            p.launches[q].to = q == nl - 1 ? BUF_DST : (q % 2 ? BUF_SCRATCH1 : BUF_SCRATCH0);
+        }
+        p.scratch_per_device = nslots * p.slot_bytes;
+        p.scratch_bytes = p.scratch_per_device * p.n_devices;
+    }
+    p.alignment = 1;
+    for (const Launch &L : p.launches) p.alignment = std::max<int>(p.alignment, int(L.geo.vec_bytes));
+    return REDIST_OK;
+}
+
+}  // namespace redist

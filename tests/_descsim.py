@@ -1,0 +1,90 @@
+"""Test-side interpreter of the launch descriptors a plan reports (``redist_plan_describe``).
+
+It replays, in numpy on host byte arrays, exactly the index arithmetic the descriptor encodes
+(boxes -> tiles and offsets, row digits, contiguous runs, fan-out), so descriptor construction can
+be checked against the oracle without a GPU.  It is not a product path.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def _prod(xs):
+    n = 1
+    for x in xs:
+        n *= int(x)
+    return n
+
+
+def run_launch(L: dict, src_bufs, dst_bufs):
+    """src_bufs / dst_bufs: callables device -> 1-D uint8 array (device -1 = the shared buffer)."""
+    G = L["geometry"]
+    vec, lanes, fan = G["vec_bytes"], G["lanes"], G["fanout"]
+    run = vec * lanes
+    unit_n = G["unit_n"]
+    n_boxes = _prod(unit_n)
+    rows = G["rows"]
+    assert rows == _prod(G["row_n"])
+    assert G["n_items"] == n_boxes * G["items_per_box"]
+    assert G["items_per_box"] * G["rows_per_item"] >= rows
+    assert G["rows_per_item"] % G["rows_per_pass"] == 0 and G["rows_per_pass"] == 256 // lanes
+    # row offsets (mixed radix, last digit fastest)
+    r = np.arange(rows, dtype=np.int64)
+    s1 = np.zeros(rows, dtype=np.int64)
+    s2 = np.zeros(rows, dtype=np.int64)
+    for q in range(len(G["row_n"]) - 1, -1, -1):
+        dg = r % G["row_n"][q]
+        r = r // G["row_n"][q]
+        s1 += dg * G["row_b1"][q]
+        s2 += dg * G["row_b2"][q]
+    col = np.arange(run, dtype=np.int64)
+    written = {}
+    for box in range(n_boxes):
+        rem, t1, t2, o1, o2 = box, 0, 0, 0, 0
+        for u in range(len(unit_n) - 1, -1, -1):
+            q = rem % unit_n[u]
+            rem //= unit_n[u]
+            a1, b1 = divmod(q, G["unit_m1"][u])
+            a2, b2 = divmod(q, G["unit_m2"][u])
+            t1 += a1 * G["unit_ts1"][u]
+            t2 += a2 * G["unit_ts2"][u]
+            o1 += b1 * G["unit_b1"][u]
+            o2 += b2 * G["unit_b2"][u]
+        src = src_bufs(L["src_holder"][t1])
+        data = src[(o1 + s1)[:, None] + col[None, :]]
+        for f in range(fan):
+            dev = L["dst_devs"][t2 * fan + f]
+            dst = dst_bufs(dev)
+            idx = (o2 + s2)[:, None] + col[None, :]
+            dst[idx] = data
+            w = written.setdefault(dev, np.zeros(dst.shape[0], dtype=np.int32))
+            np.add.at(w, idx.reshape(-1), 1)
+    return written
+
+
+def run_plan(desc: dict, src_tiles):
+    """Execute all launches; returns (dst tiles as flat uint8 arrays, per-launch write-count maps)."""
+    n = desc["n_devices"]
+    e = desc["elem_bytes"]
+    src = [np.ascontiguousarray(t).reshape(-1).view(np.uint8) for t in src_tiles]
+    dst = [np.full(desc["local_dst"] * e, 0xEE, dtype=np.uint8) for _ in range(n)]
+    slot = desc["slot_bytes"]
+    scratch = np.full(max(1, desc["scratch_bytes"]), 0xDD, dtype=np.uint8)
+
+    def buf(kind):
+        def get(dev):
+            if kind == "src":
+                return src[dev]
+            if kind == "dst":
+                return dst[dev]
+            if kind == "scratch0":
+                return scratch[dev * slot:(dev + 1) * slot]
+            if kind == "scratch1":
+                return scratch[(n + dev) * slot:(n + dev + 1) * slot]
+            return scratch
+        return get
+
+    counts = []
+    for L in desc["launches"]:
+        counts.append(run_launch(L, buf(L["from"]), buf(L["to"])))
+    return dst, counts

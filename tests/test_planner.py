@@ -1,0 +1,307 @@
+"""Planner (host) tests through the C boundary: typed sequences are replayed with the paper's rules
+on real data and compared with the oracle after every step; launch descriptors are interpreted in
+numpy; costs are compared with the paper's examples and with a brute-force optimum."""
+import heapq
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import collectives as C
+from paper_2112_01075_b200 import api, workloads as wl
+from _plancheck import check_plan, types_of
+
+MODES = [api.FUSE_ADJACENT, api.FUSE_NONE, api.FUSE_ALL, api.NAIVE]
+
+
+def small(w, shape):
+    return w.scaled(shape)
+
+
+SCALED = [
+    small(wl.config1(), (8, 8)),
+    small(wl.config1().reversed(), (8, 8)),
+    small(wl.config2(), (8, 32, 16)),
+    small(wl.config2().reversed(), (8, 32, 16)),
+    small(wl.config3("a"), (16, 32)),
+    small(wl.config3("b"), (16, 32)),
+    small(wl.config3("c"), (16, 32)),
+    small(wl.config5("a"), (64, 32)),
+    small(wl.config5("b"), (64, 64)),
+]
+
+
+@pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", MODES)
+def test_benchmark_shapes_scaled_down(w, mode):
+    src, dst = types_of(w)
+    check_plan(w.mesh_shape, src, dst, w.elem_bytes, mode)
+
+
+def test_expected_sequences_for_the_benchmark_configurations():
+    exp = {"c1": ["allpermute"], "c2": ["alltoall", "alltoall"], "c2_back": ["alltoall", "alltoall"],
+           "c3a": ["alltoall"], "c3b": ["dynslice"], "c3c": ["allgather"], "c5a": ["allpermute"],
+           "c5b": ["alltoall", "allpermute"]}
+    for name, kinds in exp.items():
+        w = wl.bench_workloads()[name]
+        p = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes)
+        assert p.step_kinds() == kinds, name
+        assert p.num_launches == 1 and p.scratch_bytes == 0
+        assert p.height <= max(p.local_elems(0), p.local_elems(1))
+        rd, wr = p.bytes_moved()
+        assert rd == w.global_elems * w.elem_bytes
+        assert wr == p.n_devices * p.local_elems(1) * w.elem_bytes
+        un = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, api.FUSE_NONE)
+        assert un.num_launches == len(kinds)
+        assert un.scratch_bytes_per_device <= 2 * (max(p.local_elems(0), p.local_elems(1)) * w.elem_bytes + 255)
+
+
+def random_problem(rng, mesh, max_rank=3, mult=2):
+    rank = int(rng.integers(1, max_rank + 1))
+
+    def draw():
+        per = [[] for _ in range(rank)]
+        for a in range(len(mesh)):
+            c = int(rng.integers(0, rank + 1))
+            if c < rank:
+                per[c].append(a)
+        return tuple(tuple(ax[i] for i in rng.permutation(len(ax))) if ax else () for ax in per)
+
+    a1, a2 = draw(), draw()
+    gshape = []
+    for k in range(rank):
+        f1 = int(np.prod([mesh[a] for a in a1[k]], dtype=np.int64))
+        f2 = int(np.prod([mesh[a] for a in a2[k]], dtype=np.int64))
+        gshape.append(int(np.lcm(f1, f2)) * int(rng.integers(1, mult + 1)))
+    return (tuple(gshape), a1), (tuple(gshape), a2)
+
+
+@pytest.mark.parametrize("mesh", [(2, 2), (4,), (2, 3), (4, 6), (2, 4, 2), (3, 3), (6, 2), (8,), (2, 2, 2, 2)])
+def test_random_problems_every_step_checked(mesh):
+    rng = np.random.default_rng(sum(mesh) * 31 + len(mesh))
+    for t in range(24):
+        src, dst = random_problem(rng, mesh)
+        e = int(rng.choice([1, 2, 4, 8, 16]))
+        mode = MODES[t % 4]
+        check_plan(mesh, src, dst, e, mode, seed=t)
+
+
+def test_random_problems_element_sized_runs():
+    """Last dimension fully sharded: runs of a single element, vector width = element size."""
+    rng = np.random.default_rng(99)
+    for t in range(20):
+        mesh = (2, 3, 2)
+        src, dst = random_problem(rng, mesh, max_rank=2, mult=1)
+        check_plan(mesh, src, dst, int(rng.choice([1, 2, 4])), MODES[t % 3], seed=t)
+
+
+def test_identity_is_a_copy():
+    mesh = (2, 2)
+    t = ((8, 8), ((0,), (1,)))
+    d = check_plan(mesh, t, t, 4)
+    assert d["steps"] == [] and len(d["launches"]) == 1 and d["launches"][0]["kernel"] == "copy"
+
+
+def test_size_one_axes_and_empty_mesh():
+    check_plan((1, 2, 1), ((4, 4), ((0, 1), (2,))), ((4, 4), ((), (1,))), 2)
+    check_plan((), ((3, 5), ((), ())), ((3, 5), ((), ())), 1)
+    check_plan((1,), ((3,), ((0,),)), ((3,), ((),)), 1)
+
+
+# ------------------------------------------------------------------------- the paper's examples
+
+def test_merged_alltoall_example():
+    """[1{a}8, 8] -> [8, 1{a}8] over {a:8}: one merged alltoall of cost 8, no permutation."""
+    d = check_plan((8,), ((8, 8), ((0,), ())), ((8, 8), ((), (0,))), 4)
+    assert [s["kind"] for s in d["steps"]] == ["alltoall"]
+    assert d["steps"][0]["factor"] == 8 and d["cost"] == 8
+    assert [p["size"] for p in d["primes"]] == [2, 2, 2]
+
+
+def test_factor_decomposition_example():
+    """[3{x}12, 2{y}12] -> [2{y}12, 3{x}12] over {x:4, y:6} without gathering everything: the
+    paper's sequence uses two alltoalls (cost 2*6) plus permutations; memory stays at 6 elements."""
+    d = check_plan((4, 6), ((12, 12), ((0,), (1,))), ((12, 12), ((1,), (0,))), 4)
+    kinds = [s["kind"] for s in d["steps"]]
+    assert kinds.count("allgather") == 0 and kinds.count("dynslice") == 0
+    assert d["height"] == 6
+    assert sum(s["cost"] for s in d["steps"] if s["kind"] == "alltoall") == 12
+    assert [p["size"] for p in d["primes"]] == [2, 2, 2, 3]
+
+
+def test_oversharding_example_cost_bounds():
+    """Mesh {x:4, y:2, z:4}: the printed sequences cost 512 and 384; the search may not do worse than
+    the better one on the weak graph (the final permutation is not a graph edge, Section 7.3)."""
+    mesh, gshape = (4, 2, 4), (8, 8, 8, 4)
+    src, dst = (gshape, ((1, 0), (), (), ())), (gshape, ((), (1,), (0,), ()))
+    d = check_plan(mesh, src, dst, 4)
+    weak_cost = sum(s["cost"] for s in d["steps"] if s["kind"] != "allpermute")
+    assert weak_cost <= 384
+    assert any(s["kind"] == "dynslice" for s in d["steps"])         # over-partitioning happens
+    d2 = check_plan(mesh, src, dst, 4, api.FUSE_ADJACENT | api.NO_OVERPARTITION)
+    assert not any(s["kind"] == "dynslice" for s in d2["steps"])
+    assert sum(s["cost"] for s in d2["steps"] if s["kind"] != "allpermute") == 512
+
+
+def test_dynslice_picks_the_axis_of_the_target():
+    """[16] -> [4{x}16] on {x:4, y:4}: slicing along y would need a permutation afterwards."""
+    d = check_plan((4, 4), ((16,), ((),)), ((16,), ((0,),)), 4)
+    assert [s["kind"] for s in d["steps"]] == ["dynslice"]
+    d = check_plan((4, 4), ((16,), ((),)), ((16,), ((1,),)), 4)
+    assert [s["kind"] for s in d["steps"]] == ["dynslice"]
+
+
+def test_permutation_examples_are_single_permutes():
+    mesh = (4, 4)
+    for src, dst in [(((1024, 128), ((1, 0), ())), ((1024, 128), ((0, 1), ()))),
+                     (((128, 64), ((0,), (1,))), ((128, 64), ((1,), (0,)))),
+                     (((128,), ((0,),)), ((128,), ((1,),)))]:
+        d = check_plan(mesh, src, dst, 2)
+        assert [s["kind"] for s in d["steps"]] == ["allpermute"]
+
+
+def test_collective_sequence_examples_cost_no_more_than_printed():
+    """Figure with six sequences on {x:4, y:4}: the search is at least as cheap as either column."""
+    mesh = (4, 4)
+    g2, g3 = (512, 128), (128, 512, 128)
+    cases = [((g2, ((0, 1), ())), (g2, ((0,), (1,))), 32 * 128 * 2),                 # alltoall + permute
+             ((g3, ((0,), (), (1,))), (g3, ((), (1, 0), ())), 2 * 32 * 512 * 32),    # two alltoalls
+             ((g3, ((0,), (), (1,))), (g3, ((), (1,), ())), 32 * 512 * 32 + 128 * 128 * 128)]
+    for src, dst, printed in cases:
+        d = check_plan(mesh, src, dst, 2)
+        assert d["cost"] <= printed
+
+
+def test_permute_is_hoisted_before_trailing_allgathers():
+    """Section 7.3: a needed permutation moves in front of the final allgathers (smaller tiles)."""
+    rng = np.random.default_rng(4)
+    seen = 0
+    for t in range(400):
+        src, dst = random_problem(rng, (2, 2, 3), max_rank=2)
+        p = api.Plan((2, 2, 3), src, dst, 4)
+        kinds = p.step_kinds()
+        if "allpermute" in kinds and "allgather" in kinds:
+            assert kinds.index("allpermute") < kinds.index("allgather")
+            i = kinds.index("allpermute")
+            assert p.step_info(i).cost <= min(p.local_elems(1), p.step_info(len(kinds) - 1).localsize_after)
+            seen += 1
+        p.close()
+    assert seen > 0
+
+
+# --------------------------------------------------------------------------------- error paths
+
+def test_error_statuses():
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((4, 8), ((512, 1024), ((), (0,))), ((1024, 1024), ((), (0,))), 4)
+    assert e.value.status == 4                                  # different global arrays
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((4, 8), ((128, 256), ((0,), (1,))), ((1024, 32), ((0, 1), ())), 4)
+    assert e.value.status == 4
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((4, 8), ((128, 256), ((0,), (0,))), ((128, 256), ((), ())), 4)
+    assert e.value.status == 2                                  # axis listed twice
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((4, 8), ((128, 256), ((5,), ())), ((128, 256), ((), ())), 4)
+    assert e.value.status == 2                                  # axis not in the mesh
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((4, 8), ((6, 256), ((0,), ())), ((6, 256), ((), ())), 4)
+    assert e.value.status == 3                                  # 4 does not divide 6
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((2,), ((4,), ((0,),)), ((4,), ((),)), 3)
+    assert e.value.status == 1                                  # element size
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((2048,), ((4096,), ((0,),)), ((4096,), ((),)), 4)
+    assert e.value.status == 10                                 # more virtual devices than supported
+    with pytest.raises(api.RedistError) as e:
+        api.Plan((2,), ((4,), ((0,),)), ((4,), ((),)), 4, flags=64)
+    assert e.value.status == 1
+
+
+def test_base_offsets_match_the_oracle():
+    import oracle
+    rng = np.random.default_rng(8)
+    for mesh in [(2, 2), (4, 6), (2, 4, 2)]:
+        for _ in range(10):
+            src, _ = random_problem(rng, mesh)
+            tile, off = api.redist_base_offsets(mesh, src)
+            otile, ooff = oracle.base_offsets(mesh, src)
+            assert tile == otile and np.array_equal(np.array(off), ooff)
+
+
+# ------------------------------------------------------------- near optimality, brute force
+
+def all_strong_types(mesh, gshape):
+    """Every well-formed type over the (prime) mesh: each axis unused or in one dimension, ordered."""
+    rank = len(gshape)
+    out = set()
+    for assign in itertools.product(range(rank + 1), repeat=len(mesh)):
+        per = [[a for a in range(len(mesh)) if assign[a] == k] for k in range(rank)]
+        for orders in itertools.product(*[list(itertools.permutations(ax)) for ax in per]):
+            t = tuple(tuple(o) for o in orders)
+            if C.well_formed(mesh, gshape, t):
+                out.add(t)
+    return out
+
+
+def brute_force_optimum(mesh, gshape, a1, a2):
+    """Dijkstra over strong types with the four typing rules (multi-axes forms included) and
+    localsize <= M; returns the minimal cost of a memory-constrained sequence."""
+    M = max(C.localsize(mesh, gshape, a1), C.localsize(mesh, gshape, a2))
+    nodes = [t for t in all_strong_types(mesh, gshape) if C.localsize(mesh, gshape, t) <= M]
+    by_local = {}
+    for t in nodes:
+        by_local.setdefault(C.localtype(mesh, gshape, t), []).append(t)
+    rank = len(gshape)
+    dist = {C.norm_axes(a1): 0}
+    pq = [(0, C.norm_axes(a1))]
+    goal = C.norm_axes(a2)
+    while pq:
+        c, t = heapq.heappop(pq)
+        if c > dist.get(t, 1 << 62):
+            continue
+        if t == goal:
+            return c
+        nxt = []
+        L = C.localsize(mesh, gshape, t)
+        for u in by_local[C.localtype(mesh, gshape, t)]:
+            if u != t:
+                nxt.append((u, L))
+        unused = [a for a in range(len(mesh)) if a not in C.used_axes(t)]
+        for i in range(rank):
+            for n_ax in range(1, len(t[i]) + 1):
+                u = C.t_allgather(mesh, gshape, t, i, n_ax)
+                nxt.append((u, C.localsize(mesh, gshape, u)))
+                for j in range(rank):
+                    if j != i:
+                        try:
+                            nxt.append((C.t_alltoall(mesh, gshape, t, i, j, n_ax), L))
+                        except C.TypeError_:
+                            pass
+            for k in range(1, len(unused) + 1):
+                for seq in itertools.permutations(unused, k):
+                    try:
+                        nxt.append((C.t_dynslice(mesh, gshape, t, i, seq), 0))
+                    except C.TypeError_:
+                        pass
+        for u, w in nxt:
+            if C.localsize(mesh, gshape, u) > M:
+                continue
+            if c + w < dist.get(u, 1 << 62):
+                dist[u] = c + w
+                heapq.heappush(pq, (c + w, u))
+    raise AssertionError("target unreachable")
+
+
+@pytest.mark.parametrize("mesh", [(2, 2), (2, 3), (2, 2, 2), (2, 2, 3)])
+def test_near_optimality_against_brute_force(mesh):
+    """cost(plan) <= optimum over all memory-constrained sequences + localsize(target)."""
+    rng = np.random.default_rng(len(mesh) * 7 + mesh[-1])
+    for _ in range(10):
+        src, dst = random_problem(rng, mesh, max_rank=2, mult=2)
+        opt = brute_force_optimum(mesh, src[0], src[1], dst[1])
+        p = api.Plan(mesh, src, dst, 4)
+        assert p.cost <= opt + p.local_elems(1), (mesh, src, dst, p.cost, opt)
+        weak = sum(p.step_info(s).cost for s in range(p.num_steps) if p.step_info(s).kind != 3)
+        assert weak <= opt                                        # permutation-free part is optimal
+        p.close()
