@@ -1,0 +1,480 @@
+#!/usr/bin/env python
+"""Benchmark: effective HBM GB/s of executing a synthesized redistribution on one B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+A *step* is one pass of the workload: for ``c2`` (the default: bf16 [8,2048,4096], mesh 4x2, 8 virtual
+devices) the forward redistribution {d0:x, d2:y} -> {d1:(x,y)} followed by the reverse, i.e. two
+plans and two fused kernel launches.  Metric: effective bytes (every global element read once plus
+every destination byte written once) per second, in GB/s.  Inputs are synthetic, seeded and
+resident in HBM before the timed region; four buffer sets rotate so that no buffer is re-read
+within 1 GiB of traffic (L2 is 126 MB).  ``e2e`` is the same step through ``redist_execute_host``
+with pinned host tiles, host<->device copies inside the timed region.
+
+With ``--gpus N`` (launched by torchrun, one rank per GPU) every rank runs an independent replica:
+the method has no inter-GPU step here (virtual devices share one GPU), so there is no collective on
+the data path; only the timing is reduced (max over ranks).
+
+``--impl reference`` times the CPU oracle (``oracle/``) on the host cores for the same metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "redistribution effective HBM GB/s (read+write)"
+UNIT = "GB/s"
+N_SETS = 4
+
+
+def legs_of(workload: str):
+    """The (source, target) problems one step executes, in order."""
+    from paper_2112_01075_b200 import workloads as wl
+    b = wl.bench_workloads()
+    if workload in ("c1", "c2"):
+        return [b[workload], b[workload + "_back"]]
+    if workload == "c3":
+        return [b["c3a"], b["c3b"], b["c3c"]]
+    if workload == "c5":
+        return [b["c5a"], b["c5b"]]
+    return [b[workload]]
+
+
+def effective_bytes(w) -> int:
+    """globalsize*e read + N*localsize(dst)*e written."""
+    n_tiles = 1
+    for s, ax in zip(w.dst.global_shape, w.dst.axes):
+        for a in ax:
+            n_tiles *= w.mesh_shape[a]
+    local_dst = w.global_elems // n_tiles
+    return w.global_elems * w.elem_bytes + w.n_devices * local_dst * w.elem_bytes
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs (read only)."""
+
+    def __init__(self, index: int, period: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop_ev = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def _sample(self):
+        nv = self.nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        try:
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+        except Exception:
+            r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                 0x80: "hw_power_brake", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
+                 0x10: "sync_boost"}
+        for bit, name in names.items():
+            if r & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_ev.is_set():
+            try:
+                self._sample()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_ev.set()
+        self.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def ncu_traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            return json.load(f).get(workload)
+    except Exception:
+        return None
+
+
+# ---------------------------------------------------------------------------------------- ours
+
+class DeviceLeg:
+    """One redistribution with N_SETS rotating sets of device tiles."""
+
+    def __init__(self, w, flags, torch, api, gen, sets=N_SETS, alias_replicas=True):
+        self.w = w
+        self.plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, flags)
+        p = self.plan
+        self.n = p.n_devices
+        sb, db = p.local_elems(0) * w.elem_bytes, p.local_elems(1) * w.elem_bytes
+        G = torch.randint(0, 256, tuple(w.src.global_shape) + (w.elem_bytes,), dtype=torch.uint8, device="cuda",
+                          generator=gen)
+        self.src, self.dst = [], []
+        _, offs = api.redist_base_offsets(w.mesh_shape, w.src)
+        for _ in range(sets):
+            tiles = api.shard_global(G, w.mesh_shape, w.src)
+            # every set owns its memory; devices that replicate a tile share one buffer per set
+            # (replicas hold identical bytes, and the boundary allows source pointers to alias)
+            owned = {}
+            for d, o in enumerate(offs):
+                key = o if alias_replicas else d
+                if key not in owned:
+                    owned[key] = tiles[d].clone()
+            self.src.append([owned[o if alias_replicas else d] for d, o in enumerate(offs)])
+            self.dst.append([torch.empty(db, dtype=torch.uint8, device="cuda") for _ in range(self.n)])
+        del G
+        self.scratch = p.alloc_scratch()
+        self.eff_bytes = effective_bytes(w)
+        self.launches = p.num_launches
+
+    def run(self, i, stream_ptr, src_override=None):
+        s = src_override if src_override is not None else self.src[i % len(self.src)]
+        d = self.dst[i % len(self.dst)]
+        sp = self.scratch.data_ptr() if self.scratch is not None else 0
+        sn = self.scratch.numel() if self.scratch is not None else 0
+        self.plan.execute_ptrs([t.data_ptr() for t in s], [t.data_ptr() for t in d], sp, sn, stream_ptr)
+
+
+def time_legs(torch, legs, steps, warmup, per_launch=True):
+    """Run `steps` timed steps (after `warmup`), each step = every leg once.  Returns
+    (total_ms, per-leg list of launch durations in ms)."""
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    for i in range(warmup):
+        for leg in legs:
+            leg.run(i, sp)
+    torch.cuda.synchronize()
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+          for _ in legs] if per_launch else None
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        for k, leg in enumerate(legs):
+            if per_launch:
+                ev[k][i][0].record(stream)
+            leg.run(warmup + i, sp)
+            if per_launch:
+                ev[k][i][1].record(stream)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    total = t0.elapsed_time(t1)
+    per = [[a.elapsed_time(b) for a, b in ev[k]] for k in range(len(legs))] if per_launch else None
+    return total, per
+
+
+def run_ours(args):
+    import torch
+    from paper_2112_01075_b200 import api
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the redistribution runs in CUDA kernels only")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    api.load()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(2112010752 + rank)
+    ws = legs_of(args.workload)
+    flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
+    legs = [DeviceLeg(w, flags, torch, api, gen) for w in ws]
+    step_bytes = sum(l.eff_bytes for l in legs)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    total_ms, per = time_legs(torch, legs, args.steps, args.warmup)
+    clocks = sampler.stop()
+    barrier()
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # dominant kernel: the launch with the largest summed duration
+    sums = [sum(p) for p in per]
+    k = max(range(len(legs)), key=lambda q: sums[q])
+    dom = legs[k]
+    li = dom.plan.launch_info(0)
+    avg_ms = statistics.mean(per[k]) / dom.launches
+    peak, how = measured_peak()
+    alg = li.bytes_read + li.bytes_written
+    achieved = alg / (avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": ncu_traffic(args.workload),
+                "kernel": "redist_%s_kernel" % api.KERNELS[li.kernel].replace("naive_gather", "allgather")
+                .replace("naive_slice", "dynslice").replace("copy", "allpermute"),
+                "algorithmic_bytes_per_launch": alg, "avg_launch_us": round(avg_ms * 1e3, 2),
+                "median_launch_us": round(statistics.median(per[k]) * 1e3 / dom.launches, 2),
+                "peak_source": how + " copy bandwidth", "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)}
+
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": describe_workload(args.workload, ws), "fuse": args.fuse,
+                   "cache": f"{N_SETS} rotating buffer sets, no buffer re-read within 1 GiB of traffic",
+                   "parallelism": "replicas only" if world > 1 else "single GPU, virtual devices"},
+        "gpu_launches": args.steps * sum(l.launches for l in legs),
+        "clocks": clocks, "roofline": roofline,
+        "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in legs),
+        "memory_bound_bytes_per_virtual_device": max(max(l.plan.local_elems(0), l.plan.local_elems(1)) *
+                                                     l.w.elem_bytes for l in legs),
+        "legs": [{"name": l.w.name, "steps": l.plan.step_kinds(), "kernels": l.plan.launch_kernels(),
+                  "gbs": round(l.eff_bytes / (statistics.mean(per[q]) * 1e-3) / 1e9, 1),
+                  "us": round(statistics.mean(per[q]) * 1e3, 2)} for q, l in enumerate(legs)],
+    }
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = run_e2e(torch, api, ws, flags, max(3, min(args.steps, 10)), world, dist)
+    elif dist is not None and not args.no_e2e:
+        run_e2e(torch, api, ws, flags, max(3, min(args.steps, 10)), world, dist)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(ws)
+    if rank == 0 and world == 1 and args.others:
+        line["others"] = run_others(torch, api, gen, args)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def describe_workload(name, ws):
+    w = ws[0]
+    dt = {2: "bf16", 4: "f32/u32"}.get(w.elem_bytes, f"{w.elem_bytes}B")
+    return (f"{name}: {dt} {list(w.src.global_shape)}, mesh {dict(zip(w.axis_names, w.mesh_shape))} "
+            f"({w.n_devices} virtual devices), " +
+            " then ".join(f"{x.src.notation(x.mesh_shape, x.axis_names)} -> {x.dst.notation(x.mesh_shape, x.axis_names)}"
+                          for x in ws))
+
+
+def run_e2e(torch, api, ws, flags, steps, world, dist):
+    """The same step through redist_execute_host: pinned host tiles in, pinned host tiles out."""
+    legs = []
+    h2d = d2h = 0
+    for w in ws:
+        p = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, flags)
+        sb, db = p.local_elems(0) * w.elem_bytes, p.local_elems(1) * w.elem_bytes
+        G = torch.randint(0, 256, tuple(w.src.global_shape) + (w.elem_bytes,), dtype=torch.uint8)
+        hs = [t.reshape(-1).pin_memory() for t in api.shard_global(G, w.mesh_shape, w.src)]
+        hd = [torch.empty(db, dtype=torch.uint8).pin_memory() for _ in range(p.n_devices)]
+        dsrc = torch.empty(p.staging_bytes(0), dtype=torch.uint8, device="cuda")
+        ddst = torch.empty(p.staging_bytes(1), dtype=torch.uint8, device="cuda")
+        legs.append((p, hs, hd, dsrc, ddst, p.alloc_scratch(), effective_bytes(w)))
+        h2d += sb * p.n_devices
+        d2h += db * p.n_devices
+    stream = torch.cuda.current_stream()
+
+    def one():
+        for p, hs, hd, dsrc, ddst, scr, _ in legs:
+            p.execute_host(hs, hd, dsrc, ddst, scr, stream)
+
+    for _ in range(2):
+        one()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(steps):
+        one()
+    t1.record(stream)
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    per_step = ms / steps
+    return {"value": round(world * sum(l[6] for l in legs) / (per_step * 1e-3) / 1e9, 2), "unit": UNIT,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(per_step, 3), "steps": steps,
+            "api": "redist_execute_host (pinned host tiles, one cudaMemcpyAsync per tile each way)"}
+
+
+def run_others(torch, api, gen, args):
+    """Short measurements of the other configurations and of the comparison modes (not the headline)."""
+    out = {}
+    names = ["c1", "c3a", "c3b", "c3c", "c5a", "c5b"]
+    for name in names:
+        for fuse, flags in (("adjacent", api.FUSE_ADJACENT), ("none", api.FUSE_NONE), ("naive", api.NAIVE)):
+            ws = legs_of(name)
+            if fuse != "adjacent" and name in ("c1",):
+                continue
+            try:
+                sets = 2 if name.startswith(("c3c", "c5")) else N_SETS
+                legs = [DeviceLeg(w, flags, torch, api, gen, sets=sets) for w in ws]
+                total, per = time_legs(torch, legs, 10, 3)
+                eff = sum(l.eff_bytes for l in legs)
+                med = statistics.median([sum(per[q][i] for q in range(len(legs))) for i in range(10)])
+                out[f"{name}/{fuse}"] = {"gbs": round(eff / (med * 1e-3) / 1e9, 1), "us": round(med * 1e3, 2),
+                                         "launches": sum(l.launches for l in legs),
+                                         "scratch_per_device": max(l.plan.scratch_bytes_per_device for l in legs)}
+                del legs
+                torch.cuda.empty_cache()
+            except Exception as ex:   # report, never hide
+                out[f"{name}/{fuse}"] = {"error": str(ex)[:200]}
+    for fuse, flags in (("none", api.FUSE_NONE), ("naive", api.NAIVE)):
+        legs = [DeviceLeg(w, flags, torch, api, gen) for w in legs_of("c2")]
+        total, per = time_legs(torch, legs, 20, 3)
+        eff = sum(l.eff_bytes for l in legs)
+        out[f"c2/{fuse}"] = {"gbs": round(eff / (total / 20 * 1e-3) / 1e9, 1), "us": round(total / 20 * 1e3, 2),
+                             "launches": sum(l.launches for l in legs),
+                             "scratch_per_device": max(l.plan.scratch_bytes_per_device for l in legs)}
+    return out
+
+
+# ------------------------------------------------------------------------------ CPU oracle arms
+
+def oracle_step_fn(ws, shrink=1):
+    """Build host inputs once; return (callable running one step on the oracle, effective bytes, note)."""
+    import oracle
+    from paper_2112_01075_b200 import workloads as wl
+    cases = []
+    eff = 0
+    for w in ws:
+        if shrink > 1:
+            # bounded sample: the same mesh and types on a global array with dimension `big` divided
+            shape = list(w.src.global_shape)
+            big = max(range(len(shape)), key=lambda k: shape[k])
+            shape[big] //= shrink
+            w = w.scaled(shape, f"_1/{shrink}")
+        src = (w.src.global_shape, w.src.axes)
+        dst = (w.dst.global_shape, w.dst.axes)
+        G = wl.global_array_bytes(w.src.global_shape, w.elem_bytes, "random_bits", w.seed)
+        tiles = oracle.reslice(w.mesh_shape, src, G)
+        cases.append((w.mesh_shape, src, dst, tiles))
+        eff += effective_bytes(w)
+
+    def step():
+        for mesh, src, dst, tiles in cases:
+            oracle.redistribute(mesh, src, dst, tiles, check=False)
+
+    return step, eff
+
+
+def cpu_baseline(ws):
+    """The oracle as it stands on the host cores: a bounded sample (about 10-30 s of CPU work)."""
+    import oracle
+    step, eff = oracle_step_fn(ws)
+    cores = oracle.max_threads()
+    res = {}
+    for threads in (1, cores):
+        oracle.set_threads(threads)
+        step()
+        t_end = time.perf_counter() + 6.0
+        times = []
+        while len(times) < 3 or (time.perf_counter() < t_end and len(times) < 50):
+            t0 = time.perf_counter()
+            step()
+            times.append(time.perf_counter() - t0)
+        res[threads] = (min(times), statistics.median(times), len(times))
+    oracle.set_threads(1)
+    best = res[cores]
+    return {"value": round(eff / best[1] / 1e9, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"the whole workload, median of {best[2]} passes of the C oracle with {cores} threads "
+                      f"(materialise the global array, re-slice per device)",
+            "single_thread_gbs": round(eff / res[1][1] / 1e9, 3),
+            "ms_per_step": round(best[1] * 1e3, 2), "ms_per_step_single_thread": round(res[1][1] * 1e3, 2)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    ws = legs_of(args.workload)
+    cores = oracle.max_threads()
+    oracle.set_threads(cores)
+    step, eff = oracle_step_fn(ws)
+    t0 = time.perf_counter()
+    step()
+    one = time.perf_counter() - t0
+    shrink = 1
+    while one / shrink * (args.steps + args.warmup) > 120.0 and shrink < 256:
+        shrink *= 2
+    if shrink > 1:
+        step, eff = oracle_step_fn(ws, shrink)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = round(eff / dt / 1e9, 3)
+    sample = ("the whole workload per step" if shrink == 1 else
+              f"1/{shrink} of the workload per step (largest dimension divided by {shrink})")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": describe_workload(args.workload, ws), "fuse": "n/a (CPU oracle)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c5", "c5a", "c5b"])
+    ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
+    ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,245 @@
+"""GPU parity: the CUDA path, called through the C boundary, against the CPU oracle, bit for bit.
+
+Inputs are seeded and synthetic (paper_2112_01075_b200.workloads); source tiles and expected tiles
+come from the oracle only.  Comparison is bytewise (the random bf16/f32 patterns include NaNs).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2112_01075_b200 import api, workloads as wl
+from _plancheck import types_of
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+MODES = [api.FUSE_ADJACENT, api.FUSE_NONE, api.FUSE_ALL, api.NAIVE]
+MODE_NAMES = {0: "adjacent", 1: "unfused", 2: "all", 3: "naive"}
+
+
+def run_gpu(mesh, src, dst, e, src_tiles, flags=api.FUSE_ADJACENT, stream=None):
+    plan = api.Plan(mesh, src, dst, e, flags)
+    dev_src = [torch.from_numpy(np.ascontiguousarray(t)).cuda() for t in src_tiles]
+    nbytes = plan.local_elems(1) * e
+    dev_dst = [torch.full((nbytes,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+    scratch = plan.alloc_scratch()
+    if scratch is not None:
+        scratch.fill_(0xDD)
+    plan.execute(dev_src, dev_dst, scratch, stream)
+    torch.cuda.synchronize()
+    out = [t.cpu().numpy() for t in dev_dst]
+    return plan, out
+
+
+def assert_same(got, want, what=""):
+    assert len(got) == len(want)
+    for d, (g, w) in enumerate(zip(got, want)):
+        w = np.ascontiguousarray(w).reshape(-1)
+        if not np.array_equal(g, w):
+            bad = np.flatnonzero(g != w)
+            raise AssertionError(f"{what}: device {d}: {bad.size} of {w.size} bytes differ, first at {bad[0]}")
+
+
+def make_case(w, seed=None):
+    src, dst = types_of(w)
+    G = wl.global_array_bytes(w.src.global_shape, w.elem_bytes, w.fill, w.seed if seed is None else seed)
+    src_tiles = oracle.reslice(w.mesh_shape, src, G)
+    want = oracle.redistribute(w.mesh_shape, src, dst, src_tiles)
+    return src, dst, src_tiles, want
+
+
+# ---------------------------------------------------------------- sizes the oracle does in seconds
+
+MEDIUM = [
+    wl.config1(), wl.config1().reversed(),
+    wl.config2().scaled((8, 512, 1024)), wl.config2().reversed().scaled((8, 512, 1024)),
+    wl.config3("a").scaled((2048, 4096)), wl.config3("b").scaled((2048, 4096)), wl.config3("c").scaled((2048, 4096)),
+    wl.config5("a").scaled((4096, 2048)), wl.config5("b").scaled((4096, 4096)),
+    # ragged: tile rows that do not fill a work item, odd primes, run lengths that are not 16-byte multiples
+    wl.config3("a").scaled((8 * 37, 8 * 101)), wl.config3("c").scaled((24, 8 * 3)),
+    wl.config2().scaled((8, 8 * 13, 2 * 77)),
+]
+
+
+@pytest.mark.parametrize("w", MEDIUM, ids=lambda w: w.name + "_" + "x".join(map(str, w.src.global_shape)))
+@pytest.mark.parametrize("mode", MODES, ids=lambda m: MODE_NAMES[m])
+def test_configurations_at_medium_size(w, mode):
+    src, dst, src_tiles, want = make_case(w)
+    plan, got = run_gpu(w.mesh_shape, src, dst, w.elem_bytes, src_tiles, mode)
+    assert_same(got, want, w.name)
+    assert plan.height <= max(plan.local_elems(0), plan.local_elems(1))
+
+
+@pytest.mark.parametrize("mode", MODES, ids=lambda m: MODE_NAMES[m])
+def test_random_sweep_reduced_shape(mode):
+    """The 100 seeded (source, target) pairs of the random sweep on [16,32,64,128] f32 (16 MiB)."""
+    pairs = wl.config4(100, (16, 32, 64, 128))
+    G = wl.global_array_bytes((16, 32, 64, 128), 4, "random_bits", wl.CONFIG4_FILL_SEED)
+    for w in pairs:
+        src, dst = types_of(w)
+        src_tiles = oracle.reslice(w.mesh_shape, src, G)
+        want = oracle.reslice(w.mesh_shape, dst, G)
+        _, got = run_gpu(w.mesh_shape, src, dst, 4, src_tiles, mode)
+        assert_same(got, want, w.name + " " + w.src.notation(w.mesh_shape) + "->" + w.dst.notation(w.mesh_shape))
+
+
+def test_random_problems_small_and_odd():
+    """Odd primes, all element sizes, element-sized runs, several steps with scratch ping-pong."""
+    rng = np.random.default_rng(2112)
+    meshes = [(2, 3), (4, 6), (3, 3, 2), (2, 2, 2, 2), (6,), (5, 2)]
+    n_multi = 0
+    for t in range(120):
+        mesh = meshes[t % len(meshes)]
+        rank = int(rng.integers(1, 4))
+
+        def draw():
+            per = [[] for _ in range(rank)]
+            for a in range(len(mesh)):
+                c = int(rng.integers(0, rank + 1))
+                if c < rank:
+                    per[c].append(a)
+            return tuple(tuple(ax[i] for i in rng.permutation(len(ax))) if ax else () for ax in per)
+
+        a1, a2 = draw(), draw()
+        gshape = []
+        for k in range(rank):
+            f1 = int(np.prod([mesh[a] for a in a1[k]], dtype=np.int64))
+            f2 = int(np.prod([mesh[a] for a in a2[k]], dtype=np.int64))
+            gshape.append(int(np.lcm(f1, f2)) * int(rng.integers(1, 6)))
+        gshape = tuple(gshape)
+        e = int(rng.choice([1, 2, 4, 8, 16]))
+        G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+        src, dst = (gshape, a1), (gshape, a2)
+        src_tiles = oracle.reslice(mesh, src, G)
+        want = oracle.redistribute(mesh, src, dst, src_tiles)
+        mode = MODES[t % 4]
+        plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
+        n_multi += plan.num_launches >= 3
+        assert_same(got, want, f"{mesh} {src} -> {dst} e={e} mode={mode}")
+    assert n_multi > 0          # the two-slot scratch ping-pong was exercised
+
+
+def test_round_trip_on_the_gpu():
+    w = wl.config2().scaled((8, 256, 512))
+    src, dst, src_tiles, want = make_case(w)
+    _, mid = run_gpu(w.mesh_shape, src, dst, w.elem_bytes, src_tiles)
+    tile_dst, _ = oracle.base_offsets(w.mesh_shape, dst)
+    mid_tiles = [m.reshape(tile_dst + (w.elem_bytes,)) for m in mid]
+    _, back = run_gpu(w.mesh_shape, dst, src, w.elem_bytes, mid_tiles)
+    assert_same(back, src_tiles, "round trip")
+
+
+def test_identity_and_non_default_stream():
+    mesh = (2, 2)
+    t = ((64, 48), ((0,), (1,)))
+    G = wl.global_array_bytes((64, 48), 2, "random_bits", 5)
+    tiles = oracle.reslice(mesh, t, G)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        plan, got = run_gpu(mesh, t, t, 2, tiles, stream=s)
+    assert plan.launch_kernels() == ["copy"]
+    assert_same(got, tiles, "identity")
+
+
+def test_replicated_sources_may_alias():
+    """Replicas hold identical bytes, so the caller may pass one buffer for all of them."""
+    w = wl.config3("b").scaled((512, 256))
+    src, dst, src_tiles, want = make_case(w)
+    plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes)
+    one = torch.from_numpy(src_tiles[0]).cuda()
+    dev_dst = [torch.empty(plan.local_elems(1) * w.elem_bytes, dtype=torch.uint8, device="cuda") for _ in range(8)]
+    plan.execute([one] * 8, dev_dst)
+    torch.cuda.synchronize()
+    assert_same([t.cpu().numpy() for t in dev_dst], want, "aliased replicas")
+
+
+def test_host_buffers_entry_point():
+    w = wl.config3("a").scaled((1024, 2048))
+    src, dst, src_tiles, want = make_case(w)
+    plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes, api.FUSE_NONE)
+    n = plan.n_devices
+    hs = [torch.from_numpy(np.ascontiguousarray(t)).reshape(-1).pin_memory() for t in src_tiles]
+    hd = [torch.zeros(plan.local_elems(1) * w.elem_bytes, dtype=torch.uint8).pin_memory() for _ in range(n)]
+    dev_src = torch.empty(plan.staging_bytes(0), dtype=torch.uint8, device="cuda")
+    dev_dst = torch.empty(plan.staging_bytes(1), dtype=torch.uint8, device="cuda")
+    plan.execute_host(hs, hd, dev_src, dev_dst, plan.alloc_scratch())
+    torch.cuda.synchronize()
+    assert_same([t.numpy() for t in hd], want, "host entry point")
+
+
+def test_misuse_is_reported_not_executed():
+    w = wl.config3("a").scaled((64, 64))
+    src, dst, src_tiles, _ = make_case(w)
+    plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes)
+    nb = plan.local_elems(1) * w.elem_bytes
+    buf = torch.zeros(8 * nb + 64, dtype=torch.uint8, device="cuda")
+    dev_src = [torch.from_numpy(t).cuda() for t in src_tiles]
+    good = [buf[d * nb:(d + 1) * nb] for d in range(8)]
+    with pytest.raises(api.RedistError) as e:
+        plan.execute(dev_src, [buf[1 + d * nb:1 + (d + 1) * nb] for d in range(8)])
+    assert e.value.status == 7
+    with pytest.raises(api.RedistError) as e:
+        plan.execute(dev_src, [good[0]] * 8)
+    assert e.value.status == 6
+    with pytest.raises(api.RedistError) as e:
+        plan.execute(good, good)
+    assert e.value.status == 6
+    plan.execute(dev_src, good)
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------------------- full sizes
+
+FULL = ["c2", "c2_back", "c3a", "c3b", "c3c", "c5a", "c5b"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_configurations_at_full_size(name):
+    """Full benchmark sizes, default mode -- the launch configuration the benchmark times."""
+    w = wl.bench_workloads()[name]
+    oracle.set_threads(oracle.max_threads())
+    try:
+        src, dst, src_tiles, want = make_case(w)
+    finally:
+        oracle.set_threads(1)
+    plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes)
+    if name == "c3b":
+        # eight identical 512 MiB replicas: upload one, alias it (the oracle checked they agree)
+        one = torch.from_numpy(src_tiles[0]).cuda()
+        dev_src = [one] * plan.n_devices
+    else:
+        dev_src = [torch.from_numpy(t).cuda() for t in src_tiles]
+    nb = plan.local_elems(1) * w.elem_bytes
+    dev_dst = [torch.full((nb,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+    plan.execute(dev_src, dev_dst)
+    torch.cuda.synchronize()
+    for d in range(plan.n_devices):
+        got = dev_dst[d].cpu().numpy()
+        assert np.array_equal(got, want[d].reshape(-1)), f"{name}: device {d} differs"
+    assert plan.scratch_bytes == 0 and plan.height <= max(plan.local_elems(0), plan.local_elems(1))
+
+
+def test_random_sweep_full_size_samples():
+    """Three pairs of the sweep at the full [64,128,256,512] f32 shape (4 GiB global), chosen by
+    device footprint; all target tiles compared."""
+    pairs = wl.config4()
+    G = wl.global_array_bytes(wl.CONFIG4_SHAPE, 4, "random_bits", wl.CONFIG4_FILL_SEED)
+    oracle.set_threads(oracle.max_threads())
+    done = 0
+    try:
+        for w in pairs:
+            src, dst = types_of(w)
+            plan = api.Plan(w.mesh_shape, src, dst, 4)
+            foot = (plan.local_elems(0) + plan.local_elems(1)) * 4 * plan.n_devices
+            if foot > 12 * 2**30 or plan.num_steps < 2:
+                continue
+            src_tiles = oracle.reslice(w.mesh_shape, src, G)
+            want = oracle.reslice(w.mesh_shape, dst, G)
+            _, got = run_gpu(w.mesh_shape, src, dst, 4, src_tiles)
+            assert_same(got, want, w.name)
+            done += 1
+            if done == 3:
+                break
+    finally:
+        oracle.set_threads(1)
+    assert done == 3
