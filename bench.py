@@ -111,6 +111,21 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def reduce_max(dist, value: float, device: str = "cuda") -> float:
+    """Max over ranks of a per-rank duration (ranks run independent replicas)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(world: int, bytes_per_rank_step: int, max_ms_per_step: float) -> float:
+    """Whole-job GB/s: the bytes all ranks processed divided by the slowest rank's time."""
+    return world * bytes_per_rank_step / (max_ms_per_step * 1e-3) / 1e9
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -159,40 +174,64 @@ class DeviceLeg:
         self.scratch = p.alloc_scratch()
         self.eff_bytes = effective_bytes(w)
         self.launches = p.num_launches
-
-    def run(self, i, stream_ptr, src_override=None):
-        s = src_override if src_override is not None else self.src[i % len(self.src)]
-        d = self.dst[i % len(self.dst)]
         sp = self.scratch.data_ptr() if self.scratch is not None else 0
         sn = self.scratch.numel() if self.scratch is not None else 0
-        self.plan.execute_ptrs([t.data_ptr() for t in s], [t.data_ptr() for t in d], sp, sn, stream_ptr)
+        self.calls = [p.bind([t.data_ptr() for t in s], [t.data_ptr() for t in d], sp, sn)
+                      for s, d in zip(self.src, self.dst)]
+
+    def run(self, i, stream_ptr):
+        self.calls[i % len(self.calls)](stream_ptr)
 
 
-def time_legs(torch, legs, steps, warmup, per_launch=True):
-    """Run `steps` timed steps (after `warmup`), each step = every leg once.  Returns
-    (total_ms, per-leg list of launch durations in ms)."""
+def capture_graphs(torch, legs):
+    """One CUDA graph per buffer set; each holds one step (every leg's redist_execute once)."""
+    sets = len(legs[0].calls)
+    side = torch.cuda.Stream()
+    graphs = []
+    for i in range(sets):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for leg in legs:
+                leg.run(i, torch.cuda.current_stream().cuda_stream)
+        graphs.append(g)
+    return graphs
+
+
+def time_legs(torch, legs, steps, warmup, per_launch=False, graphs=None):
+    """Run `steps` timed steps (after `warmup`), each step = every leg once, bracketed by CUDA
+    events on the launching stream.  Returns (total_ms, per-leg launch durations in ms or None)."""
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
+
+    def one(i):
+        if graphs is not None:
+            graphs[i % len(graphs)].replay()
+        else:
+            for leg in legs:
+                leg.run(i, sp)
+
     for i in range(warmup):
-        for leg in legs:
-            leg.run(i, sp)
+        one(i)
     torch.cuda.synchronize()
-    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-          for _ in legs] if per_launch else None
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if not per_launch:
+        t0.record(stream)
+        for i in range(steps):
+            one(warmup + i)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1), None
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+          for _ in legs]
     t0.record(stream)
     for i in range(steps):
         for k, leg in enumerate(legs):
-            if per_launch:
-                ev[k][i][0].record(stream)
+            ev[k][i][0].record(stream)
             leg.run(warmup + i, sp)
-            if per_launch:
-                ev[k][i][1].record(stream)
+            ev[k][i][1].record(stream)
     t1.record(stream)
     torch.cuda.synchronize()
-    total = t0.elapsed_time(t1)
-    per = [[a.elapsed_time(b) for a, b in ev[k]] for k in range(len(legs))] if per_launch else None
-    return total, per
+    return t0.elapsed_time(t1), [[a.elapsed_time(b) for a, b in ev[k]] for k in range(len(legs))]
 
 
 def run_ours(args):
@@ -223,34 +262,43 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    graphs = None if args.no_graph else capture_graphs(torch, legs)
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
-    total_ms, per = time_legs(torch, legs, args.steps, args.warmup)
+    total_ms, _ = time_legs(torch, legs, args.steps, args.warmup, graphs=graphs)
     clocks = sampler.stop()
     barrier()
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = reduce_max(dist, total_ms)
     ms_per_step = total_ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = aggregate_value(world, step_bytes, ms_per_step)
 
-    # dominant kernel: the launch with the largest summed duration
+    # outside the headline region: the same steps launched plainly on the stream, with an event
+    # pair around every launch (per-leg numbers; the events themselves cost a few microseconds)
+    n_side = max(3, min(args.steps, 200))
+    plain_ms, _ = time_legs(torch, legs, n_side, 3)
+    _, per = time_legs(torch, legs, n_side, 3, per_launch=True)
+
+    # roofline of the dominant kernel.  When every launch of the step runs the same kernel on the
+    # same number of bytes (the default workload), its average duration is the timed region divided
+    # by the number of launches; otherwise the per-launch event pairs decide.
+    infos = [l.plan.launch_info(0) for l in legs]
+    n_launch = sum(l.launches for l in legs)
+    same = all(l.launches == 1 for l in legs) and len({(i.kernel, i.bytes_read + i.bytes_written) for i in infos}) == 1
     sums = [sum(p) for p in per]
     k = max(range(len(legs)), key=lambda q: sums[q])
-    dom = legs[k]
-    li = dom.plan.launch_info(0)
-    avg_ms = statistics.mean(per[k]) / dom.launches
-    peak, how = measured_peak()
+    dom, li = legs[k], infos[k]
     alg = li.bytes_read + li.bytes_written
+    avg_ms = (total_ms / (args.steps * n_launch)) if same else statistics.mean(per[k]) / dom.launches
+    peak, how = measured_peak()
     achieved = alg / (avg_ms * 1e-3) / 1e9
+    kname = {"naive_gather": "allgather", "naive_slice": "dynslice", "copy": "allpermute"}.get(
+        api.KERNELS[li.kernel], api.KERNELS[li.kernel])
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "traffic": ncu_traffic(args.workload),
-                "kernel": "redist_%s_kernel" % api.KERNELS[li.kernel].replace("naive_gather", "allgather")
-                .replace("naive_slice", "dynslice").replace("copy", "allpermute"),
-                "algorithmic_bytes_per_launch": alg, "avg_launch_us": round(avg_ms * 1e3, 2),
-                "median_launch_us": round(statistics.median(per[k]) * 1e3 / dom.launches, 2),
+                "kernel": f"redist_{kname}_kernel", "algorithmic_bytes_per_launch": alg,
+                "avg_launch_us": round(avg_ms * 1e3, 2),
+                "avg_from": "timed region / launches" if same else "event pair around each launch",
                 "peak_source": how + " copy bandwidth", "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)}
 
     line = {
@@ -258,6 +306,8 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": describe_workload(args.workload, ws), "fuse": args.fuse,
+                   "launch": "redist_execute on a stream" if args.no_graph else
+                   "CUDA graph replay of captured redist_execute calls (one graph per buffer set)",
                    "cache": f"{N_SETS} rotating buffer sets, no buffer re-read within 1 GiB of traffic",
                    "parallelism": "replicas only" if world > 1 else "single GPU, virtual devices"},
         "gpu_launches": args.steps * sum(l.launches for l in legs),
@@ -265,6 +315,9 @@ def run_ours(args):
         "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in legs),
         "memory_bound_bytes_per_virtual_device": max(max(l.plan.local_elems(0), l.plan.local_elems(1)) *
                                                      l.w.elem_bytes for l in legs),
+        "stream_launch": {"value": round(world * step_bytes / (plain_ms / n_side * 1e-3) / 1e9, 1), "unit": UNIT,
+                          "ms_per_step": round(plain_ms / n_side, 5), "steps": n_side,
+                          "note": "same steps, redist_execute called per launch without a graph"},
         "legs": [{"name": l.w.name, "steps": l.plan.step_kinds(), "kernels": l.plan.launch_kernels(),
                   "gbs": round(l.eff_bytes / (statistics.mean(per[q]) * 1e-3) / 1e9, 1),
                   "us": round(statistics.mean(per[q]) * 1e3, 2)} for q, l in enumerate(legs)],
@@ -326,10 +379,7 @@ def run_e2e(torch, api, ws, flags, steps, world, dist):
     t1.record(stream)
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1)
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = reduce_max(dist, ms)
     per_step = ms / steps
     return {"value": round(world * sum(l[6] for l in legs) / (per_step * 1e-3) / 1e9, 2), "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(per_step, 3), "steps": steps,
@@ -348,7 +398,7 @@ def run_others(torch, api, gen, args):
             try:
                 sets = 2 if name.startswith(("c3c", "c5")) else N_SETS
                 legs = [DeviceLeg(w, flags, torch, api, gen, sets=sets) for w in ws]
-                total, per = time_legs(torch, legs, 10, 3)
+                total, per = time_legs(torch, legs, 10, 3, per_launch=True)
                 eff = sum(l.eff_bytes for l in legs)
                 med = statistics.median([sum(per[q][i] for q in range(len(legs))) for i in range(10)])
                 out[f"{name}/{fuse}"] = {"gbs": round(eff / (med * 1e-3) / 1e9, 1), "us": round(med * 1e3, 2),
@@ -466,6 +516,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c5", "c5a", "c5b"])
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
     ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

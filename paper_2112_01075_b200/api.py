@@ -16,7 +16,7 @@ import os
 from typing import List, Optional, Sequence
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libredist_b200.so")
+LIB_PATH = os.environ.get("REDIST_LIB") or os.path.join(HERE, "libredist_b200.so")
 
 FUSE_ADJACENT, FUSE_NONE, FUSE_ALL, NAIVE = 0, 1, 2, 3
 NO_OVERPARTITION = 16
@@ -265,6 +265,22 @@ class Plan:
                                       ctypes.c_void_p(stream or None))
         if rc:
             raise RedistError(rc, "redist_execute")
+
+    def bind(self, src_ptrs: Sequence[int], dst_ptrs: Sequence[int], scratch_ptr: int = 0,
+             scratch_bytes: int = 0):
+        """Marshal the pointer tables once; the returned callable runs ``redist_execute`` on a stream
+        (``call(stream_ptr)``) with no per-call Python work beyond the foreign call itself."""
+        s = (ctypes.c_void_p * len(src_ptrs))(*src_ptrs)
+        d = (ctypes.c_void_p * len(dst_ptrs))(*dst_ptrs)
+        sp, sn, h, fn = ctypes.c_void_p(scratch_ptr or None), ctypes.c_size_t(scratch_bytes), self._h, \
+            self._lib.redist_execute
+
+        def call(stream_ptr: int = 0):
+            rc = fn(h, s, d, sp, sn, ctypes.c_void_p(stream_ptr or None))
+            if rc:
+                raise RedistError(rc, "redist_execute")
+
+        return call
 
     def execute(self, src_shards, dst_shards, scratch=None, stream=None) -> None:
         """``redist_execute`` on lists of CUDA tensors (one per virtual device), asynchronous."""

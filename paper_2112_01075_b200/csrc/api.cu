@@ -20,22 +20,21 @@ namespace {
 
 thread_local int tl_cuda_error = 0;
 
+// One thread block per work item by default: the hardware block scheduler balances the load and
+// keeps the tail to one item.  REDIST_GRID_MULT=k (tuning knob) switches to a grid-stride loop with
+// k blocks per SM.
 int grid_for(const CopyGeometry &g)
 {
-    static int sms = 0;
-    static int mult = 0;
-    if (sms == 0) {
+    static const long long cap = [] {
+        const char *m = std::getenv("REDIST_GRID_MULT");
+        if (!m || std::atoi(m) <= 0) return 0ll;
         int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            sms = n;
-        else
-            sms = 148;
-        const char *m = std::getenv("REDIST_GRID_MULT");   // CTAs per SM of the grid-stride loop (tuning)
-        mult = m ? std::max(1, std::atoi(m)) : 8;
-    }
-    const long long cap = 1ll * sms * mult;
-    return int(std::min<long long>(g.n_items, cap));
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+        return 1ll * n * std::atoi(m);
+    }();
+    return int(cap > 0 ? std::min<long long>(g.n_items, cap) : g.n_items);
 }
 
 struct Range {

@@ -3,6 +3,7 @@
 // of adjacent collectives -- merging of adjacent operations, Section 7.1, taken one step further:
 // on one GPU any run of steps composes into a single strided copy).
 #include <algorithm>
+#include <cstdlib>
 #include <numeric>
 
 #include "plan.hpp"
@@ -134,8 +135,19 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     G.lanes_div = make_div(uint32_t(lanes));
     G.rows_per_pass = uint32_t(kBlockThreads / lanes);
     G.rows = uint32_t(n_rows);
-    // a work item: about 32 KiB, a whole number of passes
-    const i64 kItemBytes = 32 * 1024;
+    // a work item: a whole number of passes, about 32 KiB read -- less when every byte read is
+    // stored to several replicas, so that the bytes written per block stay comparable
+    static const i64 kItemKb = [] {
+        const char *v = std::getenv("REDIST_ITEM_KB");   // tuning knob: KiB read per work item
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 0);
+    }();
+    i64 fan = 1;
+    if (!b.shared_global) {
+        i64 nt = 1;
+        for (int k = 0; k < r; ++k) nt *= b.ntiles[k];
+        fan = p.n_devices / nt;
+    }
+    const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
     i64 rpi = std::max<i64>(G.rows_per_pass, kItemBytes / (lanes * vec) / G.rows_per_pass * G.rows_per_pass);
     rpi = std::min<i64>(rpi, round_up(n_rows, G.rows_per_pass));
     G.rows_per_item = uint32_t(rpi);

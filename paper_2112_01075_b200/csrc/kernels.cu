@@ -22,7 +22,10 @@ namespace redist {
 
 namespace {
 
-constexpr int kUnroll = 4;
+#ifndef REDIST_UNROLL
+#define REDIST_UNROLL 4
+#endif
+constexpr int kUnroll = REDIST_UNROLL;
 
 __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv &f)
 {
