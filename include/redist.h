@@ -175,6 +175,33 @@ redist_status redist_execute_host(const redist_plan_t *plan, const void *const *
                                   void *dev_dst, size_t dev_dst_bytes, void *scratch,
                                   size_t scratch_bytes, void *cuda_stream);
 
+/*
+ * redist_execute_static -- redist_execute for callers that cannot supply scratch memory.
+ * (The paper has no counterpart: it is a property of this library, not of the method.)
+ *
+ * Some callers have tiles but no way to allocate: a plug-in inside a server that handed all device
+ * memory to a pool at start-up and forbids cudaMalloc afterwards, or a latency-bound path on which
+ * an allocation may fail or stall.  For them the ping-pong buffers of an unfused plan come from a
+ * fixed array of REDIST_STATIC_SCRATCH_BYTES bytes built into the library image (every GPU that
+ * loads the library holds those bytes until the process exits).  The call allocates nothing on
+ * the device or the host and calls no allocating routine.
+ *
+ *   plan            any plan with redist_plan_scratch_bytes(plan) <= REDIST_STATIC_SCRATCH_BYTES;
+ *                   a larger plan is refused with REDIST_ESCRATCH and nothing runs
+ *   src_shards[N], dst_shards[N], cuda_stream    exactly as for redist_execute
+ * Set-up: the first call on each device (with that device current) looks up the device address of
+ * the built-in array; make that first call before any stream capture begins.
+ * Sharing: all calls on a device use the same array.  It keeps whatever the previous call left;
+ * nothing in it has to start at zero, because every byte a step reads from it was written by an
+ * earlier step of the same call.  Two calls whose kernels may overlap on the GPU (different
+ * streams without an ordering between them) race on the array: order them.
+ * Errors: EINVAL, ESCRATCH (plan too large), EALIGN, EOVERLAP, EUNSUPPORTED (device index >= 64),
+ * ECUDA.  Results are identical to redist_execute with a caller-provided scratch buffer.
+ */
+#define REDIST_STATIC_SCRATCH_BYTES (8u << 20)
+redist_status redist_execute_static(const redist_plan_t *plan, const void *const *src_shards,
+                                    void *const *dst_shards, void *cuda_stream);
+
 /* ---- queries (host only) -------------------------------------------------------------------- */
 
 int32_t redist_plan_num_devices(const redist_plan_t *plan);               /* N                        */

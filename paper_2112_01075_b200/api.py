@@ -21,12 +21,13 @@ LIB_PATH = os.environ.get("REDIST_LIB") or os.path.join(HERE, "libredist_b200.so
 FUSE_ADJACENT, FUSE_NONE, FUSE_ALL, NAIVE = 0, 1, 2, 3
 NO_OVERPARTITION = 16
 MAX_RANK = 8
+STATIC_SCRATCH_BYTES = 8 << 20
 
 STEP_KINDS = ("dynslice", "alltoall", "allgather", "allpermute", "copy")
 KERNELS = ("dynslice", "alltoall", "allgather", "allpermute", "copy", "fused", "naive_gather", "naive_slice")
 
 EXPORTS = (
-    "redist_plan", "redist_plan_destroy", "redist_execute", "redist_execute_host",
+    "redist_plan", "redist_plan_destroy", "redist_execute", "redist_execute_host", "redist_execute_static",
     "redist_plan_num_devices", "redist_plan_rank", "redist_plan_local_elems", "redist_plan_scratch_bytes",
     "redist_plan_scratch_bytes_per_device", "redist_plan_staging_bytes", "redist_plan_alignment",
     "redist_plan_height", "redist_plan_cost", "redist_plan_num_steps", "redist_plan_num_launches",
@@ -82,6 +83,8 @@ def load() -> ctypes.CDLL:
     lib.redist_plan_destroy.restype = None
     lib.redist_execute.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, sz, vp]
     lib.redist_execute.restype = i32
+    lib.redist_execute_static.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
+    lib.redist_execute_static.restype = i32
     lib.redist_execute_host.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, sz, vp, sz, vp, sz, vp]
     lib.redist_execute_host.restype = i32
     for name, res in (("redist_plan_num_devices", i32), ("redist_plan_rank", i32),
@@ -298,6 +301,21 @@ class Plan:
         sn = scratch.numel() * scratch.element_size() if scratch is not None else 0
         self.execute_ptrs([t.data_ptr() for t in src_shards], [t.data_ptr() for t in dst_shards], sp, sn,
                           stream.cuda_stream)
+
+    def execute_static(self, src_shards, dst_shards, stream=None) -> None:
+        """``redist_execute_static``: like ``execute`` but the scratch of an unfused plan comes from
+        the fixed array built into the library, for callers that cannot allocate device memory
+        (plans needing more than ``STATIC_SCRATCH_BYTES`` are refused)."""
+        import torch
+
+        if stream is None:
+            stream = torch.cuda.current_stream()
+        n = self.n_devices
+        s = (ctypes.c_void_p * n)(*[t.data_ptr() for t in src_shards])
+        d = (ctypes.c_void_p * n)(*[t.data_ptr() for t in dst_shards])
+        rc = self._lib.redist_execute_static(self._h, s, d, ctypes.c_void_p(stream.cuda_stream or None))
+        if rc:
+            raise RedistError(rc, "redist_execute_static")
 
     def execute_host(self, src_host, dst_host, dev_src, dev_dst, scratch=None, stream=None) -> None:
         """``redist_execute_host``: host tiles in, host tiles out, staged through ``dev_src``/``dev_dst``."""

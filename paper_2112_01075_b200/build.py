@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libredist_b200.so")
-SOURCES = ["api.cu", "kernels.cu", "planner.cpp", "descriptor.cpp", "describe.cpp"]
+SOURCES = ["api.cu", "kernels.cu", "static_scratch.cu", "planner.cpp", "descriptor.cpp", "describe.cpp"]
 HEADERS = ["plan.hpp", "copy_params.h", "kernels.h"]
 
 

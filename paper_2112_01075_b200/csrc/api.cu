@@ -16,9 +16,11 @@ struct redist_plan_s {
 
 using namespace redist;
 
-namespace {
-
+namespace redist {
 thread_local int tl_cuda_error = 0;
+}
+
+namespace {
 
 // One thread block per work item by default: the hardware block scheduler balances the load and
 // keeps the tail to one item.  REDIST_GRID_MULT=k (tuning knob) switches to a grid-stride loop with

@@ -79,6 +79,9 @@ struct Plan {
     std::string json;
 };
 
+// api.cu: last CUDA error seen by the calling thread inside the library
+extern thread_local int tl_cuda_error;
+
 // planner.cpp
 redist_status synthesize(Plan &p);
 redist_status check_type(int n_axes, const i64 *mesh, const redist_type *t, std::vector<i64> *tile);

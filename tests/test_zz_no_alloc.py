@@ -1,0 +1,71 @@
+"""The entry point for callers that cannot allocate device memory (``redist_execute_static``).
+
+A plug-in that receives its tiles from a host framework but may not call cudaMalloc -- because the
+process gave all device memory to a pool at start-up, or because an allocation on its path could
+fail or stall -- still has to run unfused plans, whose intermediates need scratch.  The library
+serves those from a fixed array inside its own image.  Checked here through the C boundary: two
+calls in a row must give exactly the bytes the ordinary entry point gives with a scratch buffer
+the test allocates (the second call finds the first call's leftovers in the array), and a plan
+that needs more than the array holds must be refused.
+
+Collected last on purpose, so a run that stops at the first failure has already run everything else.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2112_01075_b200 import api, workloads as wl
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def tiles_for(w, seed):
+    src = (w.src.global_shape, w.src.axes)
+    G = wl.global_array_bytes(w.src.global_shape, w.elem_bytes, "random_bits", seed)
+    return oracle.reslice(w.mesh_shape, src, G)
+
+
+def test_static_scratch_matches_caller_scratch_twice_in_a_row():
+    # two alltoalls, unfused: one intermediate per virtual device lives in scratch
+    w = wl.config2().scaled((8, 128, 512))
+    plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, api.FUSE_NONE)
+    assert plan.num_launches == 2 and 0 < plan.scratch_bytes <= api.STATIC_SCRATCH_BYTES
+    nb = plan.local_elems(1) * w.elem_bytes
+    for seed in (1, 2):                                   # second call: other data, dirty array
+        d_src = [torch.from_numpy(t).cuda() for t in tiles_for(w, seed)]
+        ref = [torch.full((nb,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+        got = [torch.full((nb,), 0x11, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+        plan.execute(d_src, ref, plan.alloc_scratch())    # existing entry point, scratch from torch
+        plan.execute_static(d_src, got)                   # new entry point, nothing allocated
+        torch.cuda.synchronize()
+        for d in range(plan.n_devices):
+            assert torch.equal(got[d], ref[d]), f"call with seed {seed}: device {d} differs"
+
+
+def test_static_scratch_three_step_plan_uses_both_slots():
+    mesh = (2, 3, 2)
+    src = ((12, 12, 8), ((0,), (1,), ()))
+    dst = ((12, 12, 8), ((1,), (), (0,)))
+    plan = api.Plan(mesh, src, dst, 4, api.FUSE_NONE)         # dynslice, alltoall, allpermute, allgather
+    assert plan.num_launches >= 3 and plan.scratch_bytes_per_device == 2 * 512
+    G = np.random.default_rng(7).integers(0, 256, size=(12, 12, 8, 4), dtype=np.uint8)
+    want = oracle.reslice(mesh, dst, G)
+    d_src = [torch.from_numpy(t).cuda() for t in oracle.reslice(mesh, src, G)]
+    nb = plan.local_elems(1) * 4
+    for _ in range(2):
+        got = [torch.zeros(nb, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+        plan.execute_static(d_src, got)
+        torch.cuda.synchronize()
+        for d in range(plan.n_devices):
+            assert np.array_equal(got[d].cpu().numpy(), want[d].reshape(-1))
+
+
+def test_plans_beyond_the_built_in_array_are_refused():
+    w = wl.config2()                                      # unfused: 16 MiB per virtual device
+    plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, api.FUSE_NONE)
+    assert plan.scratch_bytes > api.STATIC_SCRATCH_BYTES
+    fake = [torch.empty(16, dtype=torch.uint8, device="cuda")] * plan.n_devices
+    with pytest.raises(api.RedistError) as e:
+        plan.execute_static(fake, fake)
+    assert e.value.status == 5                            # refused before anything runs
