@@ -418,6 +418,81 @@ def run_others(torch, api, gen, args):
     return out
 
 
+def run_sweep(args):
+    """Config 4: the 100 seeded random (source, target) pairs on f32 [64,128,256,512], mesh 2x4x2.
+    Every pair is planned, executed and timed on its own (global array 4 GiB, far above L2, so no
+    buffer rotation is needed); replicated source tiles share one buffer per distinct tile."""
+    import math
+    import torch
+    from paper_2112_01075_b200 import api, workloads as wl
+
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(wl.CONFIG4_FILL_SEED)
+    if args.workload == "c4":
+        pairs, label = wl.config4(), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
+    elif args.workload == "adv":
+        pairs, label = wl.adversarial_problems(), "adv: the %d problems of the paper's table of largest slow-downs"
+    else:
+        pairs, label = wl.evaluation_like_problems(args.pairs), \
+            "eval: %d random problems shaped like the paper's evaluation sample (3 mesh axes, <= 6-D, 64-800 MB)"
+    flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
+    G = None
+    stream = torch.cuda.current_stream()
+    rows = []
+    for w in pairs[: args.pairs]:
+        if G is None or tuple(G.shape[:-1]) != tuple(w.src.global_shape):
+            G = None
+            G = torch.randint(0, 256, tuple(w.src.global_shape) + (4,), dtype=torch.uint8, device="cuda",
+                              generator=gen)
+        plan = api.Plan(w.mesh_shape, w.src, w.dst, 4, flags)
+        _, offs = api.redist_base_offsets(w.mesh_shape, w.src)
+        tiles = api.shard_global(G, w.mesh_shape, w.src)
+        owned = {}
+        for d, o in enumerate(offs):
+            if o not in owned:
+                owned[o] = tiles[d].clone()
+        src = [owned[o] for o in offs]
+        del tiles
+        db = plan.local_elems(1) * 4
+        dst = [torch.empty(db, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+        scratch = plan.alloc_scratch()
+        call = plan.bind([t.data_ptr() for t in src], [t.data_ptr() for t in dst],
+                         scratch.data_ptr() if scratch is not None else 0,
+                         scratch.numel() if scratch is not None else 0)
+        for _ in range(2):
+            call(stream.cuda_stream)
+        reps = 5 if w.global_elems > 2**28 else 20
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(reps):
+            call(stream.cuda_stream)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / reps
+        eff = effective_bytes(w)
+        li = [plan.launch_info(q) for q in range(plan.num_launches)]
+        rows.append({"name": w.name, "src": w.src.notation(w.mesh_shape, w.axis_names),
+                     "dst": w.dst.notation(w.mesh_shape, w.axis_names), "steps": plan.step_kinds(),
+                     "launches": plan.num_launches, "run_bytes": min(i.run_bytes for i in li),
+                     "fanout": max(i.fanout for i in li), "eff_bytes": eff, "us": round(ms * 1e3, 1),
+                     "gbs": round(eff / (ms * 1e-3) / 1e9, 1),
+                     "scratch_per_device": plan.scratch_bytes_per_device})
+        del src, dst, owned, scratch, call, plan
+        torch.cuda.empty_cache()
+    g = [r["gbs"] for r in rows]
+    peak, how = measured_peak()
+    line = {"metric": METRIC, "workload": label % len(rows),
+            "fuse": args.fuse, "geomean_gbs": round(math.exp(sum(math.log(x) for x in g) / len(g)), 1),
+            "min_gbs": min(g), "max_gbs": max(g), "median_gbs": statistics.median(g),
+            "total_gbs": round(sum(r["eff_bytes"] for r in rows) / sum(r["us"] * 1e-6 for r in rows) / 1e9, 1),
+            "peak": peak, "peak_source": how, "pairs_below_70pct_of_peak": sum(x < 0.7 * peak for x in g)}
+    if args.dump:
+        with open(args.dump, "w") as f:
+            json.dump({"summary": line, "pairs": rows}, f, indent=1)
+    print(json.dumps(line), flush=True)
+
+
 # ------------------------------------------------------------------------------ CPU oracle arms
 
 def oracle_step_fn(ws, shrink=1):
@@ -513,7 +588,10 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c5", "c5a", "c5b"])
+    ap.add_argument("--workload", default="c2",
+                    choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval"])
+    ap.add_argument("--pairs", type=int, default=100, help="sweeps: how many problems to run")
+    ap.add_argument("--dump", default="", help="sweeps: write the per-problem table to this JSON file")
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
     ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
@@ -521,7 +599,11 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.workload in ("c4", "adv", "eval"):
+        if args.impl == "reference":
+            raise SystemExit("the sweeps (c4, adv, eval) are GPU-side measurements; use another workload for --impl reference")
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -211,3 +211,55 @@ def bench_workloads() -> Dict[str, Workload]:
     for k in "ab":
         w["c5" + k] = config5(k)
     return w
+
+
+def adversarial_problems() -> List[Workload]:
+    """The four problems of the paper's table of largest slow-downs (Section 8), printed there with
+    their axis sizes inline (three mesh axes a, b, c of size 2): 4-byte elements, 64-162 MB global
+    data, up to six dimensions, sizes that are not powers of two."""
+    mesh, names = (2, 2, 2), ("a", "b", "c")
+    a, b, c = 0, 1, 2
+    spec = [
+        ("P1", (360, 368, 320), [[], [c], []], [[c, a], [], [b]]),
+        ("P2", (80, 80, 72, 64), [[], [c], [], []], [[b], [], [c], []]),
+        ("P3", (296, 360, 312), [[], [], [c]], [[b, c], [a], []]),
+        ("P4", (16, 16, 16, 16, 16, 16), [[c], [], [], [a], [], [b]], [[], [], [], [], [], [a]]),
+    ]
+    return [Workload(n, mesh, names, 4, dist_type(g, s), dist_type(g, d), "random_bits", 2112010760 + i,
+                     "adversarial table") for i, (n, g, s, d) in enumerate(spec)]
+
+
+def evaluation_like_problems(n: int, seed: int = 2112010770) -> List[Workload]:
+    """Random problems in the shape of the paper's evaluation sample (Section 8): three mesh axes,
+    arrays of two to six dimensions holding 64 MB-800 MB of 4-byte elements, every axis either
+    replicated or partitioning one dimension.  Used for planner throughput (no data is created)."""
+    rng = np.random.default_rng(seed)
+    lo, hi = 16 * 2**20, 200 * 2**20                      # elements
+    out: List[Workload] = []
+    while len(out) < n:
+        mesh = tuple(int(rng.choice([2, 2, 2, 4])) for _ in range(3))
+        rank = int(rng.integers(2, 7))
+        shape = [1] * rank
+        src, dst = _draw_type(rng, mesh, shape), _draw_type(rng, mesh, shape)
+        need = []
+        for k in range(rank):
+            f1 = f2 = 1
+            for a in src.axes[k]:
+                f1 *= mesh[a]
+            for a in dst.axes[k]:
+                f2 *= mesh[a]
+            need.append(int(np.lcm(f1, f2)))
+        shape = [need[k] * int(rng.integers(1, 17)) for k in range(rank)]
+        k = int(np.argmax(shape))
+        rest = 1
+        for j in range(rank):
+            if j != k:
+                rest *= shape[j]
+        target = int(rng.integers(lo, hi))
+        shape[k] = need[k] * max(1, round(target / rest / need[k]))
+        total = rest * shape[k]
+        if not lo <= total <= hi:
+            continue
+        out.append(Workload(f"eval{len(out):04d}", mesh, ("a", "b", "c"), 4, dist_type(shape, src.axes),
+                            dist_type(shape, dst.axes), "random_bits", 0, "evaluation-like"))
+    return out

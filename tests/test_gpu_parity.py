@@ -219,6 +219,43 @@ def test_configurations_at_full_size(name):
     assert plan.scratch_bytes == 0 and plan.height <= max(plan.local_elems(0), plan.local_elems(1))
 
 
+@pytest.mark.parametrize("w", wl.adversarial_problems(), ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", [api.FUSE_ADJACENT, api.FUSE_NONE], ids=lambda m: MODE_NAMES[m])
+def test_adversarial_table_problems_full_size(w, mode):
+    """P1-P4 of the paper's table (rank 3-6, sizes that are not powers of two, 64-162 MB)."""
+    oracle.set_threads(oracle.max_threads())
+    try:
+        src, dst, src_tiles, want = make_case(w)
+    finally:
+        oracle.set_threads(1)
+    _, got = run_gpu(w.mesh_shape, src, dst, w.elem_bytes, src_tiles, mode)
+    assert_same(got, want, w.name)
+
+
+def test_evaluation_like_problems_reduced():
+    """Problems shaped like the paper's evaluation sample (up to 6-D, short trailing dimensions),
+    every dimension reduced to its sharding factor times a small multiple."""
+    rng = np.random.default_rng(77)
+    for k, w in enumerate(wl.evaluation_like_problems(60)):
+        shape = []
+        for d in range(w.src.rank):
+            need = 1
+            for ax in (w.src.axes[d], w.dst.axes[d]):
+                f = 1
+                for a in ax:
+                    f *= w.mesh_shape[a]
+                need = int(np.lcm(need, f))
+            shape.append(need * int(rng.integers(1, 5)))
+        ws = w.scaled(shape)
+        e = int(rng.choice([2, 4, 8]))
+        src, dst = types_of(ws)
+        G = rng.integers(0, 256, size=tuple(shape) + (e,), dtype=np.uint8)
+        src_tiles = oracle.reslice(ws.mesh_shape, src, G)
+        want = oracle.reslice(ws.mesh_shape, dst, G)
+        _, got = run_gpu(ws.mesh_shape, src, dst, e, src_tiles, MODES[k % 3])
+        assert_same(got, want, ws.name)
+
+
 def test_random_sweep_full_size_samples():
     """Three pairs of the sweep at the full [64,128,256,512] f32 shape (4 GiB global), chosen by
     device footprint; all target tiles compared."""
