@@ -83,7 +83,7 @@ def check_plan(mesh, src, dst, elem_bytes, flags=api.FUSE_ADJACENT, seed=0, simu
         assert plan.scratch_bytes_per_device == len(slots) * desc["slot_bytes"]
         # every intermediate that is materialised fits the bound
         for L in desc["launches"][:-1]:
-            assert L["dst_tile_bytes"] <= M * elem_bytes <= desc["slot_bytes"] + 255
+            assert L["dst_tile_bytes"] <= M * elem_bytes and L["dst_tile_bytes"] <= desc["slot_bytes"]
     if simulate_launches:
         got, counts = run_plan(desc, src_tiles)
         for d in range(n):

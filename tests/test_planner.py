@@ -116,7 +116,7 @@ def test_adversarial_table_problems(w):
     shapes, and the synthesized sequences avoid the full allgather the paper says its method never
     issues (they use dynslice / alltoall / allpermute, and for P4 allgathers within the bound)."""
     mib = {"P1": 162, "P2": 113, "P3": 127, "P4": 64}[w.name]
-    assert round(w.global_elems * 4 / 2**20) == mib
+    assert abs(w.global_elems * 4 / 2**20 - mib) <= 0.5          # printed sizes are rounded MiB
     p = api.Plan(w.mesh_shape, w.src, w.dst, 4)
     assert p.height <= max(p.local_elems(0), p.local_elems(1))
     if w.name != "P4":
