@@ -232,15 +232,18 @@ def adversarial_problems() -> List[Workload]:
 def evaluation_like_problems(n: int, seed: int = 2112010770) -> List[Workload]:
     """Random problems in the shape of the paper's evaluation sample (Section 8): three mesh axes,
     arrays of two to six dimensions holding 64 MB-800 MB of 4-byte elements, every axis either
-    replicated or partitioning one dimension.  Used for planner throughput (no data is created)."""
+    replicated or partitioning one dimension.  Dimension sizes are balanced around the geometric
+    mean of the array (within a factor of four), as in the four problems the paper prints
+    ([360,368,320], [80,80,72,64], [296,360,312], [16]*6), and need not be powers of two.
+    Used for planner throughput and for the odd-shape sweep."""
     rng = np.random.default_rng(seed)
     lo, hi = 16 * 2**20, 200 * 2**20                      # elements
     out: List[Workload] = []
     while len(out) < n:
         mesh = tuple(int(rng.choice([2, 2, 2, 4])) for _ in range(3))
         rank = int(rng.integers(2, 7))
-        shape = [1] * rank
-        src, dst = _draw_type(rng, mesh, shape), _draw_type(rng, mesh, shape)
+        unit = [1] * rank
+        src, dst = _draw_type(rng, mesh, unit), _draw_type(rng, mesh, unit)
         need = []
         for k in range(rank):
             f1 = f2 = 1
@@ -249,15 +252,15 @@ def evaluation_like_problems(n: int, seed: int = 2112010770) -> List[Workload]:
             for a in dst.axes[k]:
                 f2 *= mesh[a]
             need.append(int(np.lcm(f1, f2)))
-        shape = [need[k] * int(rng.integers(1, 17)) for k in range(rank)]
-        k = int(np.argmax(shape))
-        rest = 1
-        for j in range(rank):
-            if j != k:
-                rest *= shape[j]
-        target = int(rng.integers(lo, hi))
-        shape[k] = need[k] * max(1, round(target / rest / need[k]))
-        total = rest * shape[k]
+        target = float(rng.integers(lo, hi))
+        gm = target ** (1.0 / rank)
+        shape = []
+        for k in range(rank):
+            want = gm * 2.0 ** float(rng.uniform(-2.0, 2.0))
+            shape.append(need[k] * max(1, int(round(want / need[k]))))
+        total = 1
+        for v in shape:
+            total *= v
         if not lo <= total <= hi:
             continue
         out.append(Workload(f"eval{len(out):04d}", mesh, ("a", "b", "c"), 4, dist_type(shape, src.axes),
