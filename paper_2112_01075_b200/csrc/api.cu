@@ -245,7 +245,7 @@ redist_status redist_plan_launch_info(const redist_plan_t *plan, int32_t launch,
     o.first_step = L.first_step;
     o.n_steps = L.n_steps;
     o.kernel = L.kernel;
-    o.vector_bytes = int32_t(L.geo.vec_bytes);
+    o.vector_bytes = int32_t(L.geo.unit_bytes);
     o.run_bytes = L.run_bytes;
     o.bytes_read = L.bytes_read;
     o.bytes_written = L.bytes_written;

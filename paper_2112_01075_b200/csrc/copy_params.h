@@ -7,7 +7,18 @@
 // with more than one unit); q_k / m1_k is the source tile coordinate and q_k % m1_k the unit inside
 // the source tile (m1_k = source tile size / g_k), likewise m2_k for the target.  Inside a box both
 // sides are strided sub-arrays: "row digits" (outer to inner) with byte strides on either side and
-// an innermost contiguous run of `lanes` vectors.  A work item is a chunk of rows of one box.
+// an innermost contiguous run of run_bytes.  Runs are moved in 16-byte chunks aligned on the target
+// side; when not every address is a multiple of 16 (`aligned == 0`) the source chunk is assembled
+// from two aligned loads and the ragged head and tail of a run go in `unit_bytes` pieces.
+//
+// Work items, by `mode`:
+//   kModeRows   aligned runs of at most 256 chunks: a block covers rows_per_pass rows of `lanes`
+//               chunks per pass; an item is rows_per_item rows; every thread decodes its own rows.
+//   kModeChunks all other runs of at least 256 bytes: an item is rows_per_item rows times one column
+//               block of per_block chunks; the rows are decoded once into shared memory and all
+//               threads walk the (row, chunk) space with a flat index.
+//   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
+//               (row, piece of unit_bytes).
 #pragma once
 
 #include <cstdint>
@@ -15,8 +26,10 @@
 namespace redist {
 
 constexpr int kMaxUnitDigits = 8;
-constexpr int kMaxRowDigits = 10;
+constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
+constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
+constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2;
 
 // Division of a 31-bit unsigned number by a constant: n / d == umulhi(n, mul) >> shr (d > 1).
 struct FastDiv {
@@ -27,12 +40,18 @@ struct CopyGeometry {
     uint32_t n_unit;                 // unit digits (dimensions with more than one box)
     uint32_t n_row;                  // row digits
     uint32_t fanout;                 // target replicas per box
-    uint32_t vec_bytes;              // bytes per memory access: 16, 8, 4, 2 or 1
-    uint32_t lanes;                  // vectors per run, 1..kBlockThreads
-    uint32_t rows_per_pass;          // kBlockThreads / lanes
+    uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
+    uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
+    uint32_t mode;                   // kModeRows, kModeChunks or kModeUnits
+    uint64_t run_bytes;              // contiguous run
+    uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
+    uint32_t rows_per_pass;          // kModeRows: kBlockThreads / lanes
     uint32_t rows;                   // rows per box
-    uint32_t rows_per_item;          // multiple of rows_per_pass
+    uint32_t rows_per_item;          // kModeRows: multiple of rows_per_pass; else <= kMaxRowsFlat
+    uint32_t per_block;              // flat walk: chunks (or units) of one row in a column block
     uint32_t n_items;
+    FastDiv per_block_div;           // flat walk: division by per_block
+    FastDiv col_blocks;              // flat walk: column blocks per row (1 in kModeRows)
     FastDiv items_per_box;
     FastDiv lanes_div;
     FastDiv unit_n[kMaxUnitDigits];  // boxes along the digit

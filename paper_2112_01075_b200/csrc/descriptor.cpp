@@ -108,17 +108,6 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         fit(d.b2);
     }
     const i64 vec = align;
-    i64 run_vecs = run_bytes / vec;
-    i64 lanes = run_vecs;
-    if (run_vecs > kBlockThreads) {
-        lanes = 1;
-        for (i64 c = kBlockThreads; c >= 1; --c)
-            if (run_vecs % c == 0) {
-                lanes = c;
-                break;
-            }
-        rows.push_back(RowDigit{run_vecs / lanes, lanes * vec, lanes * vec});
-    }
     if (rows.size() > size_t(kMaxRowDigits)) return REDIST_EUNSUPPORTED;
     i64 n_rows = 1;
     for (size_t q = 0; q < rows.size(); ++q) {
@@ -130,13 +119,12 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         if (n_rows >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     }
     G.n_row = uint32_t(rows.size());
-    G.vec_bytes = uint32_t(vec);
-    G.lanes = uint32_t(lanes);
-    G.lanes_div = make_div(uint32_t(lanes));
-    G.rows_per_pass = uint32_t(kBlockThreads / lanes);
+    G.unit_bytes = uint32_t(vec);
+    G.aligned = vec == 16 ? 1u : 0u;
+    G.run_bytes = uint64_t(run_bytes);
     G.rows = uint32_t(n_rows);
-    // a work item: a whole number of passes, about 32 KiB read -- less when every byte read is
-    // stored to several replicas, so that the bytes written per block stay comparable
+    // work items: about 32 KiB read each -- less when every byte read is stored to several
+    // replicas, so that the bytes written per block stay comparable
     static const i64 kItemKb = [] {
         const char *v = std::getenv("REDIST_ITEM_KB");   // tuning knob: KiB read per work item
         return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 0);
@@ -148,12 +136,42 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         fan = p.n_devices / nt;
     }
     const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
-    i64 rpi = std::max<i64>(G.rows_per_pass, kItemBytes / (lanes * vec) / G.rows_per_pass * G.rows_per_pass);
-    rpi = std::min<i64>(rpi, round_up(n_rows, G.rows_per_pass));
-    G.rows_per_item = uint32_t(rpi);
-    const i64 ipb = (n_rows + rpi - 1) / rpi;
+    const i64 max_chunks = run_bytes / 16;           // whole 16-byte chunks a run can hold
+    if (max_chunks >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+    i64 ipb;
+    G.lanes = kBlockThreads;
+    G.rows_per_pass = 1;
+    if (G.aligned && max_chunks <= kBlockThreads) {
+        // aligned short runs: `lanes` threads per row, one chunk each
+        const i64 lanes = max_chunks;
+        G.mode = kModeRows;
+        G.lanes = uint32_t(lanes);
+        G.rows_per_pass = uint32_t(kBlockThreads / lanes);
+        i64 rpi = std::max<i64>(G.rows_per_pass, kItemBytes / run_bytes / G.rows_per_pass * G.rows_per_pass);
+        rpi = std::min<i64>(rpi, round_up(n_rows, G.rows_per_pass));
+        G.rows_per_item = uint32_t(rpi);
+        G.per_block = uint32_t(max_chunks);
+        G.col_blocks = make_div(1);
+        ipb = (n_rows + rpi - 1) / rpi;
+    } else {
+        // flat walk over (row, chunk) -- or over (row, unit piece) for short ragged runs
+        const bool units = run_bytes < 256;
+        const i64 per_row = units ? run_bytes / vec : max_chunks;
+        const i64 piece = units ? vec : 16;
+        const i64 cpb = std::max<i64>(1, std::min<i64>(per_row, kItemBytes / piece));
+        const i64 ncb = std::max<i64>(1, (per_row + cpb - 1) / cpb);
+        i64 rpi = std::max<i64>(1, std::min<i64>(kMaxRowsFlat, kItemBytes / (cpb * piece)));
+        rpi = std::min<i64>(rpi, n_rows);
+        G.mode = units ? kModeUnits : kModeChunks;
+        G.rows_per_item = uint32_t(rpi);
+        G.per_block = uint32_t(cpb);
+        G.col_blocks = make_div(uint32_t(ncb));
+        ipb = (n_rows + rpi - 1) / rpi * ncb;
+    }
+    G.per_block_div = make_div(G.per_block);
+    G.lanes_div = make_div(G.lanes);
+    if (ipb >= (1ll << 31) || n_boxes * ipb >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     G.items_per_box = make_div(uint32_t(ipb));
-    if (n_boxes * ipb >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     G.n_items = uint32_t(n_boxes * ipb);
 
     // tables
@@ -288,8 +306,7 @@ redist_status build_launches(Plan &p)
         p.scratch_per_device = nslots * p.slot_bytes;
         p.scratch_bytes = p.scratch_per_device * p.n_devices;
     }
-    p.alignment = 1;
-    for (const Launch &L : p.launches) p.alignment = std::max<int>(p.alignment, int(L.geo.vec_bytes));
+    p.alignment = 16;   // every tile and scratch pointer; offsets inside a tile may be finer
     return REDIST_OK;
 }
 

@@ -4,15 +4,25 @@
 // meaning of a collective is how it changes the placement of tiles).  On one GPU, with every
 // virtual device's tile in its own buffer, a collective -- or a fused run of them -- is therefore a
 // strided gather/scatter between two layouts of the same global array, described by CopyGeometry
-// (copy_params.h).  The work is bound by HBM bandwidth: every source byte is read once, with the
-// widest access the strides allow (16 bytes in all benchmark shapes), and written once per target
-// replica from registers (allgather stores the same registers `fanout` times instead of re-reading).
+// (copy_params.h).  The work is bound by HBM bandwidth: every source byte is read once and written
+// once per target replica from registers (allgather stores the same registers `fanout` times
+// instead of re-reading).
 //
-// Thread mapping: a block of 256 threads covers rows_per_pass rows of `lanes` vectors; a thread
-// keeps its column and walks down the rows of its work item, issuing kUnroll independent loads
-// before the matching stores.  All index decoding uses multiply-shift division by constants that
-// the host precomputed; the per-item decode (box -> tiles and base offsets) is amortised over
-// ~32 KiB of data.
+// A contiguous run is moved in 16-byte chunks that are aligned on the *target* side, so stores are
+// always full 16-byte vectors.  When run length and offsets are multiples of 16 (ALIGNED) the source
+// chunk is one aligned load.  Otherwise (odd shapes) the source chunk is assembled from the two
+// aligned 16-byte blocks that contain it (byte funnel shift), and the few bytes before the first and
+// after the last target-aligned chunk of a run are copied in `unit_bytes` pieces.  Loads only ever
+// touch 16-byte blocks that hold at least one byte of the tile.
+//
+// Three item shapes (CopyGeometry::mode).  kModeRows, aligned runs of at most 4 KiB: a block of 256
+// threads covers rows_per_pass rows of `lanes` chunks; a thread keeps its column and walks down the
+// rows of its work item, kUnroll independent loads in flight before the stores.  kModeChunks, all
+// other runs of 256 bytes or more: the rows of an item are decoded once into shared memory and all
+// threads walk the (row, chunk) space of the item with a flat index.  kModeUnits, ragged runs below
+// 256 bytes: the same flat walk over (row, piece of unit_bytes).  Index decoding uses multiply-shift
+// division by host-computed constants; the per-item decode (box -> tiles and base offsets) is
+// amortised over ~32 KiB of data.
 #include <cuda_runtime.h>
 
 #include "copy_params.h"
@@ -32,102 +42,333 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv &f)
     return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
 }
 
-template <int VEC> struct VecType;
-template <> struct VecType<16> { using T = uint4; };
-template <> struct VecType<8> { using T = uint2; };
-template <> struct VecType<4> { using T = uint32_t; };
-template <> struct VecType<2> { using T = uint16_t; };
-template <> struct VecType<1> { using T = uint8_t; };
-
-// streaming accesses: the data is touched once (cache-streaming loads and stores)
+// streaming accesses: the data is touched once
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
-__device__ __forceinline__ uint2 ld_stream(const uint2 *p) { return __ldcs(p); }
-__device__ __forceinline__ uint32_t ld_stream(const uint32_t *p) { return __ldcs(p); }
-__device__ __forceinline__ uint16_t ld_stream(const uint16_t *p) { return __ldcs(p); }
-__device__ __forceinline__ uint8_t ld_stream(const uint8_t *p) { return __ldcs(p); }
-
 __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) { __stcs(p, v); }
-__device__ __forceinline__ void st_stream(uint2 *p, const uint2 &v) { __stcs(p, v); }
-__device__ __forceinline__ void st_stream(uint32_t *p, uint32_t v) { __stcs(p, v); }
-__device__ __forceinline__ void st_stream(uint16_t *p, uint16_t v) { __stcs(p, v); }
-__device__ __forceinline__ void st_stream(uint8_t *p, uint8_t v) { __stcs(p, v); }
 
-template <int VEC, int NT>
-__device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
+// 16 bytes starting at an arbitrary address: the aligned block that holds the first byte and, when
+// the address is not a multiple of 16, the next one (which then holds the last byte).
+__device__ __forceinline__ uint4 ld_shifted(const char *src)
 {
-    using T = typename VecType<VEC>::T;
+    const uint32_t m = uint32_t(reinterpret_cast<uintptr_t>(src)) & 15u;
+    const uint4 *p = reinterpret_cast<const uint4 *>(src - m);
+    const uint4 a = __ldg(p);
+    if (m == 0) return a;
+    const uint4 b = __ldg(p + 1);
+    const uint32_t bs = (m & 3u) * 8u;
+    uint4 o;
+    switch (m >> 2) {
+    case 0:
+        o.x = __funnelshift_r(a.x, a.y, bs); o.y = __funnelshift_r(a.y, a.z, bs);
+        o.z = __funnelshift_r(a.z, a.w, bs); o.w = __funnelshift_r(a.w, b.x, bs);
+        break;
+    case 1:
+        o.x = __funnelshift_r(a.y, a.z, bs); o.y = __funnelshift_r(a.z, a.w, bs);
+        o.z = __funnelshift_r(a.w, b.x, bs); o.w = __funnelshift_r(b.x, b.y, bs);
+        break;
+    case 2:
+        o.x = __funnelshift_r(a.z, a.w, bs); o.y = __funnelshift_r(a.w, b.x, bs);
+        o.z = __funnelshift_r(b.x, b.y, bs); o.w = __funnelshift_r(b.y, b.z, bs);
+        break;
+    default:
+        o.x = __funnelshift_r(a.w, b.x, bs); o.y = __funnelshift_r(b.x, b.y, bs);
+        o.z = __funnelshift_r(b.y, b.z, bs); o.w = __funnelshift_r(b.z, b.w, bs);
+        break;
+    }
+    return o;
+}
+
+// Copy `count` pieces of `unit` bytes (unit = 1, 2, 4 or 8; all addresses are multiples of it) from
+// src to every target replica; pieces are dealt to threads first, first + step, ...
+__device__ __forceinline__ void copy_units(char *const *dtab, uint32_t fanout, int64_t doff, const char *src,
+                                           uint32_t count, uint32_t unit, uint32_t first, uint32_t step)
+{
+    for (uint32_t u = first; u < count; u += step) {
+        const int64_t off = int64_t(u) * unit;
+        switch (unit) {
+        case 8: {
+            const uint2 v = *reinterpret_cast<const uint2 *>(src + off);
+            for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint2 *>(dtab[f] + doff + off) = v;
+            break;
+        }
+        case 4: {
+            const uint32_t v = *reinterpret_cast<const uint32_t *>(src + off);
+            for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint32_t *>(dtab[f] + doff + off) = v;
+            break;
+        }
+        case 2: {
+            const uint16_t v = *reinterpret_cast<const uint16_t *>(src + off);
+            for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint16_t *>(dtab[f] + doff + off) = v;
+            break;
+        }
+        default: {
+            const uint8_t v = *reinterpret_cast<const uint8_t *>(src + off);
+            for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint8_t *>(dtab[f] + doff + off) = v;
+            break;
+        }
+        }
+    }
+}
+
+// row number inside a box -> byte offsets of the row on the source and target side
+__device__ __forceinline__ void row_offsets(const CopyGeometry &g, uint32_t row, int64_t &s1, int64_t &s2)
+{
+    s1 = 0;
+    s2 = 0;
+    const int n_row = int(g.n_row);
+    uint32_t r = row;
+    for (int q = n_row - 1; q > 0; --q) {
+        const uint32_t nxt = fdiv(r, g.row_n[q]);
+        const uint32_t dg = r - nxt * g.row_n[q].d;
+        r = nxt;
+        s1 += int64_t(dg) * g.row_b1[q];
+        s2 += int64_t(dg) * g.row_b2[q];
+    }
+    if (n_row > 0) {
+        s1 += int64_t(r) * g.row_b1[0];
+        s2 += int64_t(r) * g.row_b2[0];
+    }
+}
+
+// head bytes before the first target-aligned chunk and number of whole chunks of a run
+__device__ __forceinline__ void split_run(uint64_t len, int64_t dst_off, uint32_t &head, uint32_t &chunks)
+{
+    const uint32_t h = (16u - (uint32_t(dst_off) & 15u)) & 15u;
+    head = uint64_t(h) < len ? h : uint32_t(len);
+    chunks = uint32_t((len - head) >> 4);
+}
+
+struct RowEntry {
+    int64_t s1, s2;
+};
+
+struct BoxBase {
+    const char *sbase;       // source tile base + offset of the box
+    char *const *dtab;       // target replica base pointers
+    int64_t o2;              // offset of the box inside the target tile
+    uint32_t part;           // item number inside the box
+};
+
+template <int NT>
+__device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t item)
+{
+    const CopyGeometry &g = P.g;
+    const uint32_t box = fdiv(item, g.items_per_box);
+    uint32_t t1 = 0, t2 = 0, rem = box;
+    int64_t o1 = 0, o2 = 0;
+    for (int u = int(g.n_unit) - 1; u >= 0; --u) {
+        const uint32_t nxt = fdiv(rem, g.unit_n[u]);
+        const uint32_t q = rem - nxt * g.unit_n[u].d;
+        rem = nxt;
+        const uint32_t a1 = fdiv(q, g.unit_m1[u]);
+        const uint32_t a2 = fdiv(q, g.unit_m2[u]);
+        t1 += a1 * g.unit_ts1[u];
+        t2 += a2 * g.unit_ts2[u];
+        o1 += int64_t(q - a1 * g.unit_m1[u].d) * g.unit_b1[u];
+        o2 += int64_t(q - a2 * g.unit_m2[u].d) * g.unit_b2[u];
+    }
+    BoxBase b;
+    b.sbase = P.src[t1] + o1;
+    b.dtab = &P.dst[t2 * g.fanout];
+    b.o2 = o2;
+    b.part = item - box * g.items_per_box.d;
+    return b;
+}
+
+// ---- kModeRows: thread (ty, tx) handles chunk tx of rows ty, ty + rows_per_pass, ... ------------
+template <int NT>
+__device__ __forceinline__ void rows_body(const CopyParams<NT> &P)
+{
     const CopyGeometry &g = P.g;
     const uint32_t tid = threadIdx.x;
-    const uint32_t ty = fdiv(tid, g.lanes_div);
-    const uint32_t tx = tid - ty * g.lanes;
-    const bool active = ty < g.rows_per_pass;
-    const uint32_t rpp = g.rows_per_pass;
     const uint32_t fanout = g.fanout;
-    const int n_row = int(g.n_row);
-
+    const uint32_t lanes = g.lanes;
+    const uint32_t ty = fdiv(tid, g.lanes_div);
+    const uint32_t tx = tid - ty * lanes;
+    const uint32_t rpp = g.rows_per_pass;
+    const bool active = ty < rpp;
     for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
-        const uint32_t box = fdiv(item, g.items_per_box);
-        const uint32_t chunk = item - box * g.items_per_box.d;
-        // box -> source tile / target tile and the byte offsets of the box inside them
-        uint32_t t1 = 0, t2 = 0, rem = box;
-        int64_t o1 = 0, o2 = 0;
-        for (int u = int(g.n_unit) - 1; u >= 0; --u) {
-            const uint32_t nxt = fdiv(rem, g.unit_n[u]);
-            const uint32_t q = rem - nxt * g.unit_n[u].d;
-            rem = nxt;
-            const uint32_t a1 = fdiv(q, g.unit_m1[u]);
-            const uint32_t a2 = fdiv(q, g.unit_m2[u]);
-            t1 += a1 * g.unit_ts1[u];
-            t2 += a2 * g.unit_ts2[u];
-            o1 += int64_t(q - a1 * g.unit_m1[u].d) * g.unit_b1[u];
-            o2 += int64_t(q - a2 * g.unit_m2[u].d) * g.unit_b2[u];
-        }
-        const char *sbase = P.src[t1] + o1 + int64_t(tx) * VEC;
-        const int64_t dcol = o2 + int64_t(tx) * VEC;
-        char *const *dtab = &P.dst[t2 * fanout];
-        const uint32_t row0 = chunk * g.rows_per_item;
+        const BoxBase b = decode_box(P, item);
+        const char *sb = b.sbase + int64_t(tx) * 16;
+        const int64_t dcol = b.o2 + int64_t(tx) * 16;
+        const uint32_t row0 = b.part * g.rows_per_item;
         const uint32_t row_end = min(row0 + g.rows_per_item, g.rows);
-
         for (uint32_t rb = row0; rb < row_end; rb += rpp * kUnroll) {
-            T v[kUnroll];
+            uint4 v[kUnroll];
             int64_t d2[kUnroll];
             bool ok[kUnroll];
 #pragma unroll
             for (int k = 0; k < kUnroll; ++k) {
                 const uint32_t row = rb + k * rpp + ty;
+                int64_t s1, s2;
+                row_offsets(g, row, s1, s2);
                 ok[k] = active && row < row_end;
-                int64_t s1 = 0, s2 = 0;
-                uint32_t r = row;
-                for (int q = n_row - 1; q > 0; --q) {
-                    const uint32_t nxt = fdiv(r, g.row_n[q]);
-                    const uint32_t dg = r - nxt * g.row_n[q].d;
-                    r = nxt;
-                    s1 += int64_t(dg) * g.row_b1[q];
-                    s2 += int64_t(dg) * g.row_b2[q];
-                }
-                if (n_row > 0) {
-                    s1 += int64_t(r) * g.row_b1[0];
-                    s2 += int64_t(r) * g.row_b2[0];
-                }
-                d2[k] = s2;
-                if (ok[k]) v[k] = ld_stream(reinterpret_cast<const T *>(sbase + s1));
+                d2[k] = dcol + s2;
+                if (ok[k]) v[k] = ld_stream(reinterpret_cast<const uint4 *>(sb + s1));
             }
             for (uint32_t f = 0; f < fanout; ++f) {
-                char *dbase = dtab[f] + dcol;
+                char *dbase = b.dtab[f];
 #pragma unroll
                 for (int k = 0; k < kUnroll; ++k)
-                    if (ok[k]) st_stream(reinterpret_cast<T *>(dbase + d2[k]), v[k]);
+                    if (ok[k]) st_stream(reinterpret_cast<uint4 *>(dbase + d2[k]), v[k]);
             }
         }
     }
 }
 
+// rows of the item -> shared table (decoded once, by the first threads)
+__device__ __forceinline__ uint32_t fill_rowtab(const CopyGeometry &g, RowEntry *rowtab, uint32_t group)
+{
+    const uint32_t row0 = group * g.rows_per_item;
+    const uint32_t nr = min(g.rows_per_item, g.rows - row0);
+    __syncthreads();
+    for (uint32_t r = threadIdx.x; r < nr; r += kBlockThreads) {
+        RowEntry e;
+        row_offsets(g, row0 + r, e.s1, e.s2);
+        rowtab[r] = e;
+    }
+    __syncthreads();
+    return nr;
+}
+
+// ---- kModeChunks: flat walk over (row, 16-byte chunk) ------------------------------------------
+template <bool ALIGNED, int NT>
+__device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *rowtab)
+{
+    const CopyGeometry &g = P.g;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t fanout = g.fanout;
+    const uint64_t len = g.run_bytes;
+    const uint32_t cpb = g.per_block;
+    for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
+        const BoxBase b = decode_box(P, item);
+        const uint32_t group = fdiv(b.part, g.col_blocks);
+        const uint32_t cb = b.part - group * g.col_blocks.d;
+        const uint32_t nr = fill_rowtab(g, rowtab, group);
+        const uint32_t total = nr * cpb;
+        const uint32_t c0 = cb * cpb;
+        for (uint32_t base = tid; base < total; base += kBlockThreads * kUnroll) {
+            uint4 v[kUnroll];
+            int64_t d2[kUnroll];
+            bool ok[kUnroll];
+#pragma unroll
+            for (int k = 0; k < kUnroll; ++k) {
+                const uint32_t idx = base + k * kBlockThreads;
+                const uint32_t r = fdiv(idx, g.per_block_div);
+                const uint32_t j = c0 + (idx - r * cpb);
+                const RowEntry e = rowtab[r < nr ? r : 0];
+                uint32_t head = 0, chunks = uint32_t(len >> 4);
+                if (!ALIGNED) split_run(len, b.o2 + e.s2, head, chunks);
+                ok[k] = idx < total && j < chunks;
+                const int64_t col = int64_t(head) + (int64_t(j) << 4);
+                d2[k] = b.o2 + e.s2 + col;
+                if (ok[k]) {
+                    if (ALIGNED)
+                        v[k] = ld_stream(reinterpret_cast<const uint4 *>(b.sbase + e.s1 + col));
+                    else
+                        v[k] = ld_shifted(b.sbase + e.s1 + col);
+                }
+            }
+            for (uint32_t f = 0; f < fanout; ++f) {
+                char *dbase = b.dtab[f];
+#pragma unroll
+                for (int k = 0; k < kUnroll; ++k)
+                    if (ok[k]) st_stream(reinterpret_cast<uint4 *>(dbase + d2[k]), v[k]);
+            }
+        }
+        if (!ALIGNED) {
+            // ragged ends: the bytes before the first target-aligned chunk belong to the first column
+            // block, those after the last whole chunk to the last; flat walk over (row, slot)
+            const uint32_t unit = g.unit_bytes;
+            const uint32_t slots = 16u / unit - 1u;          // at most 15 bytes on either end
+            const bool first = cb == 0, last = cb + 1 == g.col_blocks.d;
+            const uint32_t ends = (first ? 1u : 0u) + (last ? 1u : 0u);
+            for (uint32_t idx = tid; idx < nr * slots * ends; idx += kBlockThreads) {
+                const uint32_t r = idx / (slots * ends);
+                const uint32_t w = idx - r * (slots * ends);
+                const bool is_head = first && w < slots;
+                const uint32_t slot = is_head ? w : (first ? w - slots : w);
+                const RowEntry e = rowtab[r];
+                uint32_t head, chunks;
+                split_run(len, b.o2 + e.s2, head, chunks);
+                const int64_t toff = int64_t(head) + (int64_t(chunks) << 4);
+                const uint32_t count = is_head ? head / unit : uint32_t(len - uint64_t(toff)) / unit;
+                const int64_t off = is_head ? 0 : toff;
+                if (slot < count)
+                    copy_units(b.dtab, fanout, b.o2 + e.s2 + off, b.sbase + e.s1 + off, slot + 1, unit, slot, slots + 1);
+            }
+        }
+    }
+}
+
+// ---- kModeUnits: flat walk over (row, piece of UNIT bytes) -------------------------------------
+template <typename T, int NT>
+__device__ __forceinline__ void units_walk(const CopyParams<NT> &P, RowEntry *rowtab)
+{
+    constexpr int kU = 2 * kUnroll;
+    const CopyGeometry &g = P.g;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t fanout = g.fanout;
+    const uint32_t upr = g.per_block;                 // pieces per row (the whole run)
+    for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
+        const BoxBase b = decode_box(P, item);
+        const uint32_t nr = fill_rowtab(g, rowtab, b.part);
+        const uint32_t total = nr * upr;
+        for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
+            T v[kU];
+            int64_t d2[kU];
+            bool ok[kU];
+#pragma unroll
+            for (int k = 0; k < kU; ++k) {
+                const uint32_t idx = base + k * kBlockThreads;
+                const uint32_t r = fdiv(idx, g.per_block_div);
+                const uint32_t u = idx - r * upr;
+                const RowEntry e = rowtab[r < nr ? r : 0];
+                ok[k] = idx < total;
+                d2[k] = b.o2 + e.s2 + int64_t(u) * sizeof(T);
+                if (ok[k]) v[k] = __ldg(reinterpret_cast<const T *>(b.sbase + e.s1 + int64_t(u) * sizeof(T)));
+            }
+            for (uint32_t f = 0; f < fanout; ++f) {
+                char *dbase = b.dtab[f];
+#pragma unroll
+                for (int k = 0; k < kU; ++k)
+                    if (ok[k]) *reinterpret_cast<T *>(dbase + d2[k]) = v[k];
+            }
+        }
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ void units_body(const CopyParams<NT> &P, RowEntry *rowtab)
+{
+    switch (P.g.unit_bytes) {
+    case 8: units_walk<uint2, NT>(P, rowtab); break;
+    case 4: units_walk<uint32_t, NT>(P, rowtab); break;
+    case 2: units_walk<uint16_t, NT>(P, rowtab); break;
+    default: units_walk<uint8_t, NT>(P, rowtab); break;
+    }
+}
+
+// VARIANT: 0 rows (aligned), 1 chunks aligned, 2 chunks ragged, 3 units
+template <int VARIANT, int NT>
+__device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
+{
+    if (VARIANT == 0) {
+        rows_body<NT>(P);
+    } else {
+        __shared__ RowEntry rowtab[kMaxRowsFlat];
+        if (VARIANT == 1) chunks_body<true, NT>(P, rowtab);
+        if (VARIANT == 2) chunks_body<false, NT>(P, rowtab);
+        if (VARIANT == 3) units_body<NT>(P, rowtab);
+    }
+}
+
 // One entry per collective so that profiles name the step that ran.
-#define REDIST_DEFINE_KERNEL(NAME)                                                               \
-    template <int VEC, int NT>                                                                   \
-    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P) \
-    {                                                                                            \
-        copy_body<VEC, NT>(P);                                                                   \
+#define REDIST_DEFINE_KERNEL(NAME)                                                                   \
+    template <int VARIANT, int NT>                                                                   \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
+    {                                                                                                \
+        copy_body<VARIANT, NT>(P);                                                                   \
     }
 
 REDIST_DEFINE_KERNEL(redist_dynslice_kernel)
@@ -136,29 +377,30 @@ REDIST_DEFINE_KERNEL(redist_allgather_kernel)
 REDIST_DEFINE_KERNEL(redist_allpermute_kernel)
 REDIST_DEFINE_KERNEL(redist_fused_kernel)
 
-template <int VEC, int NT>
-cudaError_t launch_vec_nt(int kernel, const CopyParams<NT> &P, int grid, cudaStream_t stream)
+template <int VARIANT, int NT>
+cudaError_t launch_one(int kernel, const CopyParams<NT> &P, int grid, cudaStream_t stream)
 {
     switch (kernel) {
-    case 0: case 7: redist_dynslice_kernel<VEC, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 1: redist_alltoall_kernel<VEC, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 2: case 6: redist_allgather_kernel<VEC, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 3: case 4: redist_allpermute_kernel<VEC, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    default: redist_fused_kernel<VEC, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    case 0: case 7: redist_dynslice_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    case 1: redist_alltoall_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    case 2: case 6: redist_allgather_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    case 3: case 4: redist_allpermute_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    default: redist_fused_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
     }
     return cudaGetLastError();
 }
 
 template <int NT>
-cudaError_t launch_nt(int kernel, const CopyParams<NT> &P, int grid, cudaStream_t stream)
+cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
+                      char *const *dst_tab, int n_dst, int grid, cudaStream_t stream)
 {
-    switch (P.g.vec_bytes) {
-    case 16: return launch_vec_nt<16, NT>(kernel, P, grid, stream);
-    case 8: return launch_vec_nt<8, NT>(kernel, P, grid, stream);
-    case 4: return launch_vec_nt<4, NT>(kernel, P, grid, stream);
-    case 2: return launch_vec_nt<2, NT>(kernel, P, grid, stream);
-    default: return launch_vec_nt<1, NT>(kernel, P, grid, stream);
-    }
+    CopyParams<NT> P;
+    P.g = geo;
+    for (int i = 0; i < n_src; ++i) P.src[i] = src_tab[i];
+    for (int i = 0; i < n_dst; ++i) P.dst[i] = dst_tab[i];
+    if (geo.mode == kModeRows) return launch_one<0, NT>(kernel, P, grid, stream);
+    if (geo.mode == kModeUnits) return launch_one<3, NT>(kernel, P, grid, stream);
+    return geo.aligned ? launch_one<1, NT>(kernel, P, grid, stream) : launch_one<2, NT>(kernel, P, grid, stream);
 }
 
 }  // namespace
@@ -166,19 +408,10 @@ cudaError_t launch_nt(int kernel, const CopyParams<NT> &P, int grid, cudaStream_
 cudaError_t launch_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
                         char *const *dst_tab, int n_dst, int grid, cudaStream_t stream)
 {
-    if (n_src <= kSmallTable && n_dst <= kSmallTable) {
-        CopyParams<kSmallTable> P;
-        P.g = geo;
-        for (int i = 0; i < n_src; ++i) P.src[i] = src_tab[i];
-        for (int i = 0; i < n_dst; ++i) P.dst[i] = dst_tab[i];
-        return launch_nt<kSmallTable>(kernel, P, grid, stream);
-    }
+    if (n_src <= kSmallTable && n_dst <= kSmallTable)
+        return launch_nt<kSmallTable>(kernel, geo, src_tab, n_src, dst_tab, n_dst, grid, stream);
     if (n_src > kLargeTable || n_dst > kLargeTable) return cudaErrorInvalidValue;
-    CopyParams<kLargeTable> P;
-    P.g = geo;
-    for (int i = 0; i < n_src; ++i) P.src[i] = src_tab[i];
-    for (int i = 0; i < n_dst; ++i) P.dst[i] = dst_tab[i];
-    return launch_nt<kLargeTable>(kernel, P, grid, stream);
+    return launch_nt<kLargeTable>(kernel, geo, src_tab, n_src, dst_tab, n_dst, grid, stream);
 }
 
 }  // namespace redist

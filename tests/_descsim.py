@@ -19,15 +19,27 @@ def _prod(xs):
 def run_launch(L: dict, src_bufs, dst_bufs):
     """src_bufs / dst_bufs: callables device -> 1-D uint8 array (device -1 = the shared buffer)."""
     G = L["geometry"]
-    vec, lanes, fan = G["vec_bytes"], G["lanes"], G["fanout"]
-    run = vec * lanes
+    fan = G["fanout"]
+    run = G["run_bytes"]
+    assert run == L["run_bytes"] and run > 0
     unit_n = G["unit_n"]
     n_boxes = _prod(unit_n)
     rows = G["rows"]
     assert rows == _prod(G["row_n"])
     assert G["n_items"] == n_boxes * G["items_per_box"]
-    assert G["items_per_box"] * G["rows_per_item"] >= rows
-    assert G["rows_per_item"] % G["rows_per_pass"] == 0 and G["rows_per_pass"] == 256 // lanes
+    unit = G["unit_bytes"]
+    assert unit in (1, 2, 4, 8, 16) and (G["aligned"] == 1) == (unit == 16) and run % unit == 0
+    max_chunks = run // 16
+    if G["mode"] == 0:      # rows: aligned runs of at most 256 chunks
+        assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
+        assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0
+        assert G["items_per_box"] * G["rows_per_item"] >= rows
+    else:                   # flat walk over (row, chunk) or (row, unit piece)
+        per_row = max_chunks if G["mode"] == 1 else run // unit
+        assert (G["mode"] == 1 and run >= 256) or (G["mode"] == 2 and run < 256 and unit < 16)
+        assert 1 <= G["rows_per_item"] <= 1024
+        assert G["col_blocks"] * G["per_block"] >= per_row
+        assert G["items_per_box"] == -(-rows // G["rows_per_item"]) * G["col_blocks"]
     # row offsets (mixed radix, last digit fastest)
     r = np.arange(rows, dtype=np.int64)
     s1 = np.zeros(rows, dtype=np.int64)
@@ -50,6 +62,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             t2 += a2 * G["unit_ts2"][u]
             o1 += b1 * G["unit_b1"][u]
             o2 += b2 * G["unit_b2"][u]
+        assert o1 % unit == 0 and o2 % unit == 0 and np.all(s1 % unit == 0) and np.all(s2 % unit == 0)
         src = src_bufs(L["src_holder"][t1])
         data = src[(o1 + s1)[:, None] + col[None, :]]
         for f in range(fan):
