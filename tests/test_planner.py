@@ -325,3 +325,20 @@ def test_near_optimality_against_brute_force(mesh):
         weak = sum(p.step_info(s).cost for s in range(p.num_steps) if p.step_info(s).kind != 3)
         assert weak <= opt                                        # permutation-free part is optimal
         p.close()
+
+
+def test_planner_throughput_on_evaluation_shaped_problems():
+    """Section 8 reports synthesis in under a second per problem (unoptimised Python); the host planner
+    here must stay far below that on 300 problems of the same shape (3 mesh axes, up to 6-D)."""
+    import time
+    ws = wl.evaluation_like_problems(300)
+    worst, t0 = 0.0, time.perf_counter()
+    for w in ws:
+        t1 = time.perf_counter()
+        p = api.Plan(w.mesh_shape, w.src, w.dst, 4)
+        worst = max(worst, time.perf_counter() - t1)
+        assert p.height <= max(p.local_elems(0), p.local_elems(1))
+        assert p.step_kinds().count("allpermute") <= 1
+        p.close()
+    total = time.perf_counter() - t0
+    assert worst < 0.25 and total / len(ws) < 0.05, (worst, total)
