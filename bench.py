@@ -440,6 +440,8 @@ def run_sweep(args):
     G = None
     stream = torch.cuda.current_stream()
     rows = []
+    if args.only:
+        pairs = [w for w in pairs if w.name in args.only.split(",")]
     for w in pairs[: args.pairs]:
         if G is None or tuple(G.shape[:-1]) != tuple(w.src.global_shape):
             G = None
@@ -591,6 +593,7 @@ def main():
     ap.add_argument("--workload", default="c2",
                     choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval"])
     ap.add_argument("--pairs", type=int, default=100, help="sweeps: how many problems to run")
+    ap.add_argument("--only", default="", help="sweeps: comma-separated problem names to run")
     ap.add_argument("--dump", default="", help="sweeps: write the per-problem table to this JSON file")
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
     ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")

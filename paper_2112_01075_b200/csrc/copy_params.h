@@ -11,6 +11,11 @@
 // side; when not every address is a multiple of 16 (`aligned == 0`) the source chunk is assembled
 // from two aligned loads and the ragged head and tail of a run go in `unit_bytes` pieces.
 //
+// Item numbering: the pieces of one long row (the m1*m2 units of the last differing dimension that
+// share a source or target tile row) are consecutive items, so blocks that run at the same time fill
+// the same memory sectors and partial-sector writes merge in L2 instead of being written back alone;
+// then come the row groups of a box, then the boxes.
+//
 // Work items, by `mode`:
 //   kModeRows   aligned runs of at most 256 chunks: a block covers rows_per_pass rows of `lanes`
 //               chunks per pass; an item is rows_per_item rows; every thread decodes its own rows.
@@ -53,6 +58,8 @@ struct CopyGeometry {
     FastDiv per_block_div;           // flat walk: division by per_block
     FastDiv col_blocks;              // flat walk: column blocks per row (1 in kModeRows)
     FastDiv items_per_box;
+    FastDiv inner_n;                 // pieces of one long row that consecutive items handle (1: none)
+    uint32_t inner_digit;            // unit digit those pieces belong to
     FastDiv lanes_div;
     FastDiv unit_n[kMaxUnitDigits];  // boxes along the digit
     FastDiv unit_m1[kMaxUnitDigits];

@@ -79,6 +79,21 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         ++nu;
     }
     G.n_unit = nu;
+    // short runs: the units of dimension kp that lie in the same source or target tile row become
+    // the fastest-varying part of the item number (see copy_params.h)
+    G.inner_n = make_div(1);
+    G.inner_digit = 0xffffffffu;
+    i64 inner = 1;
+    if (kp >= 0 && run_bytes < 1024 && nq[kp] > 1 && m1[kp] * m2[kp] > 1) {
+        inner = m1[kp] * m2[kp];
+        uint32_t u = 0;
+        for (int k = 0; k < kp; ++k)
+            if (nq[k] != 1) ++u;
+        G.inner_digit = u;
+        G.inner_n = make_div(uint32_t(inner));
+        G.unit_n[u] = make_div(uint32_t(nq[kp] / inner));
+        n_boxes /= inner;
+    }
     // row digits inside a box: the dimensions before kp, merged where both sides stay contiguous
     std::vector<RowDigit> rows;
     for (int k = 0; k < kp; ++k) {
@@ -170,9 +185,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }
     G.per_block_div = make_div(G.per_block);
     G.lanes_div = make_div(G.lanes);
-    if (ipb >= (1ll << 31) || n_boxes * ipb >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+    if (ipb >= (1ll << 31) || n_boxes * ipb * inner >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     G.items_per_box = make_div(uint32_t(ipb));
-    G.n_items = uint32_t(n_boxes * ipb);
+    G.n_items = uint32_t(n_boxes * ipb * inner);
 
     // tables
     i64 nt1 = 1, nt2 = 1;

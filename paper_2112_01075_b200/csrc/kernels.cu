@@ -153,13 +153,16 @@ template <int NT>
 __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t item)
 {
     const CopyGeometry &g = P.g;
-    const uint32_t box = fdiv(item, g.items_per_box);
+    const uint32_t outer = fdiv(item, g.inner_n);
+    const uint32_t piece = item - outer * g.inner_n.d;
+    const uint32_t box = fdiv(outer, g.items_per_box);
     uint32_t t1 = 0, t2 = 0, rem = box;
     int64_t o1 = 0, o2 = 0;
     for (int u = int(g.n_unit) - 1; u >= 0; --u) {
         const uint32_t nxt = fdiv(rem, g.unit_n[u]);
-        const uint32_t q = rem - nxt * g.unit_n[u].d;
+        uint32_t q = rem - nxt * g.unit_n[u].d;
         rem = nxt;
+        if (uint32_t(u) == g.inner_digit) q = q * g.inner_n.d + piece;
         const uint32_t a1 = fdiv(q, g.unit_m1[u]);
         const uint32_t a2 = fdiv(q, g.unit_m2[u]);
         t1 += a1 * g.unit_ts1[u];
@@ -171,7 +174,7 @@ __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t 
     b.sbase = P.src[t1] + o1;
     b.dtab = &P.dst[t2 * g.fanout];
     b.o2 = o2;
-    b.part = item - box * g.items_per_box.d;
+    b.part = outer - box * g.items_per_box.d;
     return b;
 }
 

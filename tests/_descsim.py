@@ -26,7 +26,8 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     n_boxes = _prod(unit_n)
     rows = G["rows"]
     assert rows == _prod(G["row_n"])
-    assert G["n_items"] == n_boxes * G["items_per_box"]
+    inner = G["inner_n"]
+    assert G["n_items"] == n_boxes * G["items_per_box"] * inner
     unit = G["unit_bytes"]
     assert unit in (1, 2, 4, 8, 16) and (G["aligned"] == 1) == (unit == 16) and run % unit == 0
     max_chunks = run // 16
@@ -51,11 +52,14 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         s2 += dg * G["row_b2"][q]
     col = np.arange(run, dtype=np.int64)
     written = {}
-    for box in range(n_boxes):
+    for boxp in range(n_boxes * inner):
+        box, piece = divmod(boxp, inner)
         rem, t1, t2, o1, o2 = box, 0, 0, 0, 0
         for u in range(len(unit_n) - 1, -1, -1):
             q = rem % unit_n[u]
             rem //= unit_n[u]
+            if u == G["inner_digit"]:
+                q = q * inner + piece
             a1, b1 = divmod(q, G["unit_m1"][u])
             a2, b2 = divmod(q, G["unit_m2"][u])
             t1 += a1 * G["unit_ts1"][u]
