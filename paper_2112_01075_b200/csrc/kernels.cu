@@ -25,6 +25,8 @@
 // amortised over ~32 KiB of data.
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+
 #include "copy_params.h"
 #include "kernels.h"
 
@@ -356,6 +358,12 @@ __device__ __forceinline__ void units_body(const CopyParams<NT> &P, RowEntry *ro
 template <int VARIANT, int NT>
 __device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
 {
+    // Programmatic dependent launch: blocks of this grid may be scheduled while the previous kernel
+    // on the stream drains; nothing is read or written before that kernel has completed and its
+    // stores are visible.  The next kernel is released to do the same as soon as every block of this
+    // grid has started.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (VARIANT == 0) {
         rows_body<NT>(P);
     } else {
@@ -383,14 +391,26 @@ REDIST_DEFINE_KERNEL(redist_fused_kernel)
 template <int VARIANT, int NT>
 cudaError_t launch_one(int kernel, const CopyParams<NT> &P, int grid, cudaStream_t stream)
 {
+    void (*fn)(const CopyParams<NT>) = nullptr;
     switch (kernel) {
-    case 0: case 7: redist_dynslice_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 1: redist_alltoall_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 2: case 6: redist_allgather_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    case 3: case 4: redist_allpermute_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
-    default: redist_fused_kernel<VARIANT, NT><<<grid, kBlockThreads, 0, stream>>>(P); break;
+    case 0: case 7: fn = redist_dynslice_kernel<VARIANT, NT>; break;
+    case 1: fn = redist_alltoall_kernel<VARIANT, NT>; break;
+    case 2: case 6: fn = redist_allgather_kernel<VARIANT, NT>; break;
+    case 3: case 4: fn = redist_allpermute_kernel<VARIANT, NT>; break;
+    default: fn = redist_fused_kernel<VARIANT, NT>; break;
     }
-    return cudaGetLastError();
+    static const bool kSerialize = std::getenv("REDIST_NO_PDL") != nullptr;   // tuning knob
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid));
+    cfg.blockDim = dim3(kBlockThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = kSerialize ? 0 : 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, P);
 }
 
 template <int NT>
