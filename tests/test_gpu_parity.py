@@ -35,6 +35,7 @@ def assert_same(got, want, what=""):
     assert len(got) == len(want)
     for d, (g, w) in enumerate(zip(got, want)):
         w = np.ascontiguousarray(w).reshape(-1)
+        g = np.ascontiguousarray(g).reshape(-1)
         if not np.array_equal(g, w):
             bad = np.flatnonzero(g != w)
             raise AssertionError(f"{what}: device {d}: {bad.size} of {w.size} bytes differ, first at {bad[0]}")
@@ -280,3 +281,52 @@ def test_random_sweep_full_size_samples():
     finally:
         oracle.set_threads(1)
     assert done == 3
+
+
+def test_execute_can_be_captured_in_a_cuda_graph_and_replayed():
+    """redist_execute allocates nothing and copies no table to the device, so a stream capture records
+    just its kernel launches; replays on new data must still match the oracle."""
+    w = wl.config2().scaled((8, 256, 512))
+    src, dst, src_tiles, want = make_case(w, seed=11)
+    for flags in (api.FUSE_ADJACENT, api.FUSE_NONE):
+        plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes, flags)
+        d_src = [torch.zeros_like(torch.from_numpy(t)).cuda() for t in src_tiles]
+        nb = plan.local_elems(1) * w.elem_bytes
+        d_dst = [torch.zeros(nb, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+        scratch = plan.alloc_scratch()
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            plan.execute(d_src, d_dst, scratch, side)          # warm-up outside the capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            plan.execute(d_src, d_dst, scratch, torch.cuda.current_stream())
+        for seed in (11, 12):
+            _, _, tiles, expect = make_case(w, seed=seed)
+            for t, h in zip(d_src, tiles):
+                t.copy_(torch.from_numpy(h))
+            for t in d_dst:
+                t.fill_(0xEE)
+            g.replay()
+            torch.cuda.synchronize()
+            assert_same([t.cpu().numpy() for t in d_dst], expect, f"graph replay, seed {seed}, flags {flags}")
+
+
+def test_back_to_back_dependent_launches_are_ordered():
+    """Kernels use programmatic dependent launch; a redistribution that reads what the previous one on
+    the same stream wrote must still see all of it (A -> B -> A, 20 times, no synchronisation between)."""
+    w = wl.config3("a").scaled((1024, 1024))
+    src, dst, src_tiles, _ = make_case(w)
+    fwd = api.Plan(w.mesh_shape, src, dst, w.elem_bytes)
+    back = api.Plan(w.mesh_shape, dst, src, w.elem_bytes)
+    a = [torch.from_numpy(t).cuda() for t in src_tiles]
+    b = [torch.zeros(fwd.local_elems(1) * w.elem_bytes, dtype=torch.uint8, device="cuda") for _ in range(8)]
+    c = [torch.zeros(fwd.local_elems(0) * w.elem_bytes, dtype=torch.uint8, device="cuda") for _ in range(8)]
+    for _ in range(20):
+        fwd.execute(a, b)
+        back.execute(b, c)
+        fwd.execute(c, b)
+        back.execute(b, a)
+    torch.cuda.synchronize()
+    assert_same([t.cpu().numpy() for t in a], src_tiles, "A->B->A chain")
+    assert_same([t.cpu().numpy() for t in c], src_tiles, "A->B->A chain (intermediate)")
