@@ -23,7 +23,9 @@
 //               block of per_block chunks; the rows are decoded once into shared memory and all
 //               threads walk the (row, chunk) space with a flat index.
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
-//               (row, piece of unit_bytes).
+//               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
+//               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
+//               table of 1024 entries still covers tens of KiB when runs are a few bytes long.
 #pragma once
 
 #include <cstdint>
@@ -51,7 +53,7 @@ struct CopyGeometry {
     uint64_t run_bytes;              // contiguous run
     uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
     uint32_t rows_per_pass;          // kModeRows: kBlockThreads / lanes
-    uint32_t rows;                   // rows per box
+    uint32_t rows;                   // rows per box (kModeUnits: table rows, i.e. without the innermost digit)
     uint32_t rows_per_item;          // kModeRows: multiple of rows_per_pass; else <= kMaxRowsFlat
     uint32_t per_block;              // flat walk: chunks (or units) of one row in a column block
     uint32_t n_items;
@@ -68,6 +70,9 @@ struct CopyGeometry {
     uint32_t unit_ts2[kMaxUnitDigits];
     int64_t unit_b1[kMaxUnitDigits];     // byte stride of one unit inside the tile
     int64_t unit_b2[kMaxUnitDigits];
+    uint32_t n_row_tab;              // row digits decoded through the shared table (n_row, or n_row - 1)
+    FastDiv tab_inner;               // kModeUnits: runs per table row (extent of the innermost row digit, or 1)
+    FastDiv units_per_run;           // kModeUnits: run_bytes / unit_bytes
     FastDiv row_n[kMaxRowDigits];
     int64_t row_b1[kMaxRowDigits];       // byte stride of the row digit, source / target
     int64_t row_b2[kMaxRowDigits];

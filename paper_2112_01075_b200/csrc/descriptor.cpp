@@ -134,6 +134,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         if (n_rows >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     }
     G.n_row = uint32_t(rows.size());
+    G.n_row_tab = G.n_row;
+    G.tab_inner = make_div(1);
+    G.units_per_run = make_div(1);
     G.unit_bytes = uint32_t(vec);
     G.aligned = vec == 16 ? 1u : 0u;
     G.run_bytes = uint64_t(run_bytes);
@@ -169,19 +172,29 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.col_blocks = make_div(1);
         ipb = (n_rows + rpi - 1) / rpi;
     } else {
-        // flat walk over (row, chunk) -- or over (row, unit piece) for short ragged runs
+        // flat walk over (row, chunk) -- or, for short ragged runs, over (table row, unit piece) where a
+        // table row carries all the runs of the innermost row digit
         const bool units = run_bytes < 256;
-        const i64 per_row = units ? run_bytes / vec : max_chunks;
+        i64 tab_inner = 1, tab_rows = n_rows;
+        if (units && run_bytes <= 16 && !rows.empty()) {   // only when a table of rows could not fill an item
+            tab_inner = rows.back().n;
+            tab_rows = n_rows / tab_inner;
+        }
+        const i64 per_row = units ? tab_inner * (run_bytes / vec) : max_chunks;
         const i64 piece = units ? vec : 16;
         const i64 cpb = std::max<i64>(1, std::min<i64>(per_row, kItemBytes / piece));
         const i64 ncb = std::max<i64>(1, (per_row + cpb - 1) / cpb);
         i64 rpi = std::max<i64>(1, std::min<i64>(kMaxRowsFlat, kItemBytes / (cpb * piece)));
-        rpi = std::min<i64>(rpi, n_rows);
+        rpi = std::min<i64>(rpi, tab_rows);
         G.mode = units ? kModeUnits : kModeChunks;
+        G.rows = uint32_t(tab_rows);
+        G.n_row_tab = uint32_t(tab_inner > 1 ? rows.size() - 1 : rows.size());
+        G.tab_inner = make_div(uint32_t(tab_inner));
+        G.units_per_run = make_div(uint32_t(std::max<i64>(1, run_bytes / vec)));
         G.rows_per_item = uint32_t(rpi);
         G.per_block = uint32_t(cpb);
         G.col_blocks = make_div(uint32_t(ncb));
-        ipb = (n_rows + rpi - 1) / rpi * ncb;
+        ipb = (tab_rows + rpi - 1) / rpi * ncb;
     }
     G.per_block_div = make_div(G.per_block);
     G.lanes_div = make_div(G.lanes);

@@ -113,11 +113,11 @@ __device__ __forceinline__ void copy_units(char *const *dtab, uint32_t fanout, i
 }
 
 // row number inside a box -> byte offsets of the row on the source and target side
-__device__ __forceinline__ void row_offsets(const CopyGeometry &g, uint32_t row, int64_t &s1, int64_t &s2)
+__device__ __forceinline__ void row_offsets(const CopyGeometry &g, uint32_t row, int64_t &s1, int64_t &s2,
+                                            int n_row)
 {
     s1 = 0;
     s2 = 0;
-    const int n_row = int(g.n_row);
     uint32_t r = row;
     for (int q = n_row - 1; q > 0; --q) {
         const uint32_t nxt = fdiv(r, g.row_n[q]);
@@ -206,7 +206,7 @@ __device__ __forceinline__ void rows_body(const CopyParams<NT> &P)
             for (int k = 0; k < kUnroll; ++k) {
                 const uint32_t row = rb + k * rpp + ty;
                 int64_t s1, s2;
-                row_offsets(g, row, s1, s2);
+                row_offsets(g, row, s1, s2, int(g.n_row));
                 ok[k] = active && row < row_end;
                 d2[k] = dcol + s2;
                 if (ok[k]) v[k] = ld_stream(reinterpret_cast<const uint4 *>(sb + s1));
@@ -229,7 +229,7 @@ __device__ __forceinline__ uint32_t fill_rowtab(const CopyGeometry &g, RowEntry 
     __syncthreads();
     for (uint32_t r = threadIdx.x; r < nr; r += kBlockThreads) {
         RowEntry e;
-        row_offsets(g, row0 + r, e.s1, e.s2);
+        row_offsets(g, row0 + r, e.s1, e.s2, int(g.n_row_tab));
         rowtab[r] = e;
     }
     __syncthreads();
@@ -306,19 +306,26 @@ __device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *r
     }
 }
 
-// ---- kModeUnits: flat walk over (row, piece of UNIT bytes) -------------------------------------
-template <typename T, int NT>
+// ---- kModeUnits: flat walk over (table row, run of the innermost row digit, piece of UNIT bytes) --
+template <typename T, bool INNER, int NT>
 __device__ __forceinline__ void units_walk(const CopyParams<NT> &P, RowEntry *rowtab)
 {
     constexpr int kU = 2 * kUnroll;
     const CopyGeometry &g = P.g;
     const uint32_t tid = threadIdx.x;
     const uint32_t fanout = g.fanout;
-    const uint32_t upr = g.per_block;                 // pieces per row (the whole run)
+    const uint32_t cpb = g.per_block;                 // pieces of one table row in a column block
+    const uint32_t upr = g.units_per_run.d;
+    const uint32_t payload = g.tab_inner.d * upr;     // pieces per table row
+    const int64_t in1 = g.n_row_tab < g.n_row ? g.row_b1[g.n_row - 1] : 0;   // strides of the innermost digit
+    const int64_t in2 = g.n_row_tab < g.n_row ? g.row_b2[g.n_row - 1] : 0;
     for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
         const BoxBase b = decode_box(P, item);
-        const uint32_t nr = fill_rowtab(g, rowtab, b.part);
-        const uint32_t total = nr * upr;
+        const uint32_t group = fdiv(b.part, g.col_blocks);
+        const uint32_t cb = b.part - group * g.col_blocks.d;
+        const uint32_t nr = fill_rowtab(g, rowtab, group);
+        const uint32_t total = nr * cpb;
+        const uint32_t c0 = cb * cpb;
         for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
             T v[kU];
             int64_t d2[kU];
@@ -327,11 +334,18 @@ __device__ __forceinline__ void units_walk(const CopyParams<NT> &P, RowEntry *ro
             for (int k = 0; k < kU; ++k) {
                 const uint32_t idx = base + k * kBlockThreads;
                 const uint32_t r = fdiv(idx, g.per_block_div);
-                const uint32_t u = idx - r * upr;
+                const uint32_t c = c0 + (idx - r * cpb);
                 const RowEntry e = rowtab[r < nr ? r : 0];
-                ok[k] = idx < total;
-                d2[k] = b.o2 + e.s2 + int64_t(u) * sizeof(T);
-                if (ok[k]) v[k] = __ldg(reinterpret_cast<const T *>(b.sbase + e.s1 + int64_t(u) * sizeof(T)));
+                ok[k] = idx < total && c < payload;
+                int64_t a1 = e.s1 + int64_t(c) * sizeof(T), a2 = e.s2 + int64_t(c) * sizeof(T);
+                if (INNER) {   // c = run number * pieces per run + piece
+                    const uint32_t i = fdiv(c, g.units_per_run);
+                    const uint32_t u = c - i * upr;
+                    a1 = e.s1 + int64_t(i) * in1 + int64_t(u) * sizeof(T);
+                    a2 = e.s2 + int64_t(i) * in2 + int64_t(u) * sizeof(T);
+                }
+                d2[k] = b.o2 + a2;
+                if (ok[k]) v[k] = __ldg(reinterpret_cast<const T *>(b.sbase + a1));
             }
             for (uint32_t f = 0; f < fanout; ++f) {
                 char *dbase = b.dtab[f];
@@ -346,11 +360,20 @@ __device__ __forceinline__ void units_walk(const CopyParams<NT> &P, RowEntry *ro
 template <int NT>
 __device__ __forceinline__ void units_body(const CopyParams<NT> &P, RowEntry *rowtab)
 {
-    switch (P.g.unit_bytes) {
-    case 8: units_walk<uint2, NT>(P, rowtab); break;
-    case 4: units_walk<uint32_t, NT>(P, rowtab); break;
-    case 2: units_walk<uint16_t, NT>(P, rowtab); break;
-    default: units_walk<uint8_t, NT>(P, rowtab); break;
+    if (P.g.tab_inner.d > 1) {
+        switch (P.g.unit_bytes) {
+        case 8: units_walk<uint2, true, NT>(P, rowtab); break;
+        case 4: units_walk<uint32_t, true, NT>(P, rowtab); break;
+        case 2: units_walk<uint16_t, true, NT>(P, rowtab); break;
+        default: units_walk<uint8_t, true, NT>(P, rowtab); break;
+        }
+    } else {
+        switch (P.g.unit_bytes) {
+        case 8: units_walk<uint2, false, NT>(P, rowtab); break;
+        case 4: units_walk<uint32_t, false, NT>(P, rowtab); break;
+        case 2: units_walk<uint16_t, false, NT>(P, rowtab); break;
+        default: units_walk<uint8_t, false, NT>(P, rowtab); break;
+        }
     }
 }
 

@@ -24,8 +24,9 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     assert run == L["run_bytes"] and run > 0
     unit_n = G["unit_n"]
     n_boxes = _prod(unit_n)
-    rows = G["rows"]
-    assert rows == _prod(G["row_n"])
+    rows = _prod(G["row_n"])
+    tab_rows = G["rows"]
+    assert tab_rows * G["tab_inner"] == rows
     inner = G["inner_n"]
     assert G["n_items"] == n_boxes * G["items_per_box"] * inner
     unit = G["unit_bytes"]
@@ -34,13 +35,15 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     if G["mode"] == 0:      # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
         assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0
-        assert G["items_per_box"] * G["rows_per_item"] >= rows
+        assert G["items_per_box"] * G["rows_per_item"] >= rows and tab_rows == rows
     else:                   # flat walk over (row, chunk) or (row, unit piece)
-        per_row = max_chunks if G["mode"] == 1 else run // unit
+        per_row = max_chunks if G["mode"] == 1 else G["tab_inner"] * (run // unit)
         assert (G["mode"] == 1 and run >= 256) or (G["mode"] == 2 and run < 256 and unit < 16)
+        assert G["mode"] == 2 or G["tab_inner"] == 1
+        assert G["tab_inner"] == 1 or (G["tab_inner"] == G["row_n"][-1] and G["n_row_tab"] == len(G["row_n"]) - 1)
         assert 1 <= G["rows_per_item"] <= 1024
         assert G["col_blocks"] * G["per_block"] >= per_row
-        assert G["items_per_box"] == -(-rows // G["rows_per_item"]) * G["col_blocks"]
+        assert G["items_per_box"] == -(-tab_rows // G["rows_per_item"]) * G["col_blocks"]
     # row offsets (mixed radix, last digit fastest)
     r = np.arange(rows, dtype=np.int64)
     s1 = np.zeros(rows, dtype=np.int64)
