@@ -330,3 +330,37 @@ def test_back_to_back_dependent_launches_are_ordered():
     torch.cuda.synchronize()
     assert_same([t.cpu().numpy() for t in a], src_tiles, "A->B->A chain")
     assert_same([t.cpu().numpy() for t in c], src_tiles, "A->B->A chain (intermediate)")
+
+
+@pytest.mark.parametrize("mesh,src_axes,dst_axes,gshape", [
+    ((4, 4, 4, 4), ((0, 1), (2,), (3,)), ((3,), (1, 0), (2,)), (64, 64, 32)),          # 256 virtual devices
+    ((1024,), ((0,), ()), ((), (0,)), (2048, 1024)),                                   # 1024: the table limit
+    ((2, 3, 5, 7), ((0, 3), (1,), ()), ((2,), (), (3, 1)), (210, 30, 42)),             # 210 devices, odd primes
+    ((8, 16), ((), (0,)), ((1, 0), ()), (256, 64)),                                    # 128 devices, replication
+])
+@pytest.mark.parametrize("mode", [api.FUSE_ADJACENT, api.FUSE_NONE], ids=lambda m: MODE_NAMES[m])
+def test_many_virtual_devices_use_the_large_pointer_tables(mesh, src_axes, dst_axes, gshape, mode):
+    """More than 64 tiles on a side switches to the 1024-entry kernel-parameter tables."""
+    rng = np.random.default_rng(len(mesh))
+    e = 2
+    G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+    src, dst = (gshape, src_axes), (gshape, dst_axes)
+    src_tiles = oracle.reslice(mesh, src, G)
+    want = oracle.reslice(mesh, dst, G)
+    plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
+    assert plan.n_devices > 64
+    assert_same(got, want, f"{mesh}")
+
+
+def test_rank_eight_and_sixteen_byte_elements():
+    mesh = (2, 2, 2)
+    gshape = (2, 3, 4, 2, 5, 2, 3, 4)
+    src = (gshape, ((0,), (), (1,), (), (), (2,), (), ()))
+    dst = (gshape, ((), (), (2,), (0,), (), (), (), (1,)))
+    rng = np.random.default_rng(8)
+    G = rng.integers(0, 256, size=gshape + (16,), dtype=np.uint8)
+    src_tiles = oracle.reslice(mesh, src, G)
+    want = oracle.reslice(mesh, dst, G)
+    for mode in MODES:
+        _, got = run_gpu(mesh, src, dst, 16, src_tiles, mode)
+        assert_same(got, want, "rank 8, 16-byte elements")
