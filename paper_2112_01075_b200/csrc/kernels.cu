@@ -240,6 +240,8 @@ __device__ __forceinline__ uint32_t fill_rowtab(const CopyGeometry &g, RowEntry 
 template <bool ALIGNED, int NT>
 __device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *rowtab)
 {
+    // ragged chunks cost two loads and more registers each: fewer in flight per thread, more blocks per SM
+    constexpr int kU = ALIGNED ? kUnroll : 2;
     const CopyGeometry &g = P.g;
     const uint32_t tid = threadIdx.x;
     const uint32_t fanout = g.fanout;
@@ -252,12 +254,12 @@ __device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *r
         const uint32_t nr = fill_rowtab(g, rowtab, group);
         const uint32_t total = nr * cpb;
         const uint32_t c0 = cb * cpb;
-        for (uint32_t base = tid; base < total; base += kBlockThreads * kUnroll) {
-            uint4 v[kUnroll];
-            int64_t d2[kUnroll];
-            bool ok[kUnroll];
+        for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
+            uint4 v[kU];
+            int64_t d2[kU];
+            bool ok[kU];
 #pragma unroll
-            for (int k = 0; k < kUnroll; ++k) {
+            for (int k = 0; k < kU; ++k) {
                 const uint32_t idx = base + k * kBlockThreads;
                 const uint32_t r = fdiv(idx, g.per_block_div);
                 const uint32_t j = c0 + (idx - r * cpb);
@@ -277,7 +279,7 @@ __device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *r
             for (uint32_t f = 0; f < fanout; ++f) {
                 char *dbase = b.dtab[f];
 #pragma unroll
-                for (int k = 0; k < kUnroll; ++k)
+                for (int k = 0; k < kU; ++k)
                     if (ok[k]) st_stream(reinterpret_cast<uint4 *>(dbase + d2[k]), v[k]);
             }
         }
