@@ -243,6 +243,16 @@ const char *redist_status_string(redist_status status);
 /* The last CUDA error code (cudaError_t as int) seen by the calling thread inside this library. */
 int32_t redist_last_cuda_error(void);
 
+/*
+ * redist_bulk_timeouts -- health counter of the bulk-copy kernels (not part of the paper's method).
+ * Aligned runs are moved by TMA bulk copies whose completion a thread block awaits on an mbarrier
+ * with a bounded number of polls; a block whose wait runs out skips its stores, counts itself here
+ * and returns, so a faulty copy engine shows up as a non-zero count and wrong output instead of a
+ * hang.  Returns the count for the current device since the library was loaded (0 in a healthy run),
+ * or -1 on a CUDA error.  Synchronizes the device.
+ */
+int64_t redist_bulk_timeouts(void);
+
 #ifdef __cplusplus
 }
 #endif

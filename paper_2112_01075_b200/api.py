@@ -32,7 +32,7 @@ EXPORTS = (
     "redist_plan_scratch_bytes_per_device", "redist_plan_staging_bytes", "redist_plan_alignment",
     "redist_plan_height", "redist_plan_cost", "redist_plan_num_steps", "redist_plan_num_launches",
     "redist_plan_step_info", "redist_plan_launch_info", "redist_plan_describe", "redist_base_offsets",
-    "redist_status_string", "redist_last_cuda_error",
+    "redist_status_string", "redist_last_cuda_error", "redist_bulk_timeouts",
 )
 
 
@@ -110,6 +110,8 @@ def load() -> ctypes.CDLL:
     lib.redist_status_string.restype = ctypes.c_char_p
     lib.redist_last_cuda_error.argtypes = []
     lib.redist_last_cuda_error.restype = i32
+    lib.redist_bulk_timeouts.argtypes = []
+    lib.redist_bulk_timeouts.restype = i64
     _lib = lib
     return lib
 
@@ -341,6 +343,11 @@ class Plan:
 
         n = self.scratch_bytes
         return torch.empty(n, dtype=torch.uint8, device=device) if n else None
+
+
+def redist_bulk_timeouts() -> int:
+    """Work items whose bounded bulk-copy wait ran out on the current device (0 in a healthy run)."""
+    return int(load().redist_bulk_timeouts())
 
 
 def redist_plan(mesh_shape, src, dst, elem_bytes: int, flags: int = FUSE_ADJACENT) -> Plan:

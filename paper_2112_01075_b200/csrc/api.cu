@@ -92,6 +92,17 @@ const char *redist_status_string(redist_status s)
 
 int32_t redist_last_cuda_error(void) { return tl_cuda_error; }
 
+int64_t redist_bulk_timeouts(void)
+{
+    unsigned int n = 0;
+    cudaError_t ce = read_bulk_timeouts(&n);
+    if (ce != cudaSuccess) {
+        tl_cuda_error = int(ce);
+        return -1;
+    }
+    return int64_t(n);
+}
+
 redist_status redist_base_offsets(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *type,
                                   int64_t *out_tile, int64_t *out_offsets)
 {

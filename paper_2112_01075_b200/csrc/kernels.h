@@ -16,4 +16,8 @@ constexpr int kLargeTable = 1024;   // ... of the large one (REDIST_MAX_DEVICES)
 cudaError_t launch_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
                         char *const *dst_tab, int n_dst, int grid, cudaStream_t stream);
 
+// Work items of the bulk-copy kernel whose bounded wait ran out on the current device (0 in a healthy
+// run).  Synchronizes the device.
+cudaError_t read_bulk_timeouts(unsigned int *out);
+
 }  // namespace redist

@@ -364,3 +364,43 @@ def test_rank_eight_and_sixteen_byte_elements():
     for mode in MODES:
         _, got = run_gpu(mesh, src, dst, 16, src_tiles, mode)
         assert_same(got, want, "rank 8, 16-byte elements")
+
+
+def test_one_plan_executed_from_several_host_threads():
+    """A plan is immutable: host threads may execute it at the same time on their own streams and
+    buffers (the foreign call releases the interpreter lock)."""
+    import threading
+    w = wl.config2().scaled((8, 256, 512))
+    src, dst, _, _ = make_case(w)
+    plan = api.Plan(w.mesh_shape, src, dst, w.elem_bytes, api.FUSE_NONE)
+    nb = plan.local_elems(1) * w.elem_bytes
+    jobs = []
+    for t in range(4):
+        _, _, tiles, want = make_case(w, seed=100 + t)
+        jobs.append({"src": [torch.from_numpy(x).cuda() for x in tiles], "want": want,
+                     "dst": [torch.zeros(nb, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)],
+                     "scratch": plan.alloc_scratch(), "stream": torch.cuda.Stream(), "err": None})
+    torch.cuda.synchronize()
+
+    def work(j):
+        try:
+            for _ in range(50):
+                plan.execute(j["src"], j["dst"], j["scratch"], j["stream"])
+        except Exception as ex:      # surfaced below
+            j["err"] = ex
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    for j in jobs:
+        assert j["err"] is None, j["err"]
+        assert_same([t.cpu().numpy() for t in j["dst"]], j["want"], "threaded execute")
+
+
+def test_zero_bulk_copy_timeouts_after_everything_above():
+    """The bounded waits of the bulk-copy kernels never ran out."""
+    torch.cuda.synchronize()
+    assert api.redist_bulk_timeouts() == 0
