@@ -59,7 +59,7 @@ class LaunchInfo(ctypes.Structure):
     _fields_ = [("first_step", ctypes.c_int32), ("n_steps", ctypes.c_int32), ("kernel", ctypes.c_int32),
                 ("vector_bytes", ctypes.c_int32), ("run_bytes", ctypes.c_int64), ("bytes_read", ctypes.c_int64),
                 ("bytes_written", ctypes.c_int64), ("n_items", ctypes.c_int64), ("fanout", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("variant", ctypes.c_int32)]
 
 
 _lib = None

@@ -35,6 +35,7 @@ namespace redist {
 constexpr int kMaxUnitDigits = 8;
 constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
+constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
 constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2;
 
@@ -50,6 +51,7 @@ struct CopyGeometry {
     uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
     uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
     uint32_t mode;                   // kModeRows, kModeChunks or kModeUnits
+    uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes)
     uint64_t run_bytes;              // contiguous run
     uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
     uint32_t rows_per_pass;          // kModeRows: kBlockThreads / lanes

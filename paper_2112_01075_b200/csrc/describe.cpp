@@ -103,7 +103,7 @@ void describe(Plan &p)
           << ",\"run_bytes\":" << L.run_bytes << ",\"bytes_read\":" << L.bytes_read << ",\"bytes_written\":"
           << L.bytes_written << ",\"src_tile_bytes\":" << L.src_tile_bytes << ",\"dst_tile_bytes\":"
           << L.dst_tile_bytes << ",\"geometry\":{\"fanout\":" << G.fanout << ",\"aligned\":" << G.aligned
-          << ",\"unit_bytes\":" << G.unit_bytes << ",\"mode\":" << G.mode << ",\"run_bytes\":" << G.run_bytes
+          << ",\"unit_bytes\":" << G.unit_bytes << ",\"mode\":" << G.mode << ",\"bulk\":" << G.bulk << ",\"run_bytes\":" << G.run_bytes
           << ",\"per_block\":" << G.per_block << ",\"col_blocks\":" << G.col_blocks.d
           << ",\"lanes\":" << G.lanes << ",\"rows_per_pass\":" << G.rows_per_pass << ",\"rows\":" << G.rows
           << ",\"rows_per_item\":" << G.rows_per_item << ",\"items_per_box\":" << G.items_per_box.d

@@ -196,6 +196,21 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.col_blocks = make_div(uint32_t(ncb));
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     }
+    // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
+    // thread, the item staged in at most 47 KiB of shared memory)
+    static const bool kBulk = [] {
+        const char *v = std::getenv("REDIST_BULK");      // tuning knob: REDIST_BULK=0 keeps aligned runs on the register path
+        return !v || std::atoi(v) > 0;
+    }();
+    static const i64 kBulkMin = [] {
+        const char *v = std::getenv("REDIST_BULK_MIN");  // tuning knob: shortest segment moved by a bulk copy
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 512);
+    }();
+    G.bulk = 0;
+    if (kBulk && G.aligned && G.mode != kModeUnits) {
+        const i64 seg = G.mode == kModeRows ? run_bytes : i64(G.per_block) * 16;
+        if (seg >= kBulkMin && G.rows_per_item <= uint32_t(kBulkThreads) && seg * G.rows_per_item <= 47 * 1024) G.bulk = 1;
+    }
     G.per_block_div = make_div(G.per_block);
     G.lanes_div = make_div(G.lanes);
     if (ipb >= (1ll << 31) || n_boxes * ipb * inner >= (1ll << 31)) return REDIST_EUNSUPPORTED;

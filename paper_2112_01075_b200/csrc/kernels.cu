@@ -411,7 +411,6 @@ __device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
 // bulk copy shared -> global per target replica.  A handful of threads issue the copies; nothing
 // passes through registers.  No cluster multicast is used.  The wait on the mbarrier is bounded: if
 // it runs out, the block counts a timeout, skips its stores and returns.
-constexpr int kBulkThreads = 64;
 __device__ unsigned int g_bulk_timeouts = 0;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p)
@@ -559,17 +558,9 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
     P.g = geo;
     for (int i = 0; i < n_src; ++i) P.src[i] = src_tab[i];
     for (int i = 0; i < n_dst; ++i) P.dst[i] = dst_tab[i];
-    static const bool kBulk = [] {
-        const char *v = std::getenv("REDIST_BULK");      // tuning knob: REDIST_BULK=0 keeps aligned runs on the register path
-        return !v || std::atoi(v) > 0;
-    }();
-    static const uint64_t kBulkMin = [] {
-        const char *v = std::getenv("REDIST_BULK_MIN");  // tuning knob: shortest segment moved by a bulk copy
-        return uint64_t(v && std::atoi(v) > 0 ? std::atoi(v) : 512);
-    }();
-    if (kBulk && geo.aligned && geo.mode != kModeUnits) {
+    if (geo.bulk) {
         const uint64_t seg = geo.mode == kModeRows ? geo.run_bytes : uint64_t(geo.per_block) * 16u;
-        if (seg >= kBulkMin && geo.rows_per_item <= uint32_t(kBulkThreads) && seg * geo.rows_per_item <= 47u * 1024u) {
+        {
             void (*fn)(const CopyParams<NT>) = nullptr;
             switch (kernel) {
             case 0: case 7: fn = redist_dynslice_bulk_kernel<NT>; break;
