@@ -10,10 +10,6 @@
 #include "kernels.h"
 #include "plan.hpp"
 
-struct redist_plan_s {
-    redist::Plan p;
-};
-
 using namespace redist;
 
 namespace redist {

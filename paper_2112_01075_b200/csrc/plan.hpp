@@ -79,6 +79,15 @@ struct Plan {
     std::string json;
 };
 
+}  // namespace redist
+
+// The opaque handle of the C boundary.
+struct redist_plan_s {
+    redist::Plan p;
+};
+
+namespace redist {
+
 // api.cu: last CUDA error seen by the calling thread inside the library
 extern thread_local int tl_cuda_error;
 

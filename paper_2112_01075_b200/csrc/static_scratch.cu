@@ -14,11 +14,6 @@
 #include "kernels.h"
 #include "plan.hpp"
 
-// Same definition as in api.cu (the handle is opaque outside the library).
-struct redist_plan_s {
-    redist::Plan p;
-};
-
 namespace {
 
 // The scratch itself.  Every GPU that loads this library carries these bytes until the process

@@ -400,6 +400,28 @@ def test_one_plan_executed_from_several_host_threads():
         assert_same([t.cpu().numpy() for t in j["dst"]], j["want"], "threaded execute")
 
 
+def test_soak_full_size_forward_and_back_without_synchronising():
+    """Config 2 at full size, forward and back 100 times on one stream with no host synchronisation:
+    kernels overlap their ramp-up with the previous kernel's tail (programmatic dependent launch) and
+    every one reads what the previous one wrote.  The data must come back unchanged."""
+    w = wl.bench_workloads()["c2"]
+    src, dst = types_of(w)
+    G = wl.global_array_bytes(w.src.global_shape, w.elem_bytes, w.fill, w.seed)
+    tiles = oracle.reslice(w.mesh_shape, src, G)
+    fwd = api.Plan(w.mesh_shape, src, dst, w.elem_bytes)
+    back = api.Plan(w.mesh_shape, dst, src, w.elem_bytes)
+    a = [torch.from_numpy(t).cuda() for t in tiles]
+    b = [torch.zeros(fwd.local_elems(1) * w.elem_bytes, dtype=torch.uint8, device="cuda") for _ in range(8)]
+    for _ in range(100):
+        fwd.execute(a, b)
+        back.execute(b, a)
+    torch.cuda.synchronize()
+    assert_same([t.cpu().numpy() for t in a], tiles, "soak")
+    want = oracle.reslice(w.mesh_shape, dst, G)
+    assert_same([t.cpu().numpy() for t in b], want, "soak (intermediate)")
+    assert api.redist_bulk_timeouts() == 0
+
+
 def test_zero_bulk_copy_timeouts_after_everything_above():
     """The bounded waits of the bulk-copy kernels never ran out."""
     torch.cuda.synchronize()
