@@ -259,6 +259,52 @@ class Plan:
         self._lib.redist_plan_describe(self._h, buf, n + 1)
         return json.loads(buf.value.decode())
 
+    def pretty(self, axis_names: Optional[Sequence[str]] = None) -> str:
+        """The synthesized sequence in the paper's notation, one collective per line, over the
+        prime-factor mesh (axis ``x`` of size 4 appears as ``x.0, x.1``), followed by the launches."""
+        d = self.describe()
+        names = list(axis_names) if axis_names else [f"a{i}" for i in range(len(d["mesh_shape"]))]
+        count: dict = {}
+        pnames = []
+        for p in d["primes"]:
+            k = count.get(p["parent"], 0)
+            count[p["parent"]] = k + 1
+            pnames.append(f"{names[p['parent']]}.{k}")
+        multi = {par for par, c in count.items() if c > 1}
+        pnames = [n if d["primes"][i]["parent"] in multi else n.split(".")[0] for i, n in enumerate(pnames)]
+        sizes = [p["size"] for p in d["primes"]]
+
+        def fmt(axes):
+            parts = []
+            for s_k, ax in zip(d["global_shape"], axes):
+                if not ax:
+                    parts.append(str(s_k))
+                    continue
+                k = 1
+                for a in ax:
+                    k *= sizes[a]
+                parts.append(f"{s_k // k}{{{','.join(pnames[a] for a in ax)}}}{s_k}")
+            return "[" + ", ".join(parts) + "]"
+
+        lines = [fmt(d["src_axes"])]
+        for st in d["steps"]:
+            label = st["kind"]
+            if st["kind"] == "alltoall":
+                label += f"({st['i']},{st['j']})"
+            elif st["kind"] in ("allgather", "dynslice"):
+                label += f"({st['i']})"
+            if st["acting"]:
+                label += "{" + ",".join(pnames[a] for a in st["acting"]) + "}"
+            lines.append(f"  --{label}, cost {st['cost']}--> {fmt(st['post_axes'])}")
+        for L in d["launches"]:
+            g = L["geometry"]
+            how = "TMA bulk copies" if g["bulk"] else ("rows", "chunks", "units")[g["mode"]]
+            lines.append(f"  launch {L['kernel']}: steps {L['first_step']}..{L['first_step'] + L['n_steps'] - 1}, "
+                         f"{L['from']} -> {L['to']}, runs of {L['run_bytes']} B, {g['n_items']} items, {how}")
+        lines.append(f"  cost {d['cost']}, height {d['height']} <= max(localsize) "
+                     f"{max(d['local_src'], d['local_dst'])}, scratch per device {d['scratch_per_device']} B")
+        return "\n".join(lines)
+
     # ---- execution
     def execute_ptrs(self, src_ptrs: Sequence[int], dst_ptrs: Sequence[int], scratch_ptr: int = 0,
                      scratch_bytes: int = 0, stream: int = 0) -> None:

@@ -64,3 +64,12 @@ def test_execute_rejects_bad_buffers_before_touching_the_gpu():
         with pytest.raises(api.RedistError) as e:
             q.execute_ptrs([4096 * (i + 1) for i in range(4)], [65536 + 4096 * i for i in range(4)])
         assert e.value.status == 5                  # scratch missing
+
+
+def test_pretty_prints_the_sequence_in_the_papers_notation():
+    p = api.Plan((4, 2), ((8, 2048, 4096), ((0,), (), (1,))), ((8, 2048, 4096), ((), (0, 1), ())), 2)
+    text = p.pretty(("x", "y"))
+    lines = text.splitlines()
+    assert lines[0] == "[2{x.0,x.1}8, 2048, 2048{y}4096]"
+    assert lines[2].endswith("[8, 256{x.0,x.1,y}2048, 4096]") and "alltoall" in lines[1] and "alltoall" in lines[2]
+    assert "launch fused: steps 0..1, src -> dst" in text and "scratch per device 0 B" in text
