@@ -22,6 +22,12 @@
 //   kModeChunks all other runs of at least 256 bytes: an item is rows_per_item rows times one column
 //               block of per_block chunks; the rows are decoded once into shared memory and all
 //               threads walk the (row, chunk) space with a flat index.
+//   kModeStaged ragged runs shorter than 256 bytes where the rows of one side are `stage_w` runs long
+//               and come from (or go to) stage_w different tiles of the other side -- the block
+//               transpose of an alltoall or the concatenation of an allgather along the last
+//               differing dimension.  An item stages rows_per_item such rows in shared memory: the
+//               short side moves piece by piece (a thread per piece, 4-byte words), the long side in
+//               16-byte chunks, so the long rows are read or written whole.
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
 //               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
 //               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
@@ -37,7 +43,8 @@ constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
 constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
-constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2;
+constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeStaged = 3;
+constexpr int kStageRows = 256;        // rows of one item of the staged transpose
 
 // Division of a 31-bit unsigned number by a constant: n / d == umulhi(n, mul) >> shr (d > 1).
 struct FastDiv {
@@ -62,8 +69,15 @@ struct CopyGeometry {
     FastDiv per_block_div;           // flat walk: division by per_block
     FastDiv col_blocks;              // flat walk: column blocks per row (1 in kModeRows)
     FastDiv items_per_box;
-    FastDiv inner_n;                 // pieces of one long row that consecutive items handle (1: none)
+    FastDiv inner_n;                 // pieces (or windows of pieces) of one long row that consecutive items handle (1: none)
     uint32_t inner_digit;            // unit digit those pieces belong to
+    uint32_t inner_span;             // units of that digit per long row (m1 * m2)
+    uint32_t inner_mul;              // units per item along that digit: 1, or stage_w in kModeStaged
+    uint32_t stage_long_dst;         // kModeStaged: 1 the target has the long rows, 0 the source
+    uint32_t stage_pitch;            // kModeStaged: bytes between staged rows in shared memory
+    uint32_t stage_ts;               // kModeStaged: tile-index stride between the pieces on the short side
+    uint32_t stage_rows_log2;        // kModeStaged: log2(rows_per_item)
+    uint32_t stage_tpp_log2;         // kModeStaged: log2(threads per piece on the short side)
     FastDiv lanes_div;
     FastDiv unit_n[kMaxUnitDigits];  // boxes along the digit
     FastDiv unit_m1[kMaxUnitDigits];

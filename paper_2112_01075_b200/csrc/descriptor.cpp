@@ -83,6 +83,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // the fastest-varying part of the item number (see copy_params.h)
     G.inner_n = make_div(1);
     G.inner_digit = 0xffffffffu;
+    G.inner_span = 1;
+    G.inner_mul = 1;
     i64 inner = 1;
     if (kp >= 0 && run_bytes < 1024 && nq[kp] > 1 && m1[kp] * m2[kp] > 1) {
         inner = m1[kp] * m2[kp];
@@ -90,6 +92,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         for (int k = 0; k < kp; ++k)
             if (nq[k] != 1) ++u;
         G.inner_digit = u;
+        G.inner_span = uint32_t(inner);
         G.inner_n = make_div(uint32_t(inner));
         G.unit_n[u] = make_div(uint32_t(nq[kp] / inner));
         n_boxes /= inner;
@@ -159,7 +162,50 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     i64 ipb;
     G.lanes = kBlockThreads;
     G.rows_per_pass = 1;
-    if (G.aligned && max_chunks <= kBlockThreads) {
+    // staged transpose: ragged short runs whose long-side rows are `m` runs from m tiles
+    static const bool kStaged = [] {
+        const char *v = std::getenv("REDIST_STAGED");    // tuning knob: REDIST_STAGED=0 disables the staged transpose
+        return !v || std::atoi(v) > 0;
+    }();
+    i64 stage_w = 0;
+    if (kStaged && !G.aligned && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu &&
+        m1[kp] == 1 && m2[kp] > 1 && fan >= 2) {
+        // measured: staging pays when the target has the long rows (pieces are gathered) and every
+        // staged row is stored to two or more replicas; otherwise the piece-by-piece walk is as fast
+        const i64 m = std::max(m1[kp], m2[kp]);
+        for (i64 c = m; c >= 2; --c)
+            if (m % c == 0 && c * run_bytes <= 4096) {
+                stage_w = c;
+                break;
+            }
+    }
+    if (stage_w >= 2) {
+        const i64 m = std::max(m1[kp], m2[kp]);
+        const i64 wl = stage_w * run_bytes;
+        i64 pitch = round_up(wl, 16) + 16;
+        if ((pitch / 16) % 2 == 0) pitch += 16;      // odd number of 16-byte units: fewer bank conflicts
+        i64 lg = 0;
+        while ((2ll << lg) <= kStageRows && (2ll << lg) * pitch <= 40 * 1024 && (2ll << lg) * wl <= 2 * kItemBytes) ++lg;
+        const i64 rpi = 1ll << lg;
+        G.mode = kModeStaged;
+        G.inner_mul = uint32_t(stage_w);
+        G.inner_n = make_div(uint32_t(m / stage_w));
+        inner = m / stage_w;
+        G.stage_long_dst = m2[kp] > 1 ? 1u : 0u;
+        G.stage_pitch = uint32_t(pitch);
+        G.stage_ts = m2[kp] > 1 ? G.unit_ts1[G.inner_digit] : G.unit_ts2[G.inner_digit];
+        G.stage_rows_log2 = uint32_t(lg);
+        {
+            // threads per piece: about four 4-byte words each, at most a warp
+            uint32_t tl = 0;
+            while (tl < 5 && (4ll << tl) < run_bytes / 4) ++tl;
+            G.stage_tpp_log2 = tl;
+        }
+        G.rows_per_item = uint32_t(rpi);
+        G.per_block = uint32_t(wl / 16 + 1);
+        G.col_blocks = make_div(1);
+        ipb = (n_rows + rpi - 1) / rpi;
+    } else if (G.aligned && max_chunks <= kBlockThreads) {
         // aligned short runs: `lanes` threads per row, one chunk each
         const i64 lanes = max_chunks;
         G.mode = kModeRows;

@@ -153,7 +153,8 @@ struct RowEntry {
 struct BoxBase {
     const char *sbase;       // source tile base + offset of the box
     char *const *dtab;       // target replica base pointers
-    int64_t o2;              // offset of the box inside the target tile
+    int64_t o1, o2;          // offset of the box inside the source / target tile
+    uint32_t t1, t2;         // source / target tile index
     uint32_t part;           // item number inside the box
 };
 
@@ -170,7 +171,7 @@ __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t 
         const uint32_t nxt = fdiv(rem, g.unit_n[u]);
         uint32_t q = rem - nxt * g.unit_n[u].d;
         rem = nxt;
-        if (uint32_t(u) == g.inner_digit) q = q * g.inner_n.d + piece;
+        if (uint32_t(u) == g.inner_digit) q = q * g.inner_span + piece * g.inner_mul;
         const uint32_t a1 = fdiv(q, g.unit_m1[u]);
         const uint32_t a2 = fdiv(q, g.unit_m2[u]);
         t1 += a1 * g.unit_ts1[u];
@@ -181,7 +182,10 @@ __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t 
     BoxBase b;
     b.sbase = P.src[t1] + o1;
     b.dtab = &P.dst[t2 * g.fanout];
+    b.o1 = o1;
     b.o2 = o2;
+    b.t1 = t1;
+    b.t2 = t2;
     b.part = outer - box * g.items_per_box.d;
     return b;
 }
@@ -405,6 +409,120 @@ __device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
     }
 }
 
+// ---- kModeStaged: block transpose of short runs through shared memory ---------------------------
+// The long side has rows of w runs (one tile); the short side has the w runs in w different tiles.
+// Shared memory holds rows_per_item long rows, row r at r * pitch + (long-side address of the row mod
+// 16), so that 16-byte chunks of the long side are aligned in both memories.  Short side: one thread
+// per (row, piece), a loop over the 4-byte words of the piece; adjacent lanes take adjacent rows, so
+// their pieces are neighbours in memory whenever the short-side tile is contiguous.  Long side: flat
+// walk over (row, 16-byte chunk) plus the few words before and after the chunk grid of a row.
+template <bool LONG_DST, int NT>
+__device__ __forceinline__ void staged_body(const CopyParams<NT> &P)
+{
+    extern __shared__ __align__(16) unsigned char tile[];
+    __shared__ RowEntry rowtab[kStageRows];
+    const CopyGeometry &g = P.g;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t fanout = g.fanout;
+    const uint32_t w = g.inner_mul;
+    const uint32_t run = uint32_t(g.run_bytes);
+    const uint32_t wl = w * run;                  // bytes of one long row in the window
+    const uint32_t pitch = g.stage_pitch;
+    const uint32_t words = run >> 2;
+    const uint32_t cpr = g.per_block;             // chunk slots per row
+    const uint32_t lg = g.stage_rows_log2;
+    for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
+        const BoxBase b = decode_box(P, item);
+        const uint32_t nr = fill_rowtab(g, rowtab, b.part);
+        // offset of the long row r in its tile: (LONG_DST ? o2 + s2 : o1 + s1); bases are 16-byte aligned
+        auto long_off = [&](const RowEntry &e) { return LONG_DST ? b.o2 + e.s2 : b.o1 + e.s1; };
+
+        // long side -> shared (source has the long rows)
+        if (!LONG_DST) {
+            const char *lsrc = P.src[b.t1];
+            for (uint32_t idx = tid; idx < nr * cpr; idx += kBlockThreads) {
+                const uint32_t r = fdiv(idx, g.per_block_div);
+                const uint32_t c = idx - r * cpr;
+                const int64_t off = long_off(rowtab[r]);
+                const uint32_t ph = uint32_t(off) & 15u;
+                const uint32_t head = min((16u - ph) & 15u, wl);
+                const uint32_t chunks = (wl - head) >> 4;
+                if (c < chunks)
+                    *reinterpret_cast<uint4 *>(tile + r * pitch + ph + head + (c << 4)) =
+                        __ldg(reinterpret_cast<const uint4 *>(lsrc + off + head + (c << 4)));
+            }
+            for (uint32_t idx = tid; idx < nr * 6u; idx += kBlockThreads) {
+                const uint32_t r = idx / 6u, slot = idx - r * 6u;
+                const int64_t off = long_off(rowtab[r]);
+                const uint32_t ph = uint32_t(off) & 15u;
+                const uint32_t head = min((16u - ph) & 15u, wl);
+                const uint32_t tail_at = head + (((wl - head) >> 4) << 4);
+                const uint32_t at = slot < 3u ? slot * 4u : tail_at + (slot - 3u) * 4u;
+                const bool ok = slot < 3u ? at < head : at < wl;
+                if (ok)
+                    *reinterpret_cast<uint32_t *>(tile + r * pitch + ph + at) =
+                        __ldg(reinterpret_cast<const uint32_t *>(lsrc + off + at));
+            }
+            __syncthreads();
+        }
+
+        // short side <-> shared: 2^stage_tpp_log2 threads per (row, piece), striding over its words
+        const uint32_t tl = g.stage_tpp_log2;
+        for (uint32_t p = tid; p < (w << (lg + tl)); p += kBlockThreads) {
+            const uint32_t sub = p & ((1u << tl) - 1u);
+            const uint32_t pair = p >> tl;
+            const uint32_t j = pair >> lg;
+            const uint32_t r = pair - (j << lg);
+            if (r >= nr) continue;
+            const RowEntry e = rowtab[r];
+            const uint32_t ph = uint32_t(long_off(e)) & 15u;
+            uint32_t *sm = reinterpret_cast<uint32_t *>(tile + r * pitch + ph + j * run);
+            if (LONG_DST) {
+                const uint32_t *gsrc = reinterpret_cast<const uint32_t *>(P.src[b.t1 + j * g.stage_ts] + b.o1 + e.s1);
+                for (uint32_t u = sub; u < words; u += 1u << tl) sm[u] = __ldg(gsrc + u);
+            } else {
+                char *const *dt = &P.dst[(b.t2 + j * g.stage_ts) * fanout];
+                for (uint32_t f = 0; f < fanout; ++f) {
+                    uint32_t *gdst = reinterpret_cast<uint32_t *>(dt[f] + b.o2 + e.s2);
+                    for (uint32_t u = sub; u < words; u += 1u << tl) gdst[u] = sm[u];
+                }
+            }
+        }
+
+        // shared -> long side (target has the long rows)
+        if (LONG_DST) {
+            __syncthreads();
+            for (uint32_t idx = tid; idx < nr * cpr; idx += kBlockThreads) {
+                const uint32_t r = fdiv(idx, g.per_block_div);
+                const uint32_t c = idx - r * cpr;
+                const int64_t off = long_off(rowtab[r]);
+                const uint32_t ph = uint32_t(off) & 15u;
+                const uint32_t head = min((16u - ph) & 15u, wl);
+                const uint32_t chunks = (wl - head) >> 4;
+                if (c < chunks) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(tile + r * pitch + ph + head + (c << 4));
+                    for (uint32_t f = 0; f < fanout; ++f)
+                        st_stream(reinterpret_cast<uint4 *>(b.dtab[f] + off + head + (c << 4)), v);
+                }
+            }
+            for (uint32_t idx = tid; idx < nr * 6u; idx += kBlockThreads) {
+                const uint32_t r = idx / 6u, slot = idx - r * 6u;
+                const int64_t off = long_off(rowtab[r]);
+                const uint32_t ph = uint32_t(off) & 15u;
+                const uint32_t head = min((16u - ph) & 15u, wl);
+                const uint32_t tail_at = head + (((wl - head) >> 4) << 4);
+                const uint32_t at = slot < 3u ? slot * 4u : tail_at + (slot - 3u) * 4u;
+                const bool ok = slot < 3u ? at < head : at < wl;
+                if (ok) {
+                    const uint32_t v = *reinterpret_cast<const uint32_t *>(tile + r * pitch + ph + at);
+                    for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint32_t *>(b.dtab[f] + off + at) = v;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // ---- bulk-copy variant (aligned runs of at least 512 bytes): TMA moves the segments --------------
 // One work item per block.  Every row segment of the item is one bulk asynchronous copy global ->
 // shared (cp.async.bulk, completion counted in bytes on an mbarrier) and, once all have landed, one
@@ -512,6 +630,21 @@ REDIST_DEFINE_BULK_KERNEL(redist_allgather_bulk_kernel)
 REDIST_DEFINE_BULK_KERNEL(redist_allpermute_bulk_kernel)
 REDIST_DEFINE_BULK_KERNEL(redist_fused_bulk_kernel)
 
+#define REDIST_DEFINE_STAGED_KERNEL(NAME)                                                            \
+    template <bool LONG_DST, int NT>                                                                 \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
+    {                                                                                                \
+        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
+        staged_body<LONG_DST, NT>(P);                                                                \
+    }
+
+REDIST_DEFINE_STAGED_KERNEL(redist_dynslice_staged_kernel)
+REDIST_DEFINE_STAGED_KERNEL(redist_alltoall_staged_kernel)
+REDIST_DEFINE_STAGED_KERNEL(redist_allgather_staged_kernel)
+REDIST_DEFINE_STAGED_KERNEL(redist_allpermute_staged_kernel)
+REDIST_DEFINE_STAGED_KERNEL(redist_fused_staged_kernel)
+
 #define REDIST_DEFINE_KERNEL(NAME)                                                                   \
     template <int VARIANT, int NT>                                                                   \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
@@ -581,6 +714,28 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
             cfg.numAttrs = 1;
             return cudaLaunchKernelEx(&cfg, fn, P);
         }
+    }
+    if (geo.mode == kModeStaged) {
+        void (*fn)(const CopyParams<NT>) = nullptr;
+        const bool ld = geo.stage_long_dst != 0;
+        switch (kernel) {
+        case 0: case 7: fn = ld ? redist_dynslice_staged_kernel<true, NT> : redist_dynslice_staged_kernel<false, NT>; break;
+        case 1: fn = ld ? redist_alltoall_staged_kernel<true, NT> : redist_alltoall_staged_kernel<false, NT>; break;
+        case 2: case 6: fn = ld ? redist_allgather_staged_kernel<true, NT> : redist_allgather_staged_kernel<false, NT>; break;
+        case 3: case 4: fn = ld ? redist_allpermute_staged_kernel<true, NT> : redist_allpermute_staged_kernel<false, NT>; break;
+        default: fn = ld ? redist_fused_staged_kernel<true, NT> : redist_fused_staged_kernel<false, NT>; break;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(unsigned(grid));
+        cfg.blockDim = dim3(kBlockThreads);
+        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fn, P);
     }
     if (geo.mode == kModeRows) return launch_one<0, NT>(kernel, P, grid, stream);
     if (geo.mode == kModeUnits) return launch_one<3, NT>(kernel, P, grid, stream);

@@ -27,12 +27,21 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     rows = _prod(G["row_n"])
     tab_rows = G["rows"]
     assert tab_rows * G["tab_inner"] == rows
-    inner = G["inner_n"]
+    inner, span, mul = G["inner_n"], G["inner_span"], G["inner_mul"]
+    assert inner * mul == span
     assert G["n_items"] == n_boxes * G["items_per_box"] * inner
     unit = G["unit_bytes"]
     assert unit in (1, 2, 4, 8, 16) and (G["aligned"] == 1) == (unit == 16) and run % unit == 0
     max_chunks = run // 16
-    if G["mode"] == 0:      # rows: aligned runs of at most 256 chunks
+    if G["mode"] == 3:      # staged transpose: rows_per_item long rows of `mul` runs in shared memory
+        rpi = G["rows_per_item"]
+        assert unit >= 4 and unit < 16 and run < 256 and mul >= 2 and mul * run <= 4096
+        assert rpi & (rpi - 1) == 0 and 1 <= rpi <= 256
+        assert G["stage_pitch"] % 16 == 0 and G["stage_pitch"] >= mul * run + 16 and G["stage_pitch"] * rpi <= 40 * 1024
+        assert G["items_per_box"] == -(-rows // rpi) and tab_rows == rows
+        u = G["inner_digit"]
+        assert G["unit_m1"][u] == 1 and G["unit_m2"][u] > 1 and G["stage_long_dst"] == 1 and fan >= 2
+    elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
         assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0
         assert G["items_per_box"] * G["rows_per_item"] >= rows and tab_rows == rows
@@ -55,14 +64,14 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         s2 += dg * G["row_b2"][q]
     col = np.arange(run, dtype=np.int64)
     written = {}
-    for boxp in range(n_boxes * inner):
-        box, piece = divmod(boxp, inner)
+    for boxp in range(n_boxes * span):
+        box, piece = divmod(boxp, span)          # a staged item covers `mul` consecutive pieces
         rem, t1, t2, o1, o2 = box, 0, 0, 0, 0
         for u in range(len(unit_n) - 1, -1, -1):
             q = rem % unit_n[u]
             rem //= unit_n[u]
             if u == G["inner_digit"]:
-                q = q * inner + piece
+                q = q * span + piece
             a1, b1 = divmod(q, G["unit_m1"][u])
             a2, b2 = divmod(q, G["unit_m2"][u])
             t1 += a1 * G["unit_ts1"][u]

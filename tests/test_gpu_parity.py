@@ -422,6 +422,34 @@ def test_soak_full_size_forward_and_back_without_synchronising():
     assert api.redist_bulk_timeouts() == 0
 
 
+STAGED = [
+    ((2, 4), (6, 10, 24), ((), (), (1,)), ((), (), ()), 4),
+    ((2, 2, 2), (8, 6, 60), ((0,), (), (1, 2)), ((0,), (), (1,)), 4),
+    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4),
+    ((2, 3, 2), (4, 9, 180), ((0,), (), (1, 2)), ((), (), (2,)), 4),
+    ((8,), (33, 88), ((), (0,)), ((), ()), 4),
+    ((2, 2), (16, 6, 4), ((), (), (0, 1)), ((), (0,), ()), 8),
+    ((2, 2, 2), (6, 5, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4),
+    ((2, 2, 2), (700, 3, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4),      # many row groups, ragged last one
+]
+
+
+@pytest.mark.parametrize("mesh,gshape,src_axes,dst_axes,e", STAGED)
+def test_staged_transpose_kernels(mesh, gshape, src_axes, dst_axes, e):
+    """Short ragged runs gathered into long target rows that are stored to several replicas go through
+    the shared-memory staged kernels (launch variant 5)."""
+    rng = np.random.default_rng(sum(gshape))
+    G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+    src, dst = (gshape, src_axes), (gshape, dst_axes)
+    src_tiles = oracle.reslice(mesh, src, G)
+    want = oracle.reslice(mesh, dst, G)
+    plan, got = run_gpu(mesh, src, dst, e, src_tiles)
+    assert plan.launch_info(0).variant == 5
+    assert_same(got, want, f"staged {mesh} {gshape}")
+    _, got = run_gpu(mesh, src, dst, e, src_tiles, api.FUSE_NONE)
+    assert_same(got, want, f"staged, unfused {mesh} {gshape}")
+
+
 def test_zero_bulk_copy_timeouts_after_everything_above():
     """The bounded waits of the bulk-copy kernels never ran out."""
     torch.cuda.synchronize()
