@@ -149,8 +149,9 @@ void redist_plan_destroy(redist_plan_t *plan);
  *   scratch         DEVICE pointer to at least redist_plan_scratch_bytes(plan) bytes, or NULL when
  *                   that is 0.  Contents are undefined afterwards.
  *   cuda_stream     a cudaStream_t (NULL = default stream) on the current device
- * Ownership: all buffers and the stream belong to the caller.  The call allocates nothing, copies
- * no table to the device (tables travel as kernel parameters) and does not synchronize.  A plan
+ * Ownership: all buffers and the stream belong to the caller.  The call allocates no device memory
+ * (only small host-side tables), copies no table to the device (tables travel as kernel parameters)
+ * and does not synchronize; ENOMEM is returned if a host table cannot be allocated.  A plan
  * may be executed from several host threads at once on different streams and buffers.
  * Errors: EINVAL, ESCRATCH, EALIGN (pointers must be multiples of redist_plan_alignment),
  * EOVERLAP (destination and scratch ranges must be disjoint from each other and from every

@@ -102,23 +102,29 @@ int64_t redist_bulk_timeouts(void)
 redist_status redist_base_offsets(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *type,
                                   int64_t *out_tile, int64_t *out_offsets)
 {
-    if (n_mesh_axes < 0 || n_mesh_axes > REDIST_MAX_MESH_AXES || (n_mesh_axes > 0 && !mesh_shape) || !type ||
-        !out_tile || !out_offsets)
-        return REDIST_EINVAL;
-    i64 N = 1;
-    for (int a = 0; a < n_mesh_axes; ++a) {
-        if (mesh_shape[a] < 1) return REDIST_EINVAL;
-        N *= mesh_shape[a];
-        if (N > REDIST_MAX_DEVICES) return REDIST_EUNSUPPORTED;
+    try {
+        if (n_mesh_axes < 0 || n_mesh_axes > REDIST_MAX_MESH_AXES || (n_mesh_axes > 0 && !mesh_shape) || !type ||
+            !out_tile || !out_offsets)
+            return REDIST_EINVAL;
+        i64 N = 1;
+        for (int a = 0; a < n_mesh_axes; ++a) {
+            if (mesh_shape[a] < 1) return REDIST_EINVAL;
+            N *= mesh_shape[a];
+            if (N > REDIST_MAX_DEVICES) return REDIST_EUNSUPPORTED;
+        }
+        std::vector<i64> tile;
+        redist_status rc = check_type(n_mesh_axes, mesh_shape, type, &tile);
+        if (rc != REDIST_OK) return rc;
+        std::vector<i64> off(size_t(N) * type->rank);
+        base_offsets_of(n_mesh_axes, mesh_shape, type, tile, off.data());
+        std::copy(tile.begin(), tile.end(), out_tile);
+        std::copy(off.begin(), off.end(), out_offsets);
+        return REDIST_OK;
+    } catch (const std::bad_alloc &) {
+        return REDIST_ENOMEM;
+    } catch (...) {
+        return REDIST_EINTERNAL;
     }
-    std::vector<i64> tile;
-    redist_status rc = check_type(n_mesh_axes, mesh_shape, type, &tile);
-    if (rc != REDIST_OK) return rc;
-    std::vector<i64> off(size_t(N) * type->rank);
-    base_offsets_of(n_mesh_axes, mesh_shape, type, tile, off.data());
-    std::copy(tile.begin(), tile.end(), out_tile);
-    std::copy(off.begin(), off.end(), out_offsets);
-    return REDIST_OK;
 }
 
 redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *src,
@@ -278,92 +284,104 @@ size_t redist_plan_describe(const redist_plan_t *plan, char *buf, size_t cap)
 redist_status redist_execute(const redist_plan_t *plan, const void *const *src_shards, void *const *dst_shards,
                              void *scratch, size_t scratch_bytes, void *cuda_stream)
 {
-    if (!plan || !src_shards || !dst_shards) return REDIST_EINVAL;
-    const Plan &p = plan->p;
-    const int N = p.n_devices;
-    if (p.scratch_bytes > 0 && (!scratch || scratch_bytes < size_t(p.scratch_bytes))) return REDIST_ESCRATCH;
-    const uintptr_t amask = uintptr_t(p.alignment) - 1;
-    const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
-    std::vector<Range> ranges;
-    ranges.reserve(size_t(2 * N + 1));
-    for (int d = 0; d < N; ++d) {
-        if (!src_shards[d] || !dst_shards[d]) return REDIST_EINVAL;
-        const uintptr_t s = uintptr_t(src_shards[d]), t = uintptr_t(dst_shards[d]);
-        if ((s & amask) || (t & amask)) return REDIST_EALIGN;
-        ranges.push_back(Range{s, s + uintptr_t(sb), 0});
-        ranges.push_back(Range{t, t + uintptr_t(db), 1});
-    }
-    if (p.scratch_bytes > 0) {
-        if (uintptr_t(scratch) & 255) return REDIST_EALIGN;
-        ranges.push_back(Range{uintptr_t(scratch), uintptr_t(scratch) + uintptr_t(p.scratch_bytes), 1});
-    }
-    if (overlaps(ranges)) return REDIST_EOVERLAP;
+    try {
+        if (!plan || !src_shards || !dst_shards) return REDIST_EINVAL;
+        const Plan &p = plan->p;
+        const int N = p.n_devices;
+        if (p.scratch_bytes > 0 && (!scratch || scratch_bytes < size_t(p.scratch_bytes))) return REDIST_ESCRATCH;
+        const uintptr_t amask = uintptr_t(p.alignment) - 1;
+        const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
+        std::vector<Range> ranges;
+        ranges.reserve(size_t(2 * N + 1));
+        for (int d = 0; d < N; ++d) {
+            if (!src_shards[d] || !dst_shards[d]) return REDIST_EINVAL;
+            const uintptr_t s = uintptr_t(src_shards[d]), t = uintptr_t(dst_shards[d]);
+            if ((s & amask) || (t & amask)) return REDIST_EALIGN;
+            ranges.push_back(Range{s, s + uintptr_t(sb), 0});
+            ranges.push_back(Range{t, t + uintptr_t(db), 1});
+        }
+        if (p.scratch_bytes > 0) {
+            if (uintptr_t(scratch) & 255) return REDIST_EALIGN;
+            ranges.push_back(Range{uintptr_t(scratch), uintptr_t(scratch) + uintptr_t(p.scratch_bytes), 1});
+        }
+        if (overlaps(ranges)) return REDIST_EOVERLAP;
 
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    auto buffer = [&](BufKind kind, int32_t dev) -> char * {
-        switch (kind) {
-        case BUF_SRC: return static_cast<char *>(const_cast<void *>(src_shards[dev]));
-        case BUF_DST: return static_cast<char *>(dst_shards[dev]);
-        case BUF_SCRATCH0: return static_cast<char *>(scratch) + i64(dev) * p.slot_bytes;
-        case BUF_SCRATCH1: return static_cast<char *>(scratch) + (i64(N) + dev) * p.slot_bytes;
-        default: return static_cast<char *>(scratch);
+        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+        auto buffer = [&](BufKind kind, int32_t dev) -> char * {
+            switch (kind) {
+            case BUF_SRC: return static_cast<char *>(const_cast<void *>(src_shards[dev]));
+            case BUF_DST: return static_cast<char *>(dst_shards[dev]);
+            case BUF_SCRATCH0: return static_cast<char *>(scratch) + i64(dev) * p.slot_bytes;
+            case BUF_SCRATCH1: return static_cast<char *>(scratch) + (i64(N) + dev) * p.slot_bytes;
+            default: return static_cast<char *>(scratch);
+            }
+        };
+        std::vector<const char *> stab;
+        std::vector<char *> dtab;
+        for (const Launch &L : p.launches) {
+            stab.resize(L.src_holder.size());
+            dtab.resize(L.dst_devs.size());
+            for (size_t t = 0; t < stab.size(); ++t) stab[t] = buffer(L.from, L.src_holder[t] < 0 ? 0 : L.src_holder[t]);
+            for (size_t t = 0; t < dtab.size(); ++t) dtab[t] = buffer(L.to, L.dst_devs[t] < 0 ? 0 : L.dst_devs[t]);
+            if (L.geo.n_items == 0) continue;
+            cudaError_t ce = launch_copy(L.kernel, L.geo, stab.data(), int(stab.size()), dtab.data(), int(dtab.size()),
+                                         grid_for(L.geo), stream);
+            if (ce != cudaSuccess) {
+                tl_cuda_error = int(ce);
+                return REDIST_ECUDA;
+            }
         }
-    };
-    std::vector<const char *> stab;
-    std::vector<char *> dtab;
-    for (const Launch &L : p.launches) {
-        stab.resize(L.src_holder.size());
-        dtab.resize(L.dst_devs.size());
-        for (size_t t = 0; t < stab.size(); ++t) stab[t] = buffer(L.from, L.src_holder[t] < 0 ? 0 : L.src_holder[t]);
-        for (size_t t = 0; t < dtab.size(); ++t) dtab[t] = buffer(L.to, L.dst_devs[t] < 0 ? 0 : L.dst_devs[t]);
-        if (L.geo.n_items == 0) continue;
-        cudaError_t ce = launch_copy(L.kernel, L.geo, stab.data(), int(stab.size()), dtab.data(), int(dtab.size()),
-                                     grid_for(L.geo), stream);
-        if (ce != cudaSuccess) {
-            tl_cuda_error = int(ce);
-            return REDIST_ECUDA;
-        }
+        return REDIST_OK;
+    } catch (const std::bad_alloc &) {
+        return REDIST_ENOMEM;
+    } catch (...) {
+        return REDIST_EINTERNAL;
     }
-    return REDIST_OK;
 }
 
 redist_status redist_execute_host(const redist_plan_t *plan, const void *const *src_host, void *const *dst_host,
                                   void *dev_src, size_t dev_src_bytes, void *dev_dst, size_t dev_dst_bytes,
                                   void *scratch, size_t scratch_bytes, void *cuda_stream)
 {
-    if (!plan || !src_host || !dst_host || !dev_src || !dev_dst) return REDIST_EINVAL;
-    const Plan &p = plan->p;
-    const int N = p.n_devices;
-    if (dev_src_bytes < redist_plan_staging_bytes(plan, 0) || dev_dst_bytes < redist_plan_staging_bytes(plan, 1))
-        return REDIST_ESCRATCH;
-    if ((uintptr_t(dev_src) & 255) || (uintptr_t(dev_dst) & 255)) return REDIST_EALIGN;
-    const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
-    const i64 sp = (sb + 255) / 256 * 256, dp = (db + 255) / 256 * 256;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    std::vector<const void *> s(N);
-    std::vector<void *> t(N);
-    for (int d = 0; d < N; ++d) {
-        if (!src_host[d] || !dst_host[d]) return REDIST_EINVAL;
-        s[d] = static_cast<char *>(dev_src) + d * sp;
-        t[d] = static_cast<char *>(dev_dst) + d * dp;
-    }
-    for (int d = 0; d < N; ++d) {
-        cudaError_t ce = cudaMemcpyAsync(const_cast<void *>(s[d]), src_host[d], size_t(sb), cudaMemcpyHostToDevice, stream);
-        if (ce != cudaSuccess) {
-            tl_cuda_error = int(ce);
-            return REDIST_ECUDA;
+    try {
+        if (!plan || !src_host || !dst_host || !dev_src || !dev_dst) return REDIST_EINVAL;
+        const Plan &p = plan->p;
+        const int N = p.n_devices;
+        if (dev_src_bytes < redist_plan_staging_bytes(plan, 0) || dev_dst_bytes < redist_plan_staging_bytes(plan, 1))
+            return REDIST_ESCRATCH;
+        if ((uintptr_t(dev_src) & 255) || (uintptr_t(dev_dst) & 255)) return REDIST_EALIGN;
+        const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
+        const i64 sp = (sb + 255) / 256 * 256, dp = (db + 255) / 256 * 256;
+        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+        std::vector<const void *> s(N);
+        std::vector<void *> t(N);
+        for (int d = 0; d < N; ++d) {
+            if (!src_host[d] || !dst_host[d]) return REDIST_EINVAL;
+            s[d] = static_cast<char *>(dev_src) + d * sp;
+            t[d] = static_cast<char *>(dev_dst) + d * dp;
         }
-    }
-    redist_status rc = redist_execute(plan, s.data(), t.data(), scratch, scratch_bytes, cuda_stream);
-    if (rc != REDIST_OK) return rc;
-    for (int d = 0; d < N; ++d) {
-        cudaError_t ce = cudaMemcpyAsync(dst_host[d], t[d], size_t(db), cudaMemcpyDeviceToHost, stream);
-        if (ce != cudaSuccess) {
-            tl_cuda_error = int(ce);
-            return REDIST_ECUDA;
+        for (int d = 0; d < N; ++d) {
+            cudaError_t ce = cudaMemcpyAsync(const_cast<void *>(s[d]), src_host[d], size_t(sb), cudaMemcpyHostToDevice, stream);
+            if (ce != cudaSuccess) {
+                tl_cuda_error = int(ce);
+                return REDIST_ECUDA;
+            }
         }
+        redist_status rc = redist_execute(plan, s.data(), t.data(), scratch, scratch_bytes, cuda_stream);
+        if (rc != REDIST_OK) return rc;
+        for (int d = 0; d < N; ++d) {
+            cudaError_t ce = cudaMemcpyAsync(dst_host[d], t[d], size_t(db), cudaMemcpyDeviceToHost, stream);
+            if (ce != cudaSuccess) {
+                tl_cuda_error = int(ce);
+                return REDIST_ECUDA;
+            }
+        }
+        return REDIST_OK;
+    } catch (const std::bad_alloc &) {
+        return REDIST_ENOMEM;
+    } catch (...) {
+        return REDIST_EINTERNAL;
     }
-    return REDIST_OK;
 }
 
 }  // extern "C"
