@@ -64,6 +64,8 @@ struct Search {
     i64 M;                         // max(localsize src, localsize dst)
     std::vector<int> tgt_exps;     // target exponents [r*np]
 
+    bool allow_over = false;       // ignore REDIST_NO_OVERPARTITION (fallback when it leaves no path)
+
     explicit Search(const Plan &plan) : p(plan), r(plan.rank), np(0), M(0) {}
 
     i64 pow_of(const std::vector<int> &e) const
@@ -128,7 +130,7 @@ struct Search {
         Key start = key_of(p.src_pax, 0);
         Key goal = key_of(p.dst_pax, 0);
         tgt_exps.assign(goal.begin(), goal.end() - 1);
-        const bool no_over = (p.flags & REDIST_NO_OVERPARTITION) != 0;
+        const bool no_over = (p.flags & REDIST_NO_OVERPARTITION) != 0 && !allow_over;
 
         struct Info {
             i64 cost;
@@ -206,6 +208,7 @@ struct Search {
                         if (c[i] % m) return;
                         if (no_over)
                             for (int q = 0; q < np; ++q) {
+                                if (e[q] == 0) continue;
                                 int tgt_used = 0;
                                 for (int k = 0; k < r; ++k) tgt_used += tgt_exps[k * np + q];
                                 if (key[i * np + q] + e[q] > tgt_exps[i * np + q] || used[q] + e[q] > tgt_used)
@@ -595,7 +598,12 @@ redist_status synthesize(Plan &p)
     // 2. shortest paths over weak types
     Search S(p);
     std::vector<std::vector<WeakStep>> paths;
-    if (!S.run(paths, 64)) return REDIST_EINTERNAL;
+    if (!S.run(paths, 64)) {
+        // the over-partitioning ban may leave no path inside the memory bound: drop it rather than fail
+        S.allow_over = true;
+        S.P.clear();
+        if (!S.run(paths, 64)) return REDIST_EINTERNAL;
+    }
 
     // 3. lowering; the equal-cost shortest paths (e.g. the orders of commuting alltoalls) differ in
     //    where the axes end up: keep the first that reaches the target assignment without a

@@ -342,3 +342,29 @@ def test_planner_throughput_on_evaluation_shaped_problems():
         p.close()
     total = time.perf_counter() - t0
     assert worst < 0.25 and total / len(ws) < 0.05, (worst, total)
+
+
+def test_no_overpartition_flag_only_filters_the_axes_it_slices():
+    """Regression: the ban on over-partitioning must look only at the primes a dynslice introduces.
+    [7, 4{b}4... a dimension sharded 5 ways that has to end sharded 3 ways still needs dynslice(3)."""
+    mesh = (3, 2, 5)
+    src, dst = ((7, 4, 30), ((), (1,), (2,))), ((7, 4, 30), ((), (1,), (0,)))
+    a = check_plan(mesh, src, dst, 4, api.FUSE_ADJACENT)
+    b = check_plan(mesh, src, dst, 4, api.FUSE_ADJACENT | api.NO_OVERPARTITION)
+    assert [s["kind"] for s in a["steps"]] == [s["kind"] for s in b["steps"]]
+
+
+def test_random_plans_never_fail_in_any_mode():
+    """2000 random problems (odd primes, size-1 axes, rank up to 6) x four flag settings: a plan exists,
+    respects the memory bound and has at most one permutation."""
+    rng = np.random.default_rng(20211201)
+    meshes = [(2,), (6,), (2, 3), (4, 6), (6, 5), (2, 3, 2), (3, 2, 5), (4, 4, 4), (1, 2, 3), (2, 2, 2, 2),
+              (2, 3, 5, 7), (12,), (9, 4), (2, 2, 3, 3)]
+    for it in range(2000):
+        mesh = meshes[it % len(meshes)]
+        src, dst = random_problem(rng, mesh, max_rank=6, mult=7)
+        for flags in (api.FUSE_ADJACENT, api.FUSE_NONE, api.NAIVE, api.NO_OVERPARTITION):
+            p = api.Plan(mesh, src, dst, int(rng.choice([1, 2, 4, 8, 16])), flags)
+            assert p.height <= max(p.local_elems(0), p.local_elems(1))
+            assert p.step_kinds().count("allpermute") <= 1
+            p.close()
