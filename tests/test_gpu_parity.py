@@ -87,11 +87,12 @@ def test_random_sweep_reduced_shape(mode):
 def test_random_problems_small_and_odd():
     """Odd primes, all element sizes, element-sized runs, several steps with scratch ping-pong."""
     rng = np.random.default_rng(2112)
-    meshes = [(2, 3), (4, 6), (3, 3, 2), (2, 2, 2, 2), (6,), (5, 2)]
+    meshes = [(2, 3), (4, 6), (3, 3, 2), (2, 2, 2, 2), (6,), (5, 2), (4, 4, 4), (1, 2, 3), (9, 4), (16,)]
     n_multi = 0
-    for t in range(120):
+    variants = set()
+    for t in range(600):
         mesh = meshes[t % len(meshes)]
-        rank = int(rng.integers(1, 4))
+        rank = int(rng.integers(1, 5))
 
         def draw():
             per = [[] for _ in range(rank)]
@@ -106,9 +107,11 @@ def test_random_problems_small_and_odd():
         for k in range(rank):
             f1 = int(np.prod([mesh[a] for a in a1[k]], dtype=np.int64))
             f2 = int(np.prod([mesh[a] for a in a2[k]], dtype=np.int64))
-            gshape.append(int(np.lcm(f1, f2)) * int(rng.integers(1, 6)))
+            gshape.append(int(np.lcm(f1, f2)) * int(rng.integers(1, 9)))
         gshape = tuple(gshape)
-        e = int(rng.choice([1, 2, 4, 8, 16]))
+        e = int(rng.choice([1, 2, 4, 4, 8, 16]))
+        if int(np.prod(gshape)) * e > (4 << 20):
+            continue
         G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
         src, dst = (gshape, a1), (gshape, a2)
         src_tiles = oracle.reslice(mesh, src, G)
@@ -116,8 +119,10 @@ def test_random_problems_small_and_odd():
         mode = MODES[t % 4]
         plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
         n_multi += plan.num_launches >= 3
+        variants.update(plan.launch_info(q).variant for q in range(plan.num_launches))
         assert_same(got, want, f"{mesh} {src} -> {dst} e={e} mode={mode}")
     assert n_multi > 0          # the two-slot scratch ping-pong was exercised
+    assert variants >= {0, 2, 3, 4, 5}   # rows, ragged chunks, units, bulk and staged kernels all ran
 
 
 def test_round_trip_on_the_gpu():
