@@ -19,16 +19,19 @@
 // item is one TMA bulk copy global -> shared (cp.async.bulk, byte-counted completion on an mbarrier)
 // and one bulk copy shared -> global per target replica, issued by a few threads (bulk_body below;
 // measured 1-3 % faster than the register path on every benchmark configuration).  Everything else
-// uses the register kernels:
-//
-// Three item shapes (CopyGeometry::mode).  kModeRows, aligned runs of at most 4 KiB: a block of 256
-// threads covers rows_per_pass rows of `lanes` chunks; a thread keeps its column and walks down the
-// rows of its work item, kUnroll independent loads in flight before the stores.  kModeChunks, all
-// other runs of 256 bytes or more: the rows of an item are decoded once into shared memory and all
-// threads walk the (row, chunk) space of the item with a flat index.  kModeUnits, ragged runs below
-// 256 bytes: the same flat walk over (row, piece of unit_bytes).  Index decoding uses multiply-shift
-// division by host-computed constants; the per-item decode (box -> tiles and base offsets) is
-// amortised over ~32 KiB of data.
+// uses the register kernels, in four item shapes (CopyGeometry::mode):
+//   kModeRows    aligned runs below the bulk threshold: a block of 256 threads covers rows_per_pass
+//                rows of `lanes` chunks; a thread keeps its column and walks down the rows of its work
+//                item, kUnroll independent loads in flight before the stores.
+//   kModeChunks  ragged runs of 256 bytes or more (and aligned long runs when bulk copies are switched
+//                off): the rows of an item are decoded once into shared memory and all threads walk the
+//                (row, chunk) space of the item with a flat index.
+//   kModeUnits   ragged runs below 256 bytes: the same flat walk over pieces of unit_bytes.
+//   kModeStaged  ragged runs below 256 bytes that are gathered into long target rows stored to two or
+//                more replicas: the rows are assembled in shared memory and written whole.
+// Index decoding uses multiply-shift division by host-computed constants; the per-item decode (box ->
+// tiles and base offsets) is amortised over ~32 KiB of data.  Every kernel starts with
+// griddepcontrol.wait / launch_dependents (programmatic dependent launch).
 #include <cuda_runtime.h>
 
 #include <cstdlib>
