@@ -335,6 +335,19 @@ def run_ours(args):
         run_e2e(torch, api, ws, flags, max(3, min(args.steps, 10)), world, dist)
     if rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(ws)
+    if rank == 0 and world == 1 and args.fuse == "adjacent":
+        # comparison points on the same workload (short runs, outside the headline region): the
+        # sequence run collective by collective through scratch, and the naive gather-then-slice method
+        del legs
+        torch.cuda.empty_cache()
+        for key, fl in (("unfused", api.FUSE_NONE), ("naive_gpu_baseline", api.NAIVE)):
+            cmp_legs = [DeviceLeg(w, fl, torch, api, gen) for w in ws]
+            ms, _ = time_legs(torch, cmp_legs, 50, 3)
+            line[key] = {"value": round(step_bytes / (ms / 50 * 1e-3) / 1e9, 1), "unit": UNIT,
+                         "launches_per_step": sum(l.launches for l in cmp_legs),
+                         "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in cmp_legs)}
+            del cmp_legs
+            torch.cuda.empty_cache()
     if rank == 0 and world == 1 and args.others:
         line["others"] = run_others(torch, api, gen, args)
     if rank == 0:
