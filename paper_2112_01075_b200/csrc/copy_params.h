@@ -16,18 +16,21 @@
 // the same memory sectors and partial-sector writes merge in L2 instead of being written back alone;
 // then come the row groups of a box, then the boxes.
 //
+// Aligned items whose row segments are at least 512 bytes (`bulk == 1`) are moved by TMA bulk copies
+// through shared memory instead of by the register kernels; the item geometry is the same.
+//
 // Work items, by `mode`:
 //   kModeRows   aligned runs of at most 256 chunks: a block covers rows_per_pass rows of `lanes`
 //               chunks per pass; an item is rows_per_item rows; every thread decodes its own rows.
 //   kModeChunks all other runs of at least 256 bytes: an item is rows_per_item rows times one column
 //               block of per_block chunks; the rows are decoded once into shared memory and all
 //               threads walk the (row, chunk) space with a flat index.
-//   kModeStaged ragged runs shorter than 256 bytes where the rows of one side are `stage_w` runs long
-//               and come from (or go to) stage_w different tiles of the other side -- the block
-//               transpose of an alltoall or the concatenation of an allgather along the last
-//               differing dimension.  An item stages rows_per_item such rows in shared memory: the
-//               short side moves piece by piece (a thread per piece, 4-byte words), the long side in
-//               16-byte chunks, so the long rows are read or written whole.
+//   kModeStaged ragged runs shorter than 256 bytes where the rows of the target are inner_mul runs
+//               long, come from inner_mul different source tiles and are stored to two or more
+//               replicas -- the concatenation of an allgather or the block transpose of an alltoall
+//               along the last differing dimension.  An item stages rows_per_item such rows in shared
+//               memory: the pieces are loaded by a few threads each in 4-byte words, the rows are
+//               written in 16-byte chunks, whole.
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
 //               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
 //               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
@@ -57,7 +60,7 @@ struct CopyGeometry {
     uint32_t fanout;                 // target replicas per box
     uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
     uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
-    uint32_t mode;                   // kModeRows, kModeChunks or kModeUnits
+    uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits or kModeStaged
     uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes)
     uint64_t run_bytes;              // contiguous run
     uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
