@@ -615,7 +615,7 @@ __device__ __forceinline__ void bulk_body(const CopyParams<NT> &P)
                          : "memory");
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 }
 
