@@ -222,7 +222,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         // table row carries all the runs of the innermost row digit
         const bool units = run_bytes < 256;
         i64 tab_inner = 1, tab_rows = n_rows;
-        if (units && run_bytes <= 16 && !rows.empty()) {   // only when a table of rows could not fill an item
+        if (units && run_bytes <= 16 && !rows.empty() && rows.back().n * (run_bytes / vec) < (1ll << 30)) {
+            // only when a table of rows could not fill an item (and the payload index fits 32 bits)
             tab_inner = rows.back().n;
             tab_rows = n_rows / tab_inner;
         }
