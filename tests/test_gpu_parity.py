@@ -455,6 +455,32 @@ def test_staged_transpose_kernels(mesh, gshape, src_axes, dst_axes, e):
     assert_same(got, want, f"staged, unfused {mesh} {gshape}")
 
 
+def test_four_gib_tiles_need_64_bit_offsets():
+    """u32 [32768, 32768] (4 GiB, value = global linear index) on two devices: replicated -> column
+    sharded reads at offsets beyond 2^32 inside a tile, column sharded -> replicated writes there."""
+    mesh, g = (2,), (32768, 32768)
+    G = wl.global_array_bytes(g, 4, "linear_u32", 0)
+    repl, cols = (g, ((), ())), (g, ((), (0,)))
+    oracle.set_threads(oracle.max_threads())
+    try:
+        col_tiles = oracle.reslice(mesh, cols, G)
+    finally:
+        oracle.set_threads(1)
+    one = torch.from_numpy(G.reshape(-1)).cuda()
+    plan = api.Plan(mesh, repl, cols, 4)
+    nb = plan.local_elems(1) * 4
+    out = [torch.empty(nb, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    plan.execute([one, one], out)                      # replicas alias one 4 GiB buffer
+    torch.cuda.synchronize()
+    assert_same([t.cpu().numpy() for t in out], col_tiles, "replicated -> columns")
+    back = api.Plan(mesh, cols, repl, 4)
+    full = [torch.empty(4 * 2**30, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    back.execute(out, full)
+    torch.cuda.synchronize()
+    for d in range(2):
+        assert torch.equal(full[d], one), f"columns -> replicated, device {d}"
+
+
 def test_zero_bulk_copy_timeouts_after_everything_above():
     """The bounded waits of the bulk-copy kernels never ran out."""
     torch.cuda.synchronize()
