@@ -48,6 +48,7 @@ constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: o
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
 constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeStaged = 3;
 constexpr int kStageRows = 256;        // rows of one item of the staged transpose
+constexpr int kRaggedBulkRows = 256;   // rows of one item of the ragged bulk-in kernels
 
 // Division of a 31-bit unsigned number by a constant: n / d == umulhi(n, mul) >> shr (d > 1).
 struct FastDiv {
@@ -61,7 +62,8 @@ struct CopyGeometry {
     uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
     uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
     uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits or kModeStaged
-    uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes)
+    uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes);
+                                     // 2: ragged chunk walk whose loads are bulk copies into shared memory
     uint64_t run_bytes;              // contiguous run
     uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
     uint32_t rows_per_pass;          // kModeRows: kBlockThreads / lanes
@@ -77,7 +79,7 @@ struct CopyGeometry {
     uint32_t inner_span;             // units of that digit per long row (m1 * m2)
     uint32_t inner_mul;              // units per item along that digit: 1, or stage_w in kModeStaged
     uint32_t stage_long_dst;         // kModeStaged: 1 the target has the long rows, 0 the source
-    uint32_t stage_pitch;            // kModeStaged: bytes between staged rows in shared memory
+    uint32_t stage_pitch;            // kModeStaged, bulk == 2: bytes between staged rows in shared memory
     uint32_t stage_ts;               // kModeStaged: tile-index stride between the pieces on the short side
     uint32_t stage_rows_log2;        // kModeStaged: log2(rows_per_item)
     uint32_t stage_tpp_log2;         // kModeStaged: log2(threads per piece on the short side)

@@ -157,6 +157,16 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         fan = p.n_devices / nt;
     }
     const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
+    // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
+    // thread, the item staged in at most 47 KiB of shared memory)
+    static const bool kBulk = [] {
+        const char *v = std::getenv("REDIST_BULK");      // tuning knob: REDIST_BULK=0 keeps aligned runs on the register path
+        return !v || std::atoi(v) > 0;
+    }();
+    static const i64 kBulkMin = [] {
+        const char *v = std::getenv("REDIST_BULK_MIN");  // tuning knob: shortest segment moved by a bulk copy
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 512);
+    }();
     const i64 max_chunks = run_bytes / 16;           // whole 16-byte chunks a run can hold
     if (max_chunks >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     i64 ipb;
@@ -167,6 +177,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const char *v = std::getenv("REDIST_STAGED");    // tuning knob: REDIST_STAGED=0 disables the staged transpose
         return !v || std::atoi(v) > 0;
     }();
+    bool ragged_bulk = false;
     i64 stage_w = 0;
     if (kStaged && !G.aligned && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu &&
         m1[kp] == 1 && m2[kp] > 1 && fan >= 2) {
@@ -233,6 +244,18 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const i64 ncb = std::max<i64>(1, (per_row + cpb - 1) / cpb);
         i64 rpi = std::max<i64>(1, std::min<i64>(kMaxRowsFlat, kItemBytes / (cpb * piece)));
         rpi = std::min<i64>(rpi, tab_rows);
+        if (!units && !G.aligned && kBulk) {
+            // ragged rows: each row segment is loaded by one bulk copy of the 16-byte blocks that cover
+            // it (up to 15 bytes before and after, plus the ragged head), then shifted out of shared memory
+            const i64 pitch = cpb * 16 + 64;
+            static const i64 kRaggedKb = [] {
+                const char *v = std::getenv("REDIST_RBULK_KB");   // tuning knob: shared-memory tile of a ragged bulk item, KiB (at most 38)
+                return i64(v && std::atoi(v) > 0 ? std::min(std::atoi(v), 38) : 38);
+            }();
+            rpi = std::max<i64>(1, std::min<i64>(rpi, std::min<i64>(kRaggedBulkRows, kRaggedKb * 1024 / pitch)));
+            ragged_bulk = true;
+            G.stage_pitch = uint32_t(pitch);
+        }
         G.mode = units ? kModeUnits : kModeChunks;
         G.rows = uint32_t(tab_rows);
         G.n_row_tab = uint32_t(tab_inner > 1 ? rows.size() - 1 : rows.size());
@@ -243,17 +266,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.col_blocks = make_div(uint32_t(ncb));
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     }
-    // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
-    // thread, the item staged in at most 47 KiB of shared memory)
-    static const bool kBulk = [] {
-        const char *v = std::getenv("REDIST_BULK");      // tuning knob: REDIST_BULK=0 keeps aligned runs on the register path
-        return !v || std::atoi(v) > 0;
-    }();
-    static const i64 kBulkMin = [] {
-        const char *v = std::getenv("REDIST_BULK_MIN");  // tuning knob: shortest segment moved by a bulk copy
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 512);
-    }();
-    G.bulk = 0;
+    G.bulk = ragged_bulk ? 2u : 0u;
     if (kBulk && G.aligned && G.mode != kModeUnits) {
         const i64 seg = G.mode == kModeRows ? run_bytes : i64(G.per_block) * 16;
         if (seg >= kBulkMin && G.rows_per_item <= uint32_t(kBulkThreads) && seg * G.rows_per_item <= 47 * 1024) G.bulk = 1;

@@ -633,6 +633,165 @@ REDIST_DEFINE_BULK_KERNEL(redist_allgather_bulk_kernel)
 REDIST_DEFINE_BULK_KERNEL(redist_allpermute_bulk_kernel)
 REDIST_DEFINE_BULK_KERNEL(redist_fused_bulk_kernel)
 
+// ---- ragged bulk-in (bulk == 2): the ragged chunk walk with its loads done by TMA ----------------
+// Same items as the ragged chunk walk.  For every row of the item one thread posts the byte count on
+// the mbarrier and issues one bulk copy of the 16-byte blocks that cover the row's source bytes for
+// this column block; when all rows have landed, the threads walk (row, chunk) as before but read the
+// source chunk from shared memory (two aligned 16-byte reads and a funnel shift), so no thread ever
+// waits on a global load.  Ragged heads and tails are copied from shared memory in unit pieces.
+struct RaggedRow {
+    uint32_t base;           // shared-memory offset of the row-relative source byte 0 (may wrap below the slot)
+    uint32_t head, chunks;   // bytes before the first target-aligned chunk, whole chunks of the run
+    uint32_t pad;
+};
+
+__device__ __forceinline__ uint4 lds_shifted(const unsigned char *tile, uint32_t at)
+{
+    const uint32_t m = at & 15u;
+    const uint4 *p = reinterpret_cast<const uint4 *>(tile + (at - m));
+    const uint4 a = p[0];
+    if (m == 0) return a;
+    const uint4 b = p[1];
+    const uint32_t bs = (m & 3u) * 8u;
+    uint4 o;
+    switch (m >> 2) {
+    case 0:
+        o.x = __funnelshift_r(a.x, a.y, bs); o.y = __funnelshift_r(a.y, a.z, bs);
+        o.z = __funnelshift_r(a.z, a.w, bs); o.w = __funnelshift_r(a.w, b.x, bs);
+        break;
+    case 1:
+        o.x = __funnelshift_r(a.y, a.z, bs); o.y = __funnelshift_r(a.z, a.w, bs);
+        o.z = __funnelshift_r(a.w, b.x, bs); o.w = __funnelshift_r(b.x, b.y, bs);
+        break;
+    case 2:
+        o.x = __funnelshift_r(a.z, a.w, bs); o.y = __funnelshift_r(a.w, b.x, bs);
+        o.z = __funnelshift_r(b.x, b.y, bs); o.w = __funnelshift_r(b.y, b.z, bs);
+        break;
+    default:
+        o.x = __funnelshift_r(a.w, b.x, bs); o.y = __funnelshift_r(b.x, b.y, bs);
+        o.z = __funnelshift_r(b.y, b.z, bs); o.w = __funnelshift_r(b.z, b.w, bs);
+        break;
+    }
+    return o;
+}
+
+template <int NT>
+__device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
+{
+    extern __shared__ __align__(128) unsigned char tile[];
+    __shared__ RowEntry rowtab[kRaggedBulkRows];
+    __shared__ RaggedRow rinfo[kRaggedBulkRows];
+    __shared__ __align__(8) unsigned long long mbar_storage;
+    const CopyGeometry &g = P.g;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t fanout = g.fanout;
+    const uint32_t len = uint32_t(g.run_bytes);       // chunk mode with col blocks: runs below 2^32 bytes here
+    const uint32_t cpb = g.per_block;
+    const uint32_t pitch = g.stage_pitch;
+    const uint32_t mbar = smem_addr(&mbar_storage);
+    const uint32_t item = blockIdx.x;                 // one item per block (the mbarrier is used once)
+    if (item >= g.n_items) return;
+    const BoxBase b = decode_box(P, item);
+    const uint32_t group = fdiv(b.part, g.col_blocks);
+    const uint32_t cb = b.part - group * g.col_blocks.d;
+    const bool first = cb == 0, last = cb + 1 == g.col_blocks.d;
+    const uint32_t c0 = cb * cpb;
+    const uint32_t row0 = group * g.rows_per_item;
+    const uint32_t nr = min(g.rows_per_item, g.rows - row0);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(nr) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    for (uint32_t r = tid; r < nr; r += kBlockThreads) {
+        RowEntry e;
+        row_offsets(g, row0 + r, e.s1, e.s2, int(g.n_row_tab));
+        rowtab[r] = e;
+        uint32_t head, chunks;
+        split_run(len, b.o2 + e.s2, head, chunks);
+        // row-relative source bytes [b0, b1) belong to this column block
+        const uint32_t b0 = first ? 0u : min(len, head + (c0 << 4));
+        const uint32_t b1 = last ? len : min(len, head + ((c0 + cpb) << 4));
+        const char *src = b.sbase + e.s1 + b0;
+        const uint32_t m = uint32_t(reinterpret_cast<uintptr_t>(src)) & 15u;
+        RaggedRow ri;
+        ri.base = r * pitch + m - b0;                 // unsigned wrap-around is intended: base + x is used for x >= b0
+        ri.head = head;
+        ri.chunks = chunks;
+        ri.pad = 0;
+        rinfo[r] = ri;
+        if (b1 > b0) {
+            const uint32_t bytes = (m + (b1 - b0) + 15u) & ~15u;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(tile) + r * pitch), "l"(src - m), "r"(bytes), "r"(mbar)
+                         : "memory");
+        } else {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+        }
+    }
+    __syncthreads();
+    if (!mbar_wait_bounded(mbar, 0, 1u << 18)) {
+        if (tid == 0) atomicAdd(&g_bulk_timeouts, 1u);
+        mbar_wait_bounded(mbar, 0, 1u << 18);
+        return;
+    }
+    const uint32_t total = nr * cpb;
+    for (uint32_t idx = tid; idx < total; idx += kBlockThreads) {
+        const uint32_t r = fdiv(idx, g.per_block_div);
+        const uint32_t j = c0 + (idx - r * cpb);
+        const RaggedRow ri = rinfo[r];
+        if (j < ri.chunks) {
+            const uint32_t x = ri.head + (j << 4);
+            const uint4 v = lds_shifted(tile, ri.base + x);
+            const int64_t doff = b.o2 + rowtab[r].s2 + x;
+            for (uint32_t f = 0; f < fanout; ++f) st_stream(reinterpret_cast<uint4 *>(b.dtab[f] + doff), v);
+        }
+    }
+    // ragged ends out of shared memory: head with the first column block, tail with the last
+    const uint32_t unit = g.unit_bytes;
+    const uint32_t slots = 16u / unit - 1u;
+    const uint32_t ends = (first ? 1u : 0u) + (last ? 1u : 0u);
+    for (uint32_t idx = tid; idx < nr * slots * ends; idx += kBlockThreads) {
+        const uint32_t r = idx / (slots * ends);
+        const uint32_t w = idx - r * (slots * ends);
+        const bool is_head = first && w < slots;
+        const uint32_t slot = is_head ? w : (first ? w - slots : w);
+        const RaggedRow ri = rinfo[r];
+        const uint32_t toff = ri.head + (ri.chunks << 4);
+        const uint32_t count = is_head ? ri.head / unit : (len - toff) / unit;
+        if (slot < count) {
+            const uint32_t x = (is_head ? 0u : toff) + slot * unit;
+            const unsigned char *sp = tile + (ri.base + x);
+            const int64_t doff = b.o2 + rowtab[r].s2 + x;
+            for (uint32_t f = 0; f < fanout; ++f) {
+                char *dp = b.dtab[f] + doff;
+                switch (unit) {
+                case 8: *reinterpret_cast<uint2 *>(dp) = *reinterpret_cast<const uint2 *>(sp); break;
+                case 4: *reinterpret_cast<uint32_t *>(dp) = *reinterpret_cast<const uint32_t *>(sp); break;
+                case 2: *reinterpret_cast<uint16_t *>(dp) = *reinterpret_cast<const uint16_t *>(sp); break;
+                default: *reinterpret_cast<uint8_t *>(dp) = *sp; break;
+                }
+            }
+        }
+    }
+}
+
+#define REDIST_DEFINE_RAGGED_BULK_KERNEL(NAME)                                                       \
+    template <int NT>                                                                                \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
+    {                                                                                                \
+        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
+        ragged_bulk_body<NT>(P);                                                                     \
+    }
+
+REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_dynslice_ragged_bulk_kernel)
+REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_alltoall_ragged_bulk_kernel)
+REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_allgather_ragged_bulk_kernel)
+REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_allpermute_ragged_bulk_kernel)
+REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_fused_ragged_bulk_kernel)
+
 #define REDIST_DEFINE_STAGED_KERNEL(NAME)                                                            \
     template <bool LONG_DST, int NT>                                                                 \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
@@ -694,6 +853,27 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
     P.g = geo;
     for (int i = 0; i < n_src; ++i) P.src[i] = src_tab[i];
     for (int i = 0; i < n_dst; ++i) P.dst[i] = dst_tab[i];
+    if (geo.bulk == 2) {
+        void (*fn)(const CopyParams<NT>) = nullptr;
+        switch (kernel) {
+        case 0: case 7: fn = redist_dynslice_ragged_bulk_kernel<NT>; break;
+        case 1: fn = redist_alltoall_ragged_bulk_kernel<NT>; break;
+        case 2: case 6: fn = redist_allgather_ragged_bulk_kernel<NT>; break;
+        case 3: case 4: fn = redist_allpermute_ragged_bulk_kernel<NT>; break;
+        default: fn = redist_fused_ragged_bulk_kernel<NT>; break;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(geo.n_items);
+        cfg.blockDim = dim3(kBlockThreads);
+        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fn, P);
+    }
     if (geo.bulk) {
         const uint64_t seg = geo.mode == kModeRows ? geo.run_bytes : uint64_t(geo.per_block) * 16u;
         {

@@ -84,13 +84,14 @@ def test_random_sweep_reduced_shape(mode):
         assert_same(got, want, w.name + " " + w.src.notation(w.mesh_shape) + "->" + w.dst.notation(w.mesh_shape))
 
 
-def test_random_problems_small_and_odd():
-    """Odd primes, all element sizes, element-sized runs, several steps with scratch ping-pong."""
+def random_problems_small_and_odd(n_problems):
+    """Odd primes, all element sizes, element-sized runs, several steps with scratch ping-pong.
+    Returns the set of kernel variants that ran."""
     rng = np.random.default_rng(2112)
     meshes = [(2, 3), (4, 6), (3, 3, 2), (2, 2, 2, 2), (6,), (5, 2), (4, 4, 4), (1, 2, 3), (9, 4), (16,)]
     n_multi = 0
     variants = set()
-    for t in range(600):
+    for t in range(n_problems):
         mesh = meshes[t % len(meshes)]
         rank = int(rng.integers(1, 5))
 
@@ -122,7 +123,28 @@ def test_random_problems_small_and_odd():
         variants.update(plan.launch_info(q).variant for q in range(plan.num_launches))
         assert_same(got, want, f"{mesh} {src} -> {dst} e={e} mode={mode}")
     assert n_multi > 0          # the two-slot scratch ping-pong was exercised
-    assert variants >= {0, 2, 3, 4, 5}   # rows, ragged chunks, units, bulk and staged kernels all ran
+    return variants
+
+
+def test_random_problems_small_and_odd():
+    variants = random_problems_small_and_odd(600)
+    assert variants >= {0, 3, 4, 5, 6}   # rows, units, bulk, staged and ragged bulk kernels all ran
+
+
+def test_register_kernels_behind_the_tuning_knobs():
+    """With the bulk-copy and staged kernels switched off (environment read when the library first
+    builds a launch, hence a fresh process) the same problems run on the register kernels alone."""
+    import os
+    import subprocess
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    code = ("import sys; sys.path[:0] = [%r, %r]\n"
+            "from test_gpu_parity import random_problems_small_and_odd\n"
+            "v = random_problems_small_and_odd(300)\n"
+            "assert v == {0, 1, 2, 3}, v\n" % (here, os.path.dirname(here)))
+    env = dict(os.environ, REDIST_BULK="0", REDIST_STAGED="0")
+    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
 
 
 def test_round_trip_on_the_gpu():
