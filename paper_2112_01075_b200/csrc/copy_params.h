@@ -25,12 +25,14 @@
 //   kModeChunks all other runs of at least 256 bytes: an item is rows_per_item rows times one column
 //               block of per_block chunks; the rows are decoded once into shared memory and all
 //               threads walk the (row, chunk) space with a flat index.
-//   kModeStaged ragged runs shorter than 256 bytes where the rows of the target are inner_mul runs
-//               long, come from inner_mul different source tiles and are stored to two or more
-//               replicas -- the concatenation of an allgather or the block transpose of an alltoall
-//               along the last differing dimension.  An item stages rows_per_item such rows in shared
-//               memory: the pieces are loaded by a few threads each in 4-byte words, the rows are
-//               written in 16-byte chunks, whole.
+//   kModeGather runs shorter than 256 bytes whose pieces along the last differing dimension interleave
+//               on one side (the long side: m runs from m tiles form one row) while the other side
+//               keeps them in m tiles.  The target bytes of a table row -- a "stretch": the m runs of
+//               a long row, or the run of a short row, times the innermost row digits over which the
+//               target stays contiguous -- are walked in 16-byte chunks aligned on the target; every
+//               thread assembles its chunk from unit_bytes pieces whose source addresses it computes
+//               from the position inside the stretch, and stores it whole.  Stores fill whole
+//               sectors; the loads of neighbouring lanes fall into the same few cache lines.
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
 //               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
 //               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
@@ -46,8 +48,8 @@ constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
 constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
-constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeStaged = 3;
-constexpr int kStageRows = 256;        // rows of one item of the staged transpose
+constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3;
+constexpr int kMaxGatherLevels = 2;    // innermost row digits that can be part of a stretch (kModeGather)
 constexpr int kRaggedBulkRows = 256;   // rows of one item of the ragged bulk-in kernels
 
 // Division of a 31-bit unsigned number by a constant: n / d == umulhi(n, mul) >> shr (d > 1).
@@ -61,28 +63,31 @@ struct CopyGeometry {
     uint32_t fanout;                 // target replicas per box
     uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
     uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
-    uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits or kModeStaged
+    uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits or kModeGather
     uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes);
                                      // 2: ragged chunk walk whose loads are bulk copies into shared memory
     uint64_t run_bytes;              // contiguous run
     uint32_t lanes;                  // kModeRows: threads per row, 1..kBlockThreads
     uint32_t rows_per_pass;          // kModeRows: kBlockThreads / lanes
-    uint32_t rows;                   // rows per box (kModeUnits: table rows, i.e. without the innermost digit)
+    uint32_t rows;                   // rows per box (kModeUnits, kModeGather: table rows, i.e. without the digits walked flat)
     uint32_t rows_per_item;          // kModeRows: multiple of rows_per_pass; else <= kMaxRowsFlat
     uint32_t per_block;              // flat walk: chunks (or units) of one row in a column block
     uint32_t n_items;
     FastDiv per_block_div;           // flat walk: division by per_block
     FastDiv col_blocks;              // flat walk: column blocks per row (1 in kModeRows)
     FastDiv items_per_box;
-    FastDiv inner_n;                 // pieces (or windows of pieces) of one long row that consecutive items handle (1: none)
+    FastDiv inner_n;                 // pieces of one long row that consecutive items handle (1: none, or all in one item)
     uint32_t inner_digit;            // unit digit those pieces belong to
     uint32_t inner_span;             // units of that digit per long row (m1 * m2)
-    uint32_t inner_mul;              // units per item along that digit: 1, or stage_w in kModeStaged
-    uint32_t stage_long_dst;         // kModeStaged: 1 the target has the long rows, 0 the source
-    uint32_t stage_pitch;            // kModeStaged, bulk == 2: bytes between staged rows in shared memory
-    uint32_t stage_ts;               // kModeStaged: tile-index stride between the pieces on the short side
-    uint32_t stage_rows_log2;        // kModeStaged: log2(rows_per_item)
-    uint32_t stage_tpp_log2;         // kModeStaged: log2(threads per piece on the short side)
+    uint32_t inner_mul;              // units per item along that digit: 1, or all of them (inner_span) in kModeGather
+    uint32_t gl_long_dst;            // kModeGather: 1 the target has the long rows, 0 the source
+    uint32_t stage_pitch;            // bulk == 2: bytes between the rows staged in shared memory
+    uint32_t gl_ts;                  // kModeGather: tile-index stride between the pieces on the short side
+    uint32_t gl_levels;              // kModeGather: innermost row digits inside a stretch (0..kMaxGatherLevels)
+    uint32_t gl_stretch;             // kModeGather: bytes of one stretch (< 2^31)
+    FastDiv gl_m;                    // kModeGather: pieces per long row
+    FastDiv gl_n[kMaxGatherLevels];  // kModeGather: extents of those row digits, innermost first
+    int64_t gl_b1[kMaxGatherLevels]; // kModeGather: their source byte strides
     FastDiv lanes_div;
     FastDiv unit_n[kMaxUnitDigits];  // boxes along the digit
     FastDiv unit_m1[kMaxUnitDigits];
@@ -91,9 +96,9 @@ struct CopyGeometry {
     uint32_t unit_ts2[kMaxUnitDigits];
     int64_t unit_b1[kMaxUnitDigits];     // byte stride of one unit inside the tile
     int64_t unit_b2[kMaxUnitDigits];
-    uint32_t n_row_tab;              // row digits decoded through the shared table (n_row, or n_row - 1)
-    FastDiv tab_inner;               // kModeUnits: runs per table row (extent of the innermost row digit, or 1)
-    FastDiv units_per_run;           // kModeUnits: run_bytes / unit_bytes
+    uint32_t n_row_tab;              // row digits decoded through the shared table (n_row, n_row - 1, or n_row - gl_levels)
+    FastDiv tab_inner;               // kModeUnits, kModeGather: runs per table row (extent of the digits walked flat, or 1)
+    FastDiv units_per_run;           // kModeUnits, kModeGather: run_bytes / unit_bytes
     FastDiv row_n[kMaxRowDigits];
     int64_t row_b1[kMaxRowDigits];       // byte stride of the row digit, source / target
     int64_t row_b2[kMaxRowDigits];

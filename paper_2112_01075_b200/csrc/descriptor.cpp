@@ -172,50 +172,70 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     i64 ipb;
     G.lanes = kBlockThreads;
     G.rows_per_pass = 1;
-    // staged transpose: ragged short runs whose long-side rows are `m` runs from m tiles
-    static const bool kStaged = [] {
-        const char *v = std::getenv("REDIST_STAGED");    // tuning knob: REDIST_STAGED=0 disables the staged transpose
-        return !v || std::atoi(v) > 0;
-    }();
     bool ragged_bulk = false;
-    i64 stage_w = 0;
-    if (kStaged && !G.aligned && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu &&
-        m1[kp] == 1 && m2[kp] > 1 && fan >= 2) {
-        // measured: staging pays when the target has the long rows (pieces are gathered) and every
-        // staged row is stored to two or more replicas; otherwise the piece-by-piece walk is as fast
+    // gather walk: short runs whose m pieces interleave on one side; the target bytes of a table row
+    // (the stretch) are produced in whole 16-byte chunks
+    static const int kGather = [] {
+        // tuning knob: REDIST_GATHER=0 disables the gather walk, 2 uses it wherever it applies; the default
+        // (1) keeps it to the cases where it was measured faster than the walk over unit pieces
+        const char *v = std::getenv("REDIST_GATHER");
+        return v ? std::atoi(v) : 1;
+    }();
+    int g_levels = -1;
+    i64 g_stretch = 0;
+    if (kGather > 0 && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu && (m1[kp] == 1 || m2[kp] == 1)) {
+        const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);
-        for (i64 c = m; c >= 2; --c)
-            if (m % c == 0 && c * run_bytes <= 4096) {
-                stage_w = c;
-                break;
-            }
-    }
-    if (stage_w >= 2) {
-        const i64 m = std::max(m1[kp], m2[kp]);
-        const i64 wl = stage_w * run_bytes;
-        i64 pitch = round_up(wl, 16) + 16;
-        if ((pitch / 16) % 2 == 0) pitch += 16;      // odd number of 16-byte units: fewer bank conflicts
-        i64 lg = 0;
-        while ((2ll << lg) <= kStageRows && (2ll << lg) * pitch <= 40 * 1024 && (2ll << lg) * wl <= 2 * kItemBytes) ++lg;
-        const i64 rpi = 1ll << lg;
-        G.mode = kModeStaged;
-        G.inner_mul = uint32_t(stage_w);
-        G.inner_n = make_div(uint32_t(m / stage_w));
-        inner = m / stage_w;
-        G.stage_long_dst = m2[kp] > 1 ? 1u : 0u;
-        G.stage_pitch = uint32_t(pitch);
-        G.stage_ts = m2[kp] > 1 ? G.unit_ts1[G.inner_digit] : G.unit_ts2[G.inner_digit];
-        G.stage_rows_log2 = uint32_t(lg);
-        {
-            // threads per piece: about four 4-byte words each, at most a warp
-            uint32_t tl = 0;
-            while (tl < 5 && (4ll << tl) < run_bytes / 4) ++tl;
-            G.stage_tpp_log2 = tl;
+        const i64 piece_stride = long_dst ? G.unit_b2[G.inner_digit] : G.unit_b1[G.inner_digit];
+        i64 S = long_dst ? m * run_bytes : run_bytes;
+        int lv = 0;
+        for (size_t q = rows.size(); q-- > 0 && lv < kMaxGatherLevels;) {
+            if (rows[q].b2 != S || S * rows[q].n >= (1ll << 31)) break;
+            S *= rows[q].n;
+            ++lv;
         }
+        // measured: pays when the target has the long rows and either every chunk is stored to several
+        // replicas or the runs are short and come from few tiles; long source rows read badly this way
+        const bool pays = long_dst && (fan >= 2 || (run_bytes < 100 && m <= 4));
+        if (piece_stride == run_bytes && S >= 32 && (long_dst || lv > 0) && (kGather >= 2 || pays)) {
+            g_levels = lv;
+            g_stretch = S;
+        }
+    }
+    if (g_levels >= 0) {
+        const bool long_dst = m2[kp] > 1;
+        const i64 m = std::max(m1[kp], m2[kp]);
+        i64 tab_inner = 1;
+        for (int l = 0; l < g_levels; ++l) {
+            const RowDigit &d = rows[rows.size() - 1 - size_t(l)];
+            G.gl_n[l] = make_div(uint32_t(d.n));
+            G.gl_b1[l] = d.b1;
+            tab_inner *= d.n;
+        }
+        const i64 tab_rows = n_rows / tab_inner;
+        const i64 ns = long_dst ? 1 : m;                  // stretches per table row
+        const i64 per_row = g_stretch / 16;
+        const i64 cpb = std::max<i64>(1, std::min<i64>(per_row, kItemBytes / 16));
+        const i64 ncb = std::max<i64>(1, (per_row + cpb - 1) / cpb);
+        i64 rpi = std::max<i64>(1, std::min<i64>(kMaxRowsFlat, kItemBytes / (cpb * 16 * ns)));
+        rpi = std::min<i64>(rpi, tab_rows);
+        G.mode = kModeGather;
+        G.gl_levels = uint32_t(g_levels);
+        G.gl_stretch = uint32_t(g_stretch);
+        G.gl_m = make_div(uint32_t(m));
+        G.inner_mul = uint32_t(m);
+        G.inner_n = make_div(1);
+        inner = 1;
+        G.gl_long_dst = long_dst ? 1u : 0u;
+        G.gl_ts = long_dst ? G.unit_ts1[G.inner_digit] : G.unit_ts2[G.inner_digit];
+        G.rows = uint32_t(tab_rows);
+        G.n_row_tab = uint32_t(rows.size() - size_t(g_levels));
+        G.tab_inner = make_div(uint32_t(tab_inner));
+        G.units_per_run = make_div(uint32_t(run_bytes / vec));
         G.rows_per_item = uint32_t(rpi);
-        G.per_block = uint32_t(wl / 16 + 1);
-        G.col_blocks = make_div(1);
-        ipb = (n_rows + rpi - 1) / rpi;
+        G.per_block = uint32_t(cpb);
+        G.col_blocks = make_div(uint32_t(ncb));
+        ipb = (tab_rows + rpi - 1) / rpi * ncb;
     } else if (G.aligned && max_chunks <= kBlockThreads) {
         // aligned short runs: `lanes` threads per row, one chunk each
         const i64 lanes = max_chunks;
@@ -267,7 +287,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     }
     G.bulk = ragged_bulk ? 2u : 0u;
-    if (kBulk && G.aligned && G.mode != kModeUnits) {
+    if (kBulk && G.aligned && (G.mode == kModeRows || G.mode == kModeChunks)) {
         const i64 seg = G.mode == kModeRows ? run_bytes : i64(G.per_block) * 16;
         if (seg >= kBulkMin && G.rows_per_item <= uint32_t(kBulkThreads) && seg * G.rows_per_item <= 47 * 1024) G.bulk = 1;
     }

@@ -25,10 +25,12 @@
 //                item, kUnroll independent loads in flight before the stores.
 //   kModeChunks  ragged runs of 256 bytes or more (and aligned long runs when bulk copies are switched
 //                off): the rows of an item are decoded once into shared memory and all threads walk the
-//                (row, chunk) space of the item with a flat index.
+//                (row, chunk) space of the item with a flat index.  With bulk copies on, the source
+//                bytes of a ragged item are first brought into shared memory by one bulk copy per row
+//                (ragged_bulk_body) and the walk shifts its chunks out of shared memory.
 //   kModeUnits   ragged runs below 256 bytes: the same flat walk over pieces of unit_bytes.
-//   kModeStaged  ragged runs below 256 bytes that are gathered into long target rows stored to two or
-//                more replicas: the rows are assembled in shared memory and written whole.
+//   kModeGather  runs below 256 bytes that are interleaved into long target rows: the walk follows the
+//                target in whole 16-byte chunks and fetches every unit from its computed source.
 // Index decoding uses multiply-shift division by host-computed constants; the per-item decode (box ->
 // tiles and base offsets) is amortised over ~32 KiB of data.  Every kernel starts with
 // griddepcontrol.wait / launch_dependents (programmatic dependent launch).
@@ -412,119 +414,155 @@ __device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
     }
 }
 
-// ---- kModeStaged: block transpose of short runs through shared memory ---------------------------
-// The long side has rows of w runs (one tile); the short side has the w runs in w different tiles.
-// Shared memory holds rows_per_item long rows, row r at r * pitch + (long-side address of the row mod
-// 16), so that 16-byte chunks of the long side are aligned in both memories.  Short side: one thread
-// per (row, piece), a loop over the 4-byte words of the piece; adjacent lanes take adjacent rows, so
-// their pieces are neighbours in memory whenever the short-side tile is contiguous.  Long side: flat
-// walk over (row, 16-byte chunk) plus the few words before and after the chunk grid of a row.
-template <bool LONG_DST, int NT>
-__device__ __forceinline__ void staged_body(const CopyParams<NT> &P)
+// ---- kModeGather: target stretches in whole chunks, every unit fetched from its computed source ----
+// Position x (bytes, a multiple of sizeof(T)) inside the stretch of table row `e` -> source address.
+// Long target rows: x = ((row digits..., piece j), byte in run); piece j lives in source tile t1 + j * ts.
+// Long source rows: the stretch belongs to target tile j; x = ((row digits...), byte in run) and the
+// source row holds the m pieces side by side.
+template <bool LONG_DST, typename T, int NT>
+__device__ __forceinline__ const T *gather_src(const CopyParams<NT> &P, const BoxBase &b, const RowEntry &e,
+                                               uint32_t j, uint32_t x)
 {
-    extern __shared__ __align__(16) unsigned char tile[];
-    __shared__ RowEntry rowtab[kStageRows];
+    const CopyGeometry &g = P.g;
+    const uint32_t xu = x / uint32_t(sizeof(T));
+    const uint32_t k = fdiv(xu, g.units_per_run);
+    int64_t off = int64_t((xu - k * g.units_per_run.d) * uint32_t(sizeof(T)));
+    uint32_t rr = k;
+    if (LONG_DST) {
+        rr = fdiv(k, g.gl_m);
+        j = k - rr * g.gl_m.d;
+    }
+    if (g.gl_levels == 2) {
+        const uint32_t nx = fdiv(rr, g.gl_n[0]);
+        off += int64_t(rr - nx * g.gl_n[0].d) * g.gl_b1[0] + int64_t(nx) * g.gl_b1[1];
+    } else if (g.gl_levels == 1) {
+        off += int64_t(rr) * g.gl_b1[0];
+    }
+    const char *base = LONG_DST ? P.src[b.t1 + j * g.gl_ts] + b.o1 : b.sbase + int64_t(j) * int64_t(g.run_bytes);
+    return reinterpret_cast<const T *>(base + e.s1 + off);
+}
+
+template <bool LONG_DST, typename T, int NT>
+__device__ __forceinline__ uint4 gather_chunk(const CopyParams<NT> &P, const BoxBase &b, const RowEntry &e,
+                                              uint32_t j, uint32_t x)
+{
+    constexpr int kPer = 16 / int(sizeof(T));
+    union {
+        uint4 v;
+        T t[kPer];
+    } u;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) u.t[i] = __ldg(gather_src<LONG_DST, T, NT>(P, b, e, j, x + uint32_t(i * sizeof(T))));
+    return u.v;
+}
+
+template <bool LONG_DST, typename T, int NT>
+__device__ __forceinline__ void gather_body(const CopyParams<NT> &P, RowEntry *rowtab)
+{
+    constexpr int kU = 2;
     const CopyGeometry &g = P.g;
     const uint32_t tid = threadIdx.x;
     const uint32_t fanout = g.fanout;
-    const uint32_t w = g.inner_mul;
-    const uint32_t run = uint32_t(g.run_bytes);
-    const uint32_t wl = w * run;                  // bytes of one long row in the window
-    const uint32_t pitch = g.stage_pitch;
-    const uint32_t words = run >> 2;
-    const uint32_t cpr = g.per_block;             // chunk slots per row
-    const uint32_t lg = g.stage_rows_log2;
+    const uint32_t S = g.gl_stretch;
+    const uint32_t cpb = g.per_block;
+    const uint32_t ns = LONG_DST ? 1u : g.gl_m.d;         // stretches per table row
     for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
         const BoxBase b = decode_box(P, item);
-        const uint32_t nr = fill_rowtab(g, rowtab, b.part);
-        // offset of the long row r in its tile: (LONG_DST ? o2 + s2 : o1 + s1); bases are 16-byte aligned
-        auto long_off = [&](const RowEntry &e) { return LONG_DST ? b.o2 + e.s2 : b.o1 + e.s1; };
-
-        // long side -> shared (source has the long rows)
-        if (!LONG_DST) {
-            const char *lsrc = P.src[b.t1];
-            for (uint32_t idx = tid; idx < nr * cpr; idx += kBlockThreads) {
-                const uint32_t r = fdiv(idx, g.per_block_div);
-                const uint32_t c = idx - r * cpr;
-                const int64_t off = long_off(rowtab[r]);
-                const uint32_t ph = uint32_t(off) & 15u;
-                const uint32_t head = min((16u - ph) & 15u, wl);
-                const uint32_t chunks = (wl - head) >> 4;
-                if (c < chunks)
-                    *reinterpret_cast<uint4 *>(tile + r * pitch + ph + head + (c << 4)) =
-                        __ldg(reinterpret_cast<const uint4 *>(lsrc + off + head + (c << 4)));
+        const uint32_t group = fdiv(b.part, g.col_blocks);
+        const uint32_t cb = b.part - group * g.col_blocks.d;
+        const uint32_t nr = fill_rowtab(g, rowtab, group);
+        const uint32_t total = nr * ns * cpb;
+        const uint32_t c0 = cb * cpb;
+        for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
+            uint4 v[kU];
+            int64_t d2[kU];
+            uint32_t jt[kU];
+            bool ok[kU];
+#pragma unroll
+            for (int k = 0; k < kU; ++k) {
+                const uint32_t idx = base + k * kBlockThreads;
+                const uint32_t rs = fdiv(idx, g.per_block_div);
+                const uint32_t c = c0 + (idx - rs * cpb);
+                uint32_t r = rs, j = 0;
+                if (!LONG_DST) {
+                    r = fdiv(rs, g.gl_m);
+                    j = rs - r * g.gl_m.d;
+                }
+                const RowEntry e = rowtab[r < nr ? r : 0];
+                uint32_t head, chunks;
+                split_run(S, b.o2 + e.s2, head, chunks);
+                ok[k] = idx < total && c < chunks;
+                const uint32_t x = head + (c << 4);
+                d2[k] = b.o2 + e.s2 + x;
+                jt[k] = j;
+                if (ok[k]) v[k] = gather_chunk<LONG_DST, T, NT>(P, b, e, j, x);
             }
-            for (uint32_t idx = tid; idx < nr * 6u; idx += kBlockThreads) {
-                const uint32_t r = idx / 6u, slot = idx - r * 6u;
-                const int64_t off = long_off(rowtab[r]);
-                const uint32_t ph = uint32_t(off) & 15u;
-                const uint32_t head = min((16u - ph) & 15u, wl);
-                const uint32_t tail_at = head + (((wl - head) >> 4) << 4);
-                const uint32_t at = slot < 3u ? slot * 4u : tail_at + (slot - 3u) * 4u;
-                const bool ok = slot < 3u ? at < head : at < wl;
-                if (ok)
-                    *reinterpret_cast<uint32_t *>(tile + r * pitch + ph + at) =
-                        __ldg(reinterpret_cast<const uint32_t *>(lsrc + off + at));
-            }
-            __syncthreads();
-        }
-
-        // short side <-> shared: 2^stage_tpp_log2 threads per (row, piece), striding over its words
-        const uint32_t tl = g.stage_tpp_log2;
-        for (uint32_t p = tid; p < (w << (lg + tl)); p += kBlockThreads) {
-            const uint32_t sub = p & ((1u << tl) - 1u);
-            const uint32_t pair = p >> tl;
-            const uint32_t j = pair >> lg;
-            const uint32_t r = pair - (j << lg);
-            if (r >= nr) continue;
-            const RowEntry e = rowtab[r];
-            const uint32_t ph = uint32_t(long_off(e)) & 15u;
-            uint32_t *sm = reinterpret_cast<uint32_t *>(tile + r * pitch + ph + j * run);
-            if (LONG_DST) {
-                const uint32_t *gsrc = reinterpret_cast<const uint32_t *>(P.src[b.t1 + j * g.stage_ts] + b.o1 + e.s1);
-                for (uint32_t u = sub; u < words; u += 1u << tl) sm[u] = __ldg(gsrc + u);
-            } else {
-                char *const *dt = &P.dst[(b.t2 + j * g.stage_ts) * fanout];
-                for (uint32_t f = 0; f < fanout; ++f) {
-                    uint32_t *gdst = reinterpret_cast<uint32_t *>(dt[f] + b.o2 + e.s2);
-                    for (uint32_t u = sub; u < words; u += 1u << tl) gdst[u] = sm[u];
+            for (uint32_t f = 0; f < fanout; ++f) {
+#pragma unroll
+                for (int k = 0; k < kU; ++k) {
+                    char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + jt[k] * g.gl_ts) * fanout + f];
+                    if (ok[k]) st_stream(reinterpret_cast<uint4 *>(dbase + d2[k]), v[k]);
                 }
             }
         }
-
-        // shared -> long side (target has the long rows)
-        if (LONG_DST) {
-            __syncthreads();
-            for (uint32_t idx = tid; idx < nr * cpr; idx += kBlockThreads) {
-                const uint32_t r = fdiv(idx, g.per_block_div);
-                const uint32_t c = idx - r * cpr;
-                const int64_t off = long_off(rowtab[r]);
-                const uint32_t ph = uint32_t(off) & 15u;
-                const uint32_t head = min((16u - ph) & 15u, wl);
-                const uint32_t chunks = (wl - head) >> 4;
-                if (c < chunks) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(tile + r * pitch + ph + head + (c << 4));
-                    for (uint32_t f = 0; f < fanout; ++f)
-                        st_stream(reinterpret_cast<uint4 *>(b.dtab[f] + off + head + (c << 4)), v);
+        // ragged ends of the stretches, unit by unit: heads with the first column block, tails with the last
+        constexpr uint32_t kSlots = 16u / uint32_t(sizeof(T)) - 1u;
+        if constexpr (kSlots > 0) {
+            const bool first = cb == 0, last = cb + 1 == g.col_blocks.d;
+            const uint32_t ends = (first ? 1u : 0u) + (last ? 1u : 0u);
+            for (uint32_t idx = tid; idx < nr * ns * kSlots * ends; idx += kBlockThreads) {
+                const uint32_t rs = idx / (kSlots * ends);
+                const uint32_t w = idx - rs * (kSlots * ends);
+                const bool is_head = first && w < kSlots;
+                const uint32_t slot = is_head ? w : (first ? w - kSlots : w);
+                uint32_t r = rs, j = 0;
+                if (!LONG_DST) {
+                    r = fdiv(rs, g.gl_m);
+                    j = rs - r * g.gl_m.d;
                 }
-            }
-            for (uint32_t idx = tid; idx < nr * 6u; idx += kBlockThreads) {
-                const uint32_t r = idx / 6u, slot = idx - r * 6u;
-                const int64_t off = long_off(rowtab[r]);
-                const uint32_t ph = uint32_t(off) & 15u;
-                const uint32_t head = min((16u - ph) & 15u, wl);
-                const uint32_t tail_at = head + (((wl - head) >> 4) << 4);
-                const uint32_t at = slot < 3u ? slot * 4u : tail_at + (slot - 3u) * 4u;
-                const bool ok = slot < 3u ? at < head : at < wl;
-                if (ok) {
-                    const uint32_t v = *reinterpret_cast<const uint32_t *>(tile + r * pitch + ph + at);
-                    for (uint32_t f = 0; f < fanout; ++f) *reinterpret_cast<uint32_t *>(b.dtab[f] + off + at) = v;
+                const RowEntry e = rowtab[r];
+                uint32_t head, chunks;
+                split_run(S, b.o2 + e.s2, head, chunks);
+                const uint32_t toff = head + (chunks << 4);
+                const uint32_t count = (is_head ? head : S - toff) / uint32_t(sizeof(T));
+                if (slot < count) {
+                    const uint32_t x = (is_head ? 0u : toff) + slot * uint32_t(sizeof(T));
+                    const T val = __ldg(gather_src<LONG_DST, T, NT>(P, b, e, j, x));
+                    for (uint32_t f = 0; f < fanout; ++f) {
+                        char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                        *reinterpret_cast<T *>(dbase + b.o2 + e.s2 + x) = val;
+                    }
                 }
             }
         }
-        __syncthreads();
     }
 }
+
+template <bool LONG_DST, int NT>
+__device__ __forceinline__ void gather_dispatch(const CopyParams<NT> &P)
+{
+    __shared__ RowEntry rowtab[kMaxRowsFlat];
+    switch (P.g.unit_bytes) {
+    case 16: gather_body<LONG_DST, uint4, NT>(P, rowtab); break;
+    case 8: gather_body<LONG_DST, uint2, NT>(P, rowtab); break;
+    default: gather_body<LONG_DST, uint32_t, NT>(P, rowtab); break;
+    }
+}
+
+#define REDIST_DEFINE_GATHER_KERNEL(NAME)                                                            \
+    template <bool LONG_DST, int NT>                                                                 \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
+    {                                                                                                \
+        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
+        gather_dispatch<LONG_DST, NT>(P);                                                            \
+    }
+
+REDIST_DEFINE_GATHER_KERNEL(redist_dynslice_gather_kernel)
+REDIST_DEFINE_GATHER_KERNEL(redist_alltoall_gather_kernel)
+REDIST_DEFINE_GATHER_KERNEL(redist_allgather_gather_kernel)
+REDIST_DEFINE_GATHER_KERNEL(redist_allpermute_gather_kernel)
+REDIST_DEFINE_GATHER_KERNEL(redist_fused_gather_kernel)
 
 // ---- bulk-copy variant (aligned runs of at least 512 bytes): TMA moves the segments --------------
 // One work item per block.  Every row segment of the item is one bulk asynchronous copy global ->
@@ -792,20 +830,6 @@ REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_allgather_ragged_bulk_kernel)
 REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_allpermute_ragged_bulk_kernel)
 REDIST_DEFINE_RAGGED_BULK_KERNEL(redist_fused_ragged_bulk_kernel)
 
-#define REDIST_DEFINE_STAGED_KERNEL(NAME)                                                            \
-    template <bool LONG_DST, int NT>                                                                 \
-    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
-    {                                                                                                \
-        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
-        staged_body<LONG_DST, NT>(P);                                                                \
-    }
-
-REDIST_DEFINE_STAGED_KERNEL(redist_dynslice_staged_kernel)
-REDIST_DEFINE_STAGED_KERNEL(redist_alltoall_staged_kernel)
-REDIST_DEFINE_STAGED_KERNEL(redist_allgather_staged_kernel)
-REDIST_DEFINE_STAGED_KERNEL(redist_allpermute_staged_kernel)
-REDIST_DEFINE_STAGED_KERNEL(redist_fused_staged_kernel)
 
 #define REDIST_DEFINE_KERNEL(NAME)                                                                   \
     template <int VARIANT, int NT>                                                                   \
@@ -898,20 +922,19 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
             return cudaLaunchKernelEx(&cfg, fn, P);
         }
     }
-    if (geo.mode == kModeStaged) {
+    if (geo.mode == kModeGather) {
         void (*fn)(const CopyParams<NT>) = nullptr;
-        const bool ld = geo.stage_long_dst != 0;
+        const bool ld = geo.gl_long_dst != 0;
         switch (kernel) {
-        case 0: case 7: fn = ld ? redist_dynslice_staged_kernel<true, NT> : redist_dynslice_staged_kernel<false, NT>; break;
-        case 1: fn = ld ? redist_alltoall_staged_kernel<true, NT> : redist_alltoall_staged_kernel<false, NT>; break;
-        case 2: case 6: fn = ld ? redist_allgather_staged_kernel<true, NT> : redist_allgather_staged_kernel<false, NT>; break;
-        case 3: case 4: fn = ld ? redist_allpermute_staged_kernel<true, NT> : redist_allpermute_staged_kernel<false, NT>; break;
-        default: fn = ld ? redist_fused_staged_kernel<true, NT> : redist_fused_staged_kernel<false, NT>; break;
+        case 0: case 7: fn = ld ? redist_dynslice_gather_kernel<true, NT> : redist_dynslice_gather_kernel<false, NT>; break;
+        case 1: fn = ld ? redist_alltoall_gather_kernel<true, NT> : redist_alltoall_gather_kernel<false, NT>; break;
+        case 2: case 6: fn = ld ? redist_allgather_gather_kernel<true, NT> : redist_allgather_gather_kernel<false, NT>; break;
+        case 3: case 4: fn = ld ? redist_allpermute_gather_kernel<true, NT> : redist_allpermute_gather_kernel<false, NT>; break;
+        default: fn = ld ? redist_fused_gather_kernel<true, NT> : redist_fused_gather_kernel<false, NT>; break;
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(unsigned(grid));
         cfg.blockDim = dim3(kBlockThreads);
-        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -33,14 +33,23 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     unit = G["unit_bytes"]
     assert unit in (1, 2, 4, 8, 16) and (G["aligned"] == 1) == (unit == 16) and run % unit == 0
     max_chunks = run // 16
-    if G["mode"] == 3:      # staged transpose: rows_per_item long rows of `mul` runs in shared memory
-        rpi = G["rows_per_item"]
-        assert unit >= 4 and unit < 16 and run < 256 and mul >= 2 and mul * run <= 4096
-        assert rpi & (rpi - 1) == 0 and 1 <= rpi <= 256
-        assert G["stage_pitch"] % 16 == 0 and G["stage_pitch"] >= mul * run + 16 and G["stage_pitch"] * rpi <= 40 * 1024
-        assert G["items_per_box"] == -(-rows // rpi) and tab_rows == rows
+    if G["mode"] == 3:      # gather walk: target stretches of a table row in whole chunks
         u = G["inner_digit"]
-        assert G["unit_m1"][u] == 1 and G["unit_m2"][u] > 1 and G["stage_long_dst"] == 1 and fan >= 2
+        m1, m2 = G["unit_m1"][u], G["unit_m2"][u]
+        long_dst = G["gl_long_dst"] == 1
+        assert unit >= 4 and run < 256 and inner == 1 and mul == span == max(m1, m2) == G["gl_m"] and min(m1, m2) == 1
+        assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
+        assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
+        lv = G["gl_levels"]
+        assert 0 <= lv <= 2 and (long_dst or lv >= 1) and G["n_row_tab"] == len(G["row_n"]) - lv
+        S = mul * run if long_dst else run
+        for l in range(lv):
+            q = len(G["row_n"]) - 1 - l
+            assert G["row_b2"][q] == S and G["gl_n"][l] == G["row_n"][q] and G["gl_b1"][l] == G["row_b1"][q]
+            S *= G["row_n"][q]
+        assert S == G["gl_stretch"] and 32 <= S < 2 ** 31 and G["tab_inner"] == _prod(G["row_n"][len(G["row_n"]) - lv:])
+        assert 1 <= G["rows_per_item"] <= 1024 and G["col_blocks"] * G["per_block"] >= S // 16
+        assert G["items_per_box"] == -(-tab_rows // G["rows_per_item"]) * G["col_blocks"]
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
         assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0
@@ -65,7 +74,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     col = np.arange(run, dtype=np.int64)
     written = {}
     for boxp in range(n_boxes * span):
-        box, piece = divmod(boxp, span)          # a staged item covers `mul` consecutive pieces
+        box, piece = divmod(boxp, span)          # a gather item covers `mul` consecutive pieces
         rem, t1, t2, o1, o2 = box, 0, 0, 0, 0
         for u in range(len(unit_n) - 1, -1, -1):
             q = rem % unit_n[u]

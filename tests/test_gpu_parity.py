@@ -128,23 +128,33 @@ def random_problems_small_and_odd(n_problems):
 
 def test_random_problems_small_and_odd():
     variants = random_problems_small_and_odd(600)
-    assert variants >= {0, 3, 4, 5, 6}   # rows, units, bulk, staged and ragged bulk kernels all ran
+    assert variants >= {0, 3, 4, 5, 6}   # rows, units, bulk, gather and ragged bulk kernels all ran
 
 
-def test_register_kernels_behind_the_tuning_knobs():
-    """With the bulk-copy and staged kernels switched off (environment read when the library first
-    builds a launch, hence a fresh process) the same problems run on the register kernels alone."""
+def _random_problems_in_a_fresh_process(env, n_problems, expect):
     import os
     import subprocess
     import sys
     here = os.path.dirname(os.path.abspath(__file__))
     code = ("import sys; sys.path[:0] = [%r, %r]\n"
             "from test_gpu_parity import random_problems_small_and_odd\n"
-            "v = random_problems_small_and_odd(300)\n"
-            "assert v == {0, 1, 2, 3}, v\n" % (here, os.path.dirname(here)))
-    env = dict(os.environ, REDIST_BULK="0", REDIST_STAGED="0")
-    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+            "v = random_problems_small_and_odd(%d)\n"
+            "assert %s, v\n" % (here, os.path.dirname(here), n_problems, expect))
+    res = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, **env), capture_output=True,
+                         text=True, timeout=600)
     assert res.returncode == 0, res.stderr[-2000:]
+
+
+def test_register_kernels_behind_the_tuning_knobs():
+    """With the bulk-copy kernels and the gather walk switched off (environment read when the library
+    first builds a launch, hence a fresh process) the same problems run on the plain register kernels."""
+    _random_problems_in_a_fresh_process({"REDIST_BULK": "0", "REDIST_GATHER": "0"}, 300, "v == {0, 1, 2, 3}")
+
+
+def test_gather_walk_wherever_it_applies():
+    """REDIST_GATHER=2 sends every eligible launch through the gather walk, including long source rows
+    that are scattered into several target tiles and 16-byte units (not chosen by default)."""
+    _random_problems_in_a_fresh_process({"REDIST_GATHER": "2"}, 600, "5 in v")
 
 
 def test_round_trip_on_the_gpu():
@@ -449,7 +459,7 @@ def test_soak_full_size_forward_and_back_without_synchronising():
     assert api.redist_bulk_timeouts() == 0
 
 
-STAGED = [
+GATHER = [
     ((2, 4), (6, 10, 24), ((), (), (1,)), ((), (), ()), 4),
     ((2, 2, 2), (8, 6, 60), ((0,), (), (1, 2)), ((0,), (), (1,)), 4),
     ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4),
@@ -461,10 +471,10 @@ STAGED = [
 ]
 
 
-@pytest.mark.parametrize("mesh,gshape,src_axes,dst_axes,e", STAGED)
-def test_staged_transpose_kernels(mesh, gshape, src_axes, dst_axes, e):
-    """Short ragged runs gathered into long target rows that are stored to several replicas go through
-    the shared-memory staged kernels (launch variant 5)."""
+@pytest.mark.parametrize("mesh,gshape,src_axes,dst_axes,e", GATHER)
+def test_gather_walk_kernels(mesh, gshape, src_axes, dst_axes, e):
+    """Short ragged runs interleaved into long target rows that are stored to several replicas go
+    through the gather walk (launch variant 5)."""
     rng = np.random.default_rng(sum(gshape))
     G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
     src, dst = (gshape, src_axes), (gshape, dst_axes)
@@ -472,9 +482,9 @@ def test_staged_transpose_kernels(mesh, gshape, src_axes, dst_axes, e):
     want = oracle.reslice(mesh, dst, G)
     plan, got = run_gpu(mesh, src, dst, e, src_tiles)
     assert plan.launch_info(0).variant == 5
-    assert_same(got, want, f"staged {mesh} {gshape}")
+    assert_same(got, want, f"gather {mesh} {gshape}")
     _, got = run_gpu(mesh, src, dst, e, src_tiles, api.FUSE_NONE)
-    assert_same(got, want, f"staged, unfused {mesh} {gshape}")
+    assert_same(got, want, f"gather, unfused {mesh} {gshape}")
 
 
 def test_four_gib_tiles_need_64_bit_offsets():
