@@ -311,7 +311,7 @@ def run_ours(args):
         api.KERNELS[li.kernel], api.KERNELS[li.kernel])
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "traffic": ncu_traffic(args.workload),
-                "kernel": f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk'}.get(li.variant, '') }_kernel",
+                "kernel": f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk', 7: '_zip'}.get(li.variant, '') }_kernel",
                 "algorithmic_bytes_per_launch": alg,
                 "avg_launch_us": round(avg_ms * 1e3, 2),
                 "avg_from": "timed region / launches" if same else "event pair around each launch",

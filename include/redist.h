@@ -109,8 +109,8 @@ typedef struct redist_launch_info {
     int32_t fanout;                /* destination replicas stored per element read                     */
     int32_t variant;               /* kernel variant: 0 rows, 1 chunks, 2 ragged chunks, 3 units (register
                                       kernels), 4 TMA bulk copies, 5 gather walk, 6 ragged rows loaded by
-                                      TMA bulk copies; the kernel is named
-                                      redist_<collective>[_bulk|_gather|_ragged_bulk]_kernel           */
+                                      TMA bulk copies, 7 zip through shared memory; the kernel is named
+                                      redist_<collective>[_bulk|_gather|_ragged_bulk|_zip]_kernel      */
 } redist_launch_info;
 
 /*

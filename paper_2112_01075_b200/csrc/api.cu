@@ -264,7 +264,7 @@ redist_status redist_plan_launch_info(const redist_plan_t *plan, int32_t launch,
     o.bytes_written = L.bytes_written;
     o.n_items = L.geo.n_items;
     o.fanout = int32_t(L.geo.fanout);
-    o.variant = L.geo.bulk == 2 ? 6 : L.geo.bulk ? 4 : (L.geo.mode == kModeGather ? 5 : L.geo.mode == kModeRows ? 0 : L.geo.mode == kModeUnits ? 3 : (L.geo.aligned ? 1 : 2));
+    o.variant = L.geo.bulk == 2 ? 6 : L.geo.bulk ? 4 : (L.geo.mode == kModeZip ? 7 : L.geo.mode == kModeGather ? 5 : L.geo.mode == kModeRows ? 0 : L.geo.mode == kModeUnits ? 3 : (L.geo.aligned ? 1 : 2));
     *out = o;
     return REDIST_OK;
 }

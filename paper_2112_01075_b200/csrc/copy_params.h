@@ -33,6 +33,13 @@
 //               thread assembles its chunk from unit_bytes pieces whose source addresses it computes
 //               from the position inside the stretch, and stores it whole.  Stores fill whole
 //               sectors; the loads of neighbouring lanes fall into the same few cache lines.
+//   kModeZip    the same interleaving of m short runs, when both sides stay contiguous across the
+//               innermost row digit (n rows): a table row is then m source streams of n runs zipped
+//               into one target stream of n long rows, or the reverse.  An item covers rows_per_item
+//               table rows times a block of per_block rows of that digit; its source bytes -- one
+//               contiguous segment per stream -- are brought into shared memory by bulk copies, and
+//               the threads assemble target-aligned 16-byte chunks from shared memory, where a
+//               scattered access costs no cache-line lookups.
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
 //               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
 //               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
@@ -48,7 +55,8 @@ constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
 constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
-constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3;
+constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3, kModeZip = 4;
+constexpr int kZipSegments = 256;      // source segments (table rows times streams) of one kModeZip item
 constexpr int kMaxGatherLevels = 2;    // innermost row digits that can be part of a stretch (kModeGather)
 constexpr int kRaggedBulkRows = 256;   // rows of one item of the ragged bulk-in kernels
 
@@ -63,7 +71,7 @@ struct CopyGeometry {
     uint32_t fanout;                 // target replicas per box
     uint32_t aligned;                // 1: run length and every offset are multiples of 16 bytes
     uint32_t unit_bytes;             // largest power of two (<= 16) dividing run length and offsets
-    uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits or kModeGather
+    uint32_t mode;                   // kModeRows, kModeChunks, kModeUnits, kModeGather or kModeZip
     uint32_t bulk;                   // 1: the item's row segments move by TMA bulk copies (aligned, >= 512 bytes);
                                      // 2: ragged chunk walk whose loads are bulk copies into shared memory
     uint64_t run_bytes;              // contiguous run
@@ -80,12 +88,15 @@ struct CopyGeometry {
     uint32_t inner_digit;            // unit digit those pieces belong to
     uint32_t inner_span;             // units of that digit per long row (m1 * m2)
     uint32_t inner_mul;              // units per item along that digit: 1, or all of them (inner_span) in kModeGather
-    uint32_t gl_long_dst;            // kModeGather: 1 the target has the long rows, 0 the source
-    uint32_t stage_pitch;            // bulk == 2: bytes between the rows staged in shared memory
-    uint32_t gl_ts;                  // kModeGather: tile-index stride between the pieces on the short side
+    uint32_t gl_long_dst;            // kModeGather, kModeZip: 1 the target has the long rows, 0 the source
+    uint32_t stage_pitch;            // bulk == 2, kModeZip: bytes between the rows staged in shared memory
+    uint32_t gl_ts;                  // kModeGather, kModeZip: tile-index stride between the pieces on the short side
     uint32_t gl_levels;              // kModeGather: innermost row digits inside a stretch (0..kMaxGatherLevels)
     uint32_t gl_stretch;             // kModeGather: bytes of one stretch (< 2^31)
-    FastDiv gl_m;                    // kModeGather: pieces per long row
+    FastDiv gl_m;                    // kModeGather, kModeZip: pieces per long row
+    uint32_t zip_seg_pitch;          // kModeZip: shared-memory bytes reserved per source segment
+    FastDiv zip_slots;               // kModeZip: chunk slots per target range of an item
+    uint32_t zip_tile_fastest;       // kModeZip, long source rows: 1 = neighbouring lanes write to neighbouring target tiles
     FastDiv gl_n[kMaxGatherLevels];  // kModeGather: extents of those row digits, innermost first
     int64_t gl_b1[kMaxGatherLevels]; // kModeGather: their source byte strides
     FastDiv lanes_div;

@@ -202,7 +202,68 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             g_stretch = S;
         }
     }
-    if (g_levels >= 0) {
+    // zip: the same interleaving when the innermost row digit is contiguous on both sides -- the source
+    // segments of an item are then long enough for bulk copies into shared memory
+    static const int kZip = [] {
+        // tuning knob: REDIST_ZIP=0 disables the zip kernels, 1 uses them only where the gather walk is
+        // not chosen; the default (2) wherever they apply (measured: within 0.3 % of the best choice per
+        // problem on the odd-shape sweep)
+        const char *v = std::getenv("REDIST_ZIP");
+        return v ? std::atoi(v) : 2;
+    }();
+    static const i64 kZipMinRange = [] {
+        const char *v = std::getenv("REDIST_ZIP_MIN");   // tuning knob: shortest target range of a table row for the zip kernels
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 128);
+    }();
+    i64 zip_n = 0;
+    if (kZip > 0 && kBulk && (kZip >= 2 || g_levels < 0) && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu &&
+        (m1[kp] == 1 || m2[kp] == 1) && !rows.empty()) {
+        const bool long_dst = m2[kp] > 1;
+        const i64 m = std::max(m1[kp], m2[kp]);
+        const i64 piece_stride = long_dst ? G.unit_b2[G.inner_digit] : G.unit_b1[G.inner_digit];
+        const RowDigit &d = rows.back();
+        const i64 bs = long_dst ? run_bytes : m * run_bytes, bd = long_dst ? m * run_bytes : run_bytes;
+        // a source segment of a full item should be worth a bulk copy
+        if (piece_stride == run_bytes && d.b1 == bs && d.b2 == bd && d.n * bs >= 256 && d.n * bd >= kZipMinRange && m <= 16) zip_n = d.n;
+    }
+    if (zip_n > 0) {
+        const bool long_dst = m2[kp] > 1;
+        const i64 m = std::max(m1[kp], m2[kp]);
+        const i64 nseg = long_dst ? m : 1;                 // source segments per table row
+        const i64 row_bytes = m * run_bytes;               // both sides, per row of the zipped digit
+        const i64 tab_rows = n_rows / zip_n;
+        const i64 seg_row = long_dst ? run_bytes : row_bytes;   // bytes of one row in a source segment
+        const i64 kTile = 38 * 1024;                            // shared-memory tile of an item, at most
+        i64 rpb = std::max<i64>(1, std::min<i64>(zip_n, kItemBytes / row_bytes));
+        rpb = std::max<i64>(1, std::min<i64>(rpb, (kTile / nseg - 48) / seg_row));
+        const i64 ncb = (zip_n + rpb - 1) / rpb;
+        const i64 seg_pitch = round_up(rpb * seg_row, 16) + 32;
+        i64 rpi = std::max<i64>(1, kItemBytes / (rpb * row_bytes));
+        rpi = std::min<i64>(std::min<i64>(rpi, tab_rows), std::max<i64>(1, kZipSegments / nseg));
+        rpi = std::max<i64>(1, std::min<i64>(rpi, kTile / (seg_pitch * nseg)));
+        if (seg_pitch * nseg * rpi > kTile) return REDIST_EINTERNAL;
+        G.mode = kModeZip;
+        G.gl_levels = 0;
+        G.gl_stretch = 0;
+        G.gl_m = make_div(uint32_t(m));
+        G.inner_mul = uint32_t(m);
+        G.inner_n = make_div(1);
+        inner = 1;
+        G.gl_long_dst = long_dst ? 1u : 0u;
+        G.gl_ts = long_dst ? G.unit_ts1[G.inner_digit] : G.unit_ts2[G.inner_digit];
+        G.rows = uint32_t(tab_rows);
+        G.n_row_tab = uint32_t(rows.size() - 1);
+        G.tab_inner = make_div(uint32_t(zip_n));
+        G.units_per_run = make_div(uint32_t(run_bytes / vec));
+        G.rows_per_item = uint32_t(rpi);
+        G.per_block = uint32_t(rpb);
+        G.col_blocks = make_div(uint32_t(ncb));
+        G.zip_seg_pitch = uint32_t(seg_pitch);
+        G.zip_tile_fastest = !long_dst && run_bytes <= 16 ? 1u : 0u;
+        G.stage_pitch = uint32_t(seg_pitch * nseg);
+        G.zip_slots = make_div(uint32_t(rpb * (long_dst ? row_bytes : run_bytes) / 16 + 1));
+        ipb = (tab_rows + rpi - 1) / rpi * ncb;
+    } else if (g_levels >= 0) {
         const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);
         i64 tab_inner = 1;

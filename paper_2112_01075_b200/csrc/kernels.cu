@@ -19,7 +19,7 @@
 // item is one TMA bulk copy global -> shared (cp.async.bulk, byte-counted completion on an mbarrier)
 // and one bulk copy shared -> global per target replica, issued by a few threads (bulk_body below;
 // measured 1-3 % faster than the register path on every benchmark configuration).  Everything else
-// uses the register kernels, in four item shapes (CopyGeometry::mode):
+// uses the item shapes below (CopyGeometry::mode):
 //   kModeRows    aligned runs below the bulk threshold: a block of 256 threads covers rows_per_pass
 //                rows of `lanes` chunks; a thread keeps its column and walks down the rows of its work
 //                item, kUnroll independent loads in flight before the stores.
@@ -31,6 +31,8 @@
 //   kModeUnits   ragged runs below 256 bytes: the same flat walk over pieces of unit_bytes.
 //   kModeGather  runs below 256 bytes that are interleaved into long target rows: the walk follows the
 //                target in whole 16-byte chunks and fetches every unit from its computed source.
+//   kModeZip     the same interleaving (either direction) when the row digit next to it is contiguous
+//                on both sides: source segments staged in shared memory by bulk copies (zip_body).
 // Index decoding uses multiply-shift division by host-computed constants; the per-item decode (box ->
 // tiles and base offsets) is amortised over ~32 KiB of data.  Every kernel starts with
 // griddepcontrol.wait / launch_dependents (programmatic dependent launch).
@@ -815,6 +817,175 @@ __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
     }
 }
 
+// ---- kModeZip: m source streams <-> one target stream, through shared memory ---------------------
+// One item per block.  Table row r of the item and rows [a, a + cnt) of the zipped digit: the source
+// bytes are m segments of cnt runs (long target rows: one per source tile) or one segment of cnt long
+// rows (long source rows).  One thread per segment posts its byte count and issues the bulk copy of
+// the covering 16-byte blocks; segbase[] remembers where byte 0 of the segment sits in shared memory.
+// Then the target ranges -- one per table row, or one per (table row, target tile) -- are written in
+// target-aligned 16-byte chunks assembled unit by unit from shared memory, ends in single units.
+template <bool LONG_DST, typename T, int NT>
+__device__ __forceinline__ const T *zip_src(const CopyGeometry &g, const unsigned char *tile, const uint32_t *segbase,
+                                            uint32_t r, uint32_t j, uint32_t x)
+{
+    const uint32_t xu = x / uint32_t(sizeof(T));
+    const uint32_t k = fdiv(xu, g.units_per_run);            // run number inside the range
+    const uint32_t w = (xu - k * g.units_per_run.d) * uint32_t(sizeof(T));
+    const uint32_t run = uint32_t(g.run_bytes);
+    uint32_t at;
+    if (LONG_DST) {
+        const uint32_t rr = fdiv(k, g.gl_m);
+        const uint32_t jj = k - rr * g.gl_m.d;
+        at = segbase[r * g.gl_m.d + jj] + rr * run + w;
+    } else {
+        at = segbase[r] + (k * g.gl_m.d + j) * run + w;
+    }
+    return reinterpret_cast<const T *>(tile + at);
+}
+
+template <bool LONG_DST, typename T, int NT>
+__device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char *tile, RowEntry *rowtab,
+                                         uint32_t *segbase, uint32_t mbar)
+{
+    constexpr int kPer = 16 / int(sizeof(T));
+    const CopyGeometry &g = P.g;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t fanout = g.fanout;
+    const uint32_t m = g.gl_m.d;
+    const uint32_t run = uint32_t(g.run_bytes);
+    const uint32_t nseg = LONG_DST ? m : 1u;
+    const uint32_t nrng = LONG_DST ? 1u : m;              // target ranges per table row
+    const uint32_t item = blockIdx.x;
+    if (item >= g.n_items) return;
+    const BoxBase b = decode_box(P, item);
+    const uint32_t group = fdiv(b.part, g.col_blocks);
+    const uint32_t cb = b.part - group * g.col_blocks.d;
+    const uint32_t row0 = group * g.rows_per_item;
+    const uint32_t nr = min(g.rows_per_item, g.rows - row0);
+    const uint32_t a = cb * g.per_block;
+    const uint32_t cnt = min(g.per_block, g.tab_inner.d - a);
+    const uint32_t seg_bytes = cnt * run * (LONG_DST ? 1u : m);
+    const uint32_t rng_bytes = cnt * run * (LONG_DST ? m : 1u);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(nr * nseg) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    for (uint32_t t = tid; t < nr * nseg; t += kBlockThreads) {
+        const uint32_t r = fdiv(t, g.gl_m);
+        const uint32_t j = LONG_DST ? t - r * m : 0u;
+        const uint32_t rr = LONG_DST ? r : t;
+        RowEntry e;
+        row_offsets(g, row0 + rr, e.s1, e.s2, int(g.n_row_tab));
+        if (j == 0) rowtab[rr] = e;
+        const char *src = LONG_DST ? P.src[b.t1 + j * g.gl_ts] + b.o1 + e.s1 + int64_t(a) * run
+                                   : b.sbase + e.s1 + int64_t(a) * run * m;
+        const uint32_t mis = uint32_t(reinterpret_cast<uintptr_t>(src)) & 15u;
+        const uint32_t slot = t * g.zip_seg_pitch;
+        segbase[t] = slot + mis;
+        const uint32_t bytes = (mis + seg_bytes + 15u) & ~15u;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(tile) + slot), "l"(src - mis), "r"(bytes), "r"(mbar)
+                     : "memory");
+    }
+    __syncthreads();
+    if (!mbar_wait_bounded(mbar, 0, 1u << 18)) {
+        if (tid == 0) atomicAdd(&g_bulk_timeouts, 1u);
+        mbar_wait_bounded(mbar, 0, 1u << 18);
+        return;
+    }
+    // whole chunks of the target ranges
+    const uint32_t slots = g.zip_slots.d;
+    const uint32_t total = nr * nrng * slots;
+    for (uint32_t idx = tid; idx < total; idx += kBlockThreads) {
+        // long source rows of very short runs: neighbouring lanes take the same chunk of neighbouring
+        // target tiles, whose units are neighbours in the staged long row (no bank conflicts); with
+        // longer runs neighbouring lanes stay in one run and in one target tile (wider stores)
+        uint32_t r, c, j = 0;
+        if (LONG_DST) {
+            r = fdiv(idx, g.zip_slots);
+            c = idx - r * slots;
+        } else if (g.zip_tile_fastest) {
+            const uint32_t t = fdiv(idx, g.gl_m);
+            j = idx - t * m;
+            r = fdiv(t, g.zip_slots);
+            c = t - r * slots;
+        } else {
+            const uint32_t q = fdiv(idx, g.zip_slots);
+            c = idx - q * slots;
+            r = fdiv(q, g.gl_m);
+            j = q - r * m;
+        }
+        const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+        uint32_t head, chunks;
+        split_run(rng_bytes, d0, head, chunks);
+        if (c < chunks) {
+            const uint32_t x = head + (c << 4);
+            union {
+                uint4 v;
+                T t[kPer];
+            } u;
+#pragma unroll
+            for (int i = 0; i < kPer; ++i)
+                u.t[i] = *zip_src<LONG_DST, T, NT>(g, tile, segbase, r, j, x + uint32_t(i * sizeof(T)));
+            for (uint32_t f = 0; f < fanout; ++f) {
+                char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
+            }
+        }
+    }
+    // ragged ends of the ranges, unit by unit
+    constexpr uint32_t kSlots = 16u / uint32_t(sizeof(T)) - 1u;
+    if constexpr (kSlots > 0) {
+        for (uint32_t idx = tid; idx < nr * nrng * kSlots * 2u; idx += kBlockThreads) {
+            const uint32_t q = idx / (kSlots * 2u);
+            const uint32_t w = idx - q * (kSlots * 2u);
+            const bool is_head = w < kSlots;
+            const uint32_t slot = is_head ? w : w - kSlots;
+            const uint32_t r = LONG_DST ? q : fdiv(q, g.gl_m);
+            const uint32_t j = LONG_DST ? 0u : q - r * m;
+            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+            uint32_t head, chunks;
+            split_run(rng_bytes, d0, head, chunks);
+            const uint32_t toff = head + (chunks << 4);
+            const uint32_t count = (is_head ? head : rng_bytes - toff) / uint32_t(sizeof(T));
+            if (slot < count) {
+                const uint32_t x = (is_head ? 0u : toff) + slot * uint32_t(sizeof(T));
+                const T val = *zip_src<LONG_DST, T, NT>(g, tile, segbase, r, j, x);
+                for (uint32_t f = 0; f < fanout; ++f) {
+                    char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                    *reinterpret_cast<T *>(dbase + d0 + x) = val;
+                }
+            }
+        }
+    }
+}
+
+#define REDIST_DEFINE_ZIP_KERNEL(NAME)                                                               \
+    template <bool LONG_DST, int NT>                                                                 \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
+    {                                                                                                \
+        extern __shared__ __align__(128) unsigned char tile[];                                       \
+        __shared__ RowEntry rowtab[kZipSegments];                                                    \
+        __shared__ uint32_t segbase[kZipSegments];                                                   \
+        __shared__ __align__(8) unsigned long long mbar_storage;                                     \
+        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
+        const uint32_t mbar = smem_addr(&mbar_storage);                                              \
+        switch (P.g.unit_bytes) {                                                                    \
+        case 16: zip_body<LONG_DST, uint4, NT>(P, tile, rowtab, segbase, mbar); break;               \
+        case 8: zip_body<LONG_DST, uint2, NT>(P, tile, rowtab, segbase, mbar); break;                \
+        default: zip_body<LONG_DST, uint32_t, NT>(P, tile, rowtab, segbase, mbar); break;            \
+        }                                                                                            \
+    }
+
+REDIST_DEFINE_ZIP_KERNEL(redist_dynslice_zip_kernel)
+REDIST_DEFINE_ZIP_KERNEL(redist_alltoall_zip_kernel)
+REDIST_DEFINE_ZIP_KERNEL(redist_allgather_zip_kernel)
+REDIST_DEFINE_ZIP_KERNEL(redist_allpermute_zip_kernel)
+REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
+
 #define REDIST_DEFINE_RAGGED_BULK_KERNEL(NAME)                                                       \
     template <int NT>                                                                                \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
@@ -921,6 +1092,28 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
             cfg.numAttrs = 1;
             return cudaLaunchKernelEx(&cfg, fn, P);
         }
+    }
+    if (geo.mode == kModeZip) {
+        void (*fn)(const CopyParams<NT>) = nullptr;
+        const bool ld = geo.gl_long_dst != 0;
+        switch (kernel) {
+        case 0: case 7: fn = ld ? redist_dynslice_zip_kernel<true, NT> : redist_dynslice_zip_kernel<false, NT>; break;
+        case 1: fn = ld ? redist_alltoall_zip_kernel<true, NT> : redist_alltoall_zip_kernel<false, NT>; break;
+        case 2: case 6: fn = ld ? redist_allgather_zip_kernel<true, NT> : redist_allgather_zip_kernel<false, NT>; break;
+        case 3: case 4: fn = ld ? redist_allpermute_zip_kernel<true, NT> : redist_allpermute_zip_kernel<false, NT>; break;
+        default: fn = ld ? redist_fused_zip_kernel<true, NT> : redist_fused_zip_kernel<false, NT>; break;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(geo.n_items);
+        cfg.blockDim = dim3(kBlockThreads);
+        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, fn, P);
     }
     if (geo.mode == kModeGather) {
         void (*fn)(const CopyParams<NT>) = nullptr;

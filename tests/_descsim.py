@@ -50,6 +50,24 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         assert S == G["gl_stretch"] and 32 <= S < 2 ** 31 and G["tab_inner"] == _prod(G["row_n"][len(G["row_n"]) - lv:])
         assert 1 <= G["rows_per_item"] <= 1024 and G["col_blocks"] * G["per_block"] >= S // 16
         assert G["items_per_box"] == -(-tab_rows // G["rows_per_item"]) * G["col_blocks"]
+    elif G["mode"] == 4:    # zip: both sides contiguous across the innermost row digit, staged by bulk copies
+        u = G["inner_digit"]
+        m1, m2 = G["unit_m1"][u], G["unit_m2"][u]
+        long_dst = G["gl_long_dst"] == 1
+        m = max(m1, m2)
+        assert unit >= 4 and run < 256 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 16
+        assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
+        assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
+        n = G["row_n"][-1]
+        assert G["tab_inner"] == n and G["n_row_tab"] == len(G["row_n"]) - 1
+        assert G["row_b1"][-1] == (run if long_dst else m * run) and G["row_b2"][-1] == (m * run if long_dst else run)
+        rpb, rpi, nseg = G["per_block"], G["rows_per_item"], (m if long_dst else 1)
+        assert 1 <= rpb <= n and G["col_blocks"] == -(-n // rpb) and 1 <= rpi and rpi * nseg <= 256
+        seg = rpb * (run if long_dst else m * run)
+        assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= seg + 30
+        assert G["stage_pitch"] == G["zip_seg_pitch"] * nseg and G["stage_pitch"] * rpi <= 38 * 1024
+        assert G["zip_slots"] >= rpb * (m * run if long_dst else run) // 16
+        assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
         assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0

@@ -128,7 +128,7 @@ def random_problems_small_and_odd(n_problems):
 
 def test_random_problems_small_and_odd():
     variants = random_problems_small_and_odd(600)
-    assert variants >= {0, 3, 4, 5, 6}   # rows, units, bulk, gather and ragged bulk kernels all ran
+    assert variants >= {0, 3, 4, 5, 6, 7}   # rows, units, bulk, gather, ragged bulk and zip kernels all ran
 
 
 def _random_problems_in_a_fresh_process(env, n_problems, expect):
@@ -146,15 +146,16 @@ def _random_problems_in_a_fresh_process(env, n_problems, expect):
 
 
 def test_register_kernels_behind_the_tuning_knobs():
-    """With the bulk-copy kernels and the gather walk switched off (environment read when the library
-    first builds a launch, hence a fresh process) the same problems run on the plain register kernels."""
+    """With the bulk-copy kernels (zip included) and the gather walk switched off (environment read when
+    the library first builds a launch, hence a fresh process) the same problems run on the plain
+    register kernels."""
     _random_problems_in_a_fresh_process({"REDIST_BULK": "0", "REDIST_GATHER": "0"}, 300, "v == {0, 1, 2, 3}")
 
 
 def test_gather_walk_wherever_it_applies():
     """REDIST_GATHER=2 sends every eligible launch through the gather walk, including long source rows
     that are scattered into several target tiles and 16-byte units (not chosen by default)."""
-    _random_problems_in_a_fresh_process({"REDIST_GATHER": "2"}, 600, "5 in v")
+    _random_problems_in_a_fresh_process({"REDIST_GATHER": "2", "REDIST_ZIP": "0"}, 600, "5 in v and 7 not in v")
 
 
 def test_round_trip_on_the_gpu():
@@ -459,32 +460,34 @@ def test_soak_full_size_forward_and_back_without_synchronising():
     assert api.redist_bulk_timeouts() == 0
 
 
-GATHER = [
-    ((2, 4), (6, 10, 24), ((), (), (1,)), ((), (), ()), 4),
-    ((2, 2, 2), (8, 6, 60), ((0,), (), (1, 2)), ((0,), (), (1,)), 4),
-    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4),
-    ((2, 3, 2), (4, 9, 180), ((0,), (), (1, 2)), ((), (), (2,)), 4),
-    ((8,), (33, 88), ((), (0,)), ((), ()), 4),
-    ((2, 2), (16, 6, 4), ((), (), (0, 1)), ((), (0,), ()), 8),
-    ((2, 2, 2), (6, 5, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4),
-    ((2, 2, 2), (700, 3, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4),      # many row groups, ragged last one
+INTERLEAVED = [   # mesh, global shape, sharded type, gathered type, element bytes, variant there, variant back
+    ((2, 4), (6, 10, 24), ((), (), (1,)), ((), (), ()), 4, 7, 7),
+    ((2, 2, 2), (8, 6, 60), ((0,), (), (1, 2)), ((0,), (), (1,)), 4, 7, 7),
+    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4, 5, 7),
+    ((2, 3, 2), (4, 9, 180), ((0,), (), (1, 2)), ((), (), (2,)), 4, 7, 7),
+    ((8,), (33, 88), ((), (0,)), ((), ()), 4, 7, 7),
+    ((2, 2), (16, 6, 4), ((), (), (0, 1)), ((), (0,), ()), 8, 5, 3),
+    ((2, 2, 2), (6, 5, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4, 7, 7),
+    ((2, 2, 2), (700, 3, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4, 7, 7),      # many row groups, ragged last one
 ]
 
 
-@pytest.mark.parametrize("mesh,gshape,src_axes,dst_axes,e", GATHER)
-def test_gather_walk_kernels(mesh, gshape, src_axes, dst_axes, e):
-    """Short ragged runs interleaved into long target rows that are stored to several replicas go
-    through the gather walk (launch variant 5)."""
+@pytest.mark.parametrize("mesh,gshape,sharded,gathered,e,v_there,v_back", INTERLEAVED)
+def test_gather_walk_and_zip_kernels(mesh, gshape, sharded, gathered, e, v_there, v_back):
+    """Short ragged runs interleaved into long target rows go through the zip kernels (launch variant 7;
+    source segments staged in shared memory by bulk copies) or the gather walk (variant 5); the way
+    back scatters long source rows over several target tiles."""
     rng = np.random.default_rng(sum(gshape))
     G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
-    src, dst = (gshape, src_axes), (gshape, dst_axes)
-    src_tiles = oracle.reslice(mesh, src, G)
-    want = oracle.reslice(mesh, dst, G)
-    plan, got = run_gpu(mesh, src, dst, e, src_tiles)
-    assert plan.launch_info(0).variant == 5
-    assert_same(got, want, f"gather {mesh} {gshape}")
-    _, got = run_gpu(mesh, src, dst, e, src_tiles, api.FUSE_NONE)
-    assert_same(got, want, f"gather, unfused {mesh} {gshape}")
+    for src, dst, variant in (((gshape, sharded), (gshape, gathered), v_there),
+                              ((gshape, gathered), (gshape, sharded), v_back)):
+        src_tiles = oracle.reslice(mesh, src, G)
+        want = oracle.reslice(mesh, dst, G)
+        plan, got = run_gpu(mesh, src, dst, e, src_tiles)
+        assert plan.launch_info(0).variant == variant
+        assert_same(got, want, f"interleaved {mesh} {src} -> {dst}")
+        _, got = run_gpu(mesh, src, dst, e, src_tiles, api.FUSE_NONE)
+        assert_same(got, want, f"interleaved, unfused {mesh} {src} -> {dst}")
 
 
 def test_four_gib_tiles_need_64_bit_offsets():
