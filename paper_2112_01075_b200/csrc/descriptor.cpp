@@ -86,7 +86,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     G.inner_span = 1;
     G.inner_mul = 1;
     i64 inner = 1;
-    if (kp >= 0 && run_bytes < 1024 && nq[kp] > 1 && m1[kp] * m2[kp] > 1) {
+    static const i64 kInnerRun = [] {
+        const char *v = std::getenv("REDIST_INNER_RUN");   // tuning knob: runs below this many bytes get adjacent-piece item numbering
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 16384);
+    }();
+    if (kp >= 0 && run_bytes < kInnerRun && nq[kp] > 1 && m1[kp] * m2[kp] > 1) {
         inner = m1[kp] * m2[kp];
         uint32_t u = 0;
         for (int k = 0; k < kp; ++k)
@@ -241,11 +245,16 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const i64 tab_rows = n_rows / zip_n;
         const i64 seg_row = long_dst ? run_bytes : row_bytes;   // bytes of one row in a source segment
         const i64 kTile = 38 * 1024;                            // shared-memory tile of an item, at most
-        i64 rpb = std::max<i64>(1, std::min<i64>(zip_n, kItemBytes / row_bytes));
+        static const i64 kZipKb = [] {
+            const char *v = std::getenv("REDIST_ZIP_KB");    // tuning knob: KiB read per zip item
+            return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 0);
+        }();
+        const i64 kZipBytes = kZipKb > 0 ? kZipKb * 1024 : kItemBytes;
+        i64 rpb = std::max<i64>(1, std::min<i64>(zip_n, kZipBytes / row_bytes));
         rpb = std::max<i64>(1, std::min<i64>(rpb, (kTile / nseg - 48) / seg_row));
         const i64 ncb = (zip_n + rpb - 1) / rpb;
         const i64 seg_pitch = round_up(rpb * seg_row, 16) + 32;
-        i64 rpi = std::max<i64>(1, kItemBytes / (rpb * row_bytes));
+        i64 rpi = std::max<i64>(1, kZipBytes / (rpb * row_bytes));
         rpi = std::min<i64>(std::min<i64>(rpi, tab_rows), std::max<i64>(1, kZipSegments / nseg));
         rpi = std::max<i64>(1, std::min<i64>(rpi, kTile / (seg_pitch * nseg)));
         if (seg_pitch * nseg * rpi > kTile) return REDIST_EINTERNAL;
