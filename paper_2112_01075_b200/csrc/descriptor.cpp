@@ -277,7 +277,20 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.zip_seg_pitch = uint32_t(seg_pitch);
         G.zip_tile_fastest = !long_dst && run_bytes <= 16 ? 1u : 0u;
         G.stage_pitch = uint32_t(seg_pitch * nseg);
-        G.zip_slots = make_div(uint32_t(rpb * (long_dst ? row_bytes : run_bytes) / 16 + 1));
+        static const i64 kZipPerRun = [] {
+            const char *v = std::getenv("REDIST_ZIP_PER_RUN");   // tuning knob: shortest run whose chunks are numbered per run (0: never)
+            return i64(v ? std::atoi(v) : 32);
+        }();
+        // measured: pays from 32-byte runs of 4-byte units (four divisions per chunk saved), from 64-byte
+        // runs of 8-byte units; nothing to gain with 16-byte units
+        if (kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16) {
+            const i64 cpr = (run_bytes + 15) / 16;
+            G.zip_cpr = make_div(uint32_t(cpr));
+            G.zip_slots = make_div(uint32_t(rpb * (long_dst ? m : 1) * cpr));
+        } else {
+            G.zip_cpr = FastDiv{0, 0, 0};
+            G.zip_slots = make_div(uint32_t(rpb * (long_dst ? row_bytes : run_bytes) / 16 + 1));
+        }
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     } else if (g_levels >= 0) {
         const bool long_dst = m2[kp] > 1;

@@ -898,6 +898,50 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
     // whole chunks of the target ranges
     const uint32_t slots = g.zip_slots.d;
     const uint32_t total = nr * nrng * slots;
+    if (g.zip_cpr.d != 0) {
+        // runs of 32 bytes and more (same branch for every thread): slot = (run k of the range, i-th
+        // target-aligned chunk that starts inside the run).  Such a chunk takes its units from run k and,
+        // past its end, from run k + 1 -- two base addresses and a compare per unit, no division.
+        const uint32_t cpr = g.zip_cpr.d;
+        const uint32_t nruns = cnt * (LONG_DST ? m : 1u);
+        for (uint32_t idx = tid; idx < total; idx += kBlockThreads) {
+            const uint32_t q = fdiv(idx, g.zip_slots);
+            const uint32_t rem = idx - q * slots;
+            const uint32_t k = fdiv(rem, g.zip_cpr);
+            const uint32_t ci = rem - k * cpr;
+            const uint32_t r = LONG_DST ? q : fdiv(q, g.gl_m);
+            const uint32_t j = LONG_DST ? 0u : q - r * m;
+            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+            const uint32_t xs = k * run;
+            const uint32_t x = xs + ((16u - ((uint32_t(d0) + xs) & 15u)) & 15u) + (ci << 4);
+            if (k < nruns && x < xs + run && x + 16u <= rng_bytes) {
+                uint32_t base0, base1;      // shared-memory address of target byte p: base + p
+                if (LONG_DST) {
+                    const uint32_t rr = fdiv(k, g.gl_m);
+                    const uint32_t jj = k - rr * m;
+                    const bool wrap = jj + 1u == m;
+                    base0 = segbase[r * m + jj] + rr * run - xs;
+                    base1 = segbase[r * m + (wrap ? 0u : jj + 1u)] + (wrap ? rr + 1u : rr) * run - (xs + run);
+                } else {
+                    base0 = segbase[r] + (k * m + j) * run - xs;
+                    base1 = base0 + (m - 1u) * run;
+                }
+                union {
+                    uint4 v;
+                    T t[kPer];
+                } u;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    const uint32_t p = x + uint32_t(i * sizeof(T));
+                    u.t[i] = *reinterpret_cast<const T *>(tile + ((p >= xs + run ? base1 : base0) + p));
+                }
+                for (uint32_t f = 0; f < fanout; ++f) {
+                    char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                    st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
+                }
+            }
+        }
+    } else
     for (uint32_t idx = tid; idx < total; idx += kBlockThreads) {
         // long source rows of very short runs: neighbouring lanes take the same chunk of neighbouring
         // target tiles, whose units are neighbours in the staged long row (no bank conflicts); with
