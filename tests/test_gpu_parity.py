@@ -490,10 +490,14 @@ def test_gather_walk_and_zip_kernels(mesh, gshape, sharded, gathered, e, v_there
         assert_same(got, want, f"interleaved, unfused {mesh} {src} -> {dst}")
 
 
-def test_four_gib_tiles_need_64_bit_offsets():
-    """u32 [32768, 32768] (4 GiB, value = global linear index) on two devices: replicated -> column
-    sharded reads at offsets beyond 2^32 inside a tile, column sharded -> replicated writes there."""
-    mesh, g = (2,), (32768, 32768)
+@pytest.mark.parametrize("g,variant", [((32768, 32768), 4), ((44739243, 24), 7)])
+def test_four_gib_tiles_need_64_bit_offsets(g, variant):
+    """u32 arrays of 4 GiB and a little more (value = global linear index) on two devices: replicated
+    -> column sharded reads at offsets beyond 2^32 inside a tile, column sharded -> replicated writes
+    there.  64 KiB rows go by bulk copies, 96-byte rows (48-byte runs) through the zip kernels."""
+    mesh = (2,)
+    total = g[0] * g[1] * 4
+    assert total >= 2**32
     G = wl.global_array_bytes(g, 4, "linear_u32", 0)
     repl, cols = (g, ((), ())), (g, ((), (0,)))
     oracle.set_threads(oracle.max_threads())
@@ -503,17 +507,21 @@ def test_four_gib_tiles_need_64_bit_offsets():
         oracle.set_threads(1)
     one = torch.from_numpy(G.reshape(-1)).cuda()
     plan = api.Plan(mesh, repl, cols, 4)
+    assert plan.launch_info(0).variant == variant
     nb = plan.local_elems(1) * 4
     out = [torch.empty(nb, dtype=torch.uint8, device="cuda") for _ in range(2)]
-    plan.execute([one, one], out)                      # replicas alias one 4 GiB buffer
+    plan.execute([one, one], out)                      # replicas alias one buffer
     torch.cuda.synchronize()
     assert_same([t.cpu().numpy() for t in out], col_tiles, "replicated -> columns")
     back = api.Plan(mesh, cols, repl, 4)
-    full = [torch.empty(4 * 2**30, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    assert back.launch_info(0).variant == variant
+    full = [torch.empty(total, dtype=torch.uint8, device="cuda") for _ in range(2)]
     back.execute(out, full)
     torch.cuda.synchronize()
     for d in range(2):
         assert torch.equal(full[d], one), f"columns -> replicated, device {d}"
+    del full, out, one
+    torch.cuda.empty_cache()
 
 
 def test_zero_bulk_copy_timeouts_after_everything_above():
