@@ -221,11 +221,10 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }();
     static const i64 kZipRun = [] {
         const char *v = std::getenv("REDIST_ZIP_RUN");   // tuning knob: runs below this many bytes may take the zip kernels
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 1024);
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 2048);
     }();
-    // measured: with runs of 512 bytes and more the plain bulk copy (aligned runs) is faster, and so is
-    // the ragged chunk walk unless every chunk is stored to several replicas
-    const bool zip_run_ok = run_bytes < kZipRun && (run_bytes < 512 || (!G.aligned && fan >= 2));
+    // measured: aligned runs of 512 bytes and more are faster as plain bulk copies
+    const bool zip_run_ok = run_bytes < (G.aligned ? std::min<i64>(512, kZipRun) : kZipRun);
     i64 zip_n = 0;
     if (kZip > 0 && kBulk && (kZip >= 2 || g_levels < 0) && vec >= 4 && zip_run_ok && G.inner_digit != 0xffffffffu &&
         (m1[kp] == 1 || m2[kp] == 1) && !rows.empty()) {
