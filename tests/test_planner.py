@@ -368,3 +368,23 @@ def test_random_plans_never_fail_in_any_mode():
             assert p.height <= max(p.local_elems(0), p.local_elems(1))
             assert p.step_kinds().count("allpermute") <= 1
             p.close()
+
+
+KERNEL_CHOICE = [   # mesh, global shape, source axes, target axes, element bytes, expected launch variants
+    ((4, 2), (8, 2048, 4096), ((0,), (), (1,)), ((), (0, 1), ()), 2, [4]),             # 4 KiB aligned runs: bulk copies
+    ((2,), (64, 24), ((), ()), ((), (0,)), 4, [7]),                                    # 48-byte runs unzipped into 2 tiles
+    ((2,), (64, 24), ((), (0,)), ((), ()), 4, [7]),                                    # and zipped back
+    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4, [5]),                      # interleave without a contiguous row digit
+    ((2, 2), (16, 6, 4), ((), (0,), ()), ((), (), (0, 1)), 8, [3]),                    # 8-byte runs scattered: unit walk
+    ((2,), (6, 70), ((0,), ()), ((), ()), 4, [6]),                                     # ragged 840-byte runs: bulk-loaded chunk walk
+    ((4,), (16, 16), ((0,), ()), ((), (0,)), 4, [0]),                                  # aligned 16-byte runs, too few rows to zip: rows
+]
+
+
+@pytest.mark.parametrize("mesh,gshape,a1,a2,e,variants", KERNEL_CHOICE)
+def test_kernel_variant_chosen_for_a_shape(mesh, gshape, a1, a2, e, variants):
+    """The host picks the kernel by run length, alignment and how the pieces interleave (no GPU needed)."""
+    p = api.Plan(mesh, (gshape, a1), (gshape, a2), e)
+    assert [p.launch_info(q).variant for q in range(p.num_launches)] == variants
+    p.close()
+    check_plan(mesh, (gshape, a1), (gshape, a2), e, api.FUSE_ADJACENT)
