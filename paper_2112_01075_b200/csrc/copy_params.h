@@ -56,6 +56,7 @@ constexpr int kBlockThreads = 256;
 constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
 constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3, kModeZip = 4;
+constexpr int kZipSmallTile = 23 * 1024; // kModeZip items with at most this much shared memory run with 128 threads
 constexpr int kZipSegments = 256;      // source segments (table rows times streams) of one kModeZip item
 constexpr int kMaxGatherLevels = 2;    // innermost row digits that can be part of a stretch (kModeGather)
 constexpr int kRaggedBulkRows = 256;   // rows of one item of the ragged bulk-in kernels
