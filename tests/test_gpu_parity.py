@@ -295,6 +295,26 @@ def test_evaluation_like_problems_reduced():
         assert_same(got, want, ws.name)
 
 
+EVAL_FULL = ["eval0007", "eval0019", "eval0023", "eval0070", "eval0079", "eval0082", "eval0093", "eval0115",
+             "eval0134", "eval0175"]
+
+
+@pytest.mark.parametrize("name", EVAL_FULL)
+def test_evaluation_like_problems_full_size(name):
+    """Ten problems of the odd-shape sweep at the size the sweep times them (64-800 MB, f32): unit walk,
+    gather walk, zip in both directions, ragged bulk and plain bulk kernels; every target tile compared."""
+    w = {p.name: p for p in wl.evaluation_like_problems(200)}[name]
+    oracle.set_threads(oracle.max_threads())
+    try:
+        src, dst, src_tiles, want = make_case(w)
+    finally:
+        oracle.set_threads(1)
+    _, got = run_gpu(w.mesh_shape, src, dst, w.elem_bytes, src_tiles)
+    assert_same(got, want, w.name)
+    del got, src_tiles, want
+    torch.cuda.empty_cache()
+
+
 def test_random_sweep_full_size_samples():
     """Three pairs of the sweep at the full [64,128,256,512] f32 shape (4 GiB global), chosen by
     device footprint; all target tiles compared."""
