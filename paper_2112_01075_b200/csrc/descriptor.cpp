@@ -284,10 +284,16 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         // runs of 8-byte units; nothing to gain with 16-byte units
         if (kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16) {
             const i64 cpr = (run_bytes + 15) / 16;
+            static const i64 kZipByRange = [] {
+                const char *v = std::getenv("REDIST_ZIP_BY_RANGE");   // tuning knob: fewest chunk slots of a range walked on its own (0: never)
+                return i64(v ? std::atoi(v) : 256);
+            }();
             G.zip_cpr = make_div(uint32_t(cpr));
             G.zip_slots = make_div(uint32_t(rpb * (long_dst ? m : 1) * cpr));
+            G.zip_by_range = kZipByRange > 0 && rpb * (long_dst ? m : 1) * cpr >= kZipByRange ? 1u : 0u;
         } else {
             G.zip_cpr = FastDiv{0, 0, 0};
+            G.zip_by_range = 0;
             G.zip_slots = make_div(uint32_t(rpb * (long_dst ? row_bytes : run_bytes) / 16 + 1));
         }
         ipb = (tab_rows + rpi - 1) / rpi * ncb;

@@ -899,7 +899,54 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
     // whole chunks of the target ranges
     const uint32_t slots = g.zip_slots.d;
     const uint32_t total = nr * nrng * slots;
-    if (g.zip_cpr.d != 0) {
+    if (g.zip_cpr.d != 0 && g.zip_by_range != 0) {
+        // long ranges of runs of 32 bytes and more (same branch for every thread): the block goes through
+        // the ranges one after the other; a thread keeps its chunk number inside a run (ci) and walks down
+        // the runs k, k + kstep, ... of the range, so everything that depends on the range is computed
+        // once and a chunk costs a few multiply-adds, the unit reads and the stores
+        const uint32_t cpr = g.zip_cpr.d;
+        const uint32_t kstep = fdiv(nthreads, g.zip_cpr);
+        const uint32_t kk = fdiv(tid, g.zip_cpr);
+        const uint32_t ci = tid - kk * cpr;
+        const uint32_t nruns = cnt * (LONG_DST ? m : 1u);
+        for (uint32_t q = 0; q < nr * nrng && kk < kstep; ++q) {
+            const uint32_t r = LONG_DST ? q : fdiv(q, g.gl_m);
+            const uint32_t j = LONG_DST ? 0u : q - r * m;
+            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+            const uint32_t d0lo = uint32_t(d0);
+            const uint32_t sb = LONG_DST ? 0u : segbase[r] + j * run;
+            for (uint32_t k = kk; k < nruns; k += kstep) {
+                const uint32_t xs = k * run;
+                const uint32_t x = xs + ((16u - ((d0lo + xs) & 15u)) & 15u) + (ci << 4);
+                if (x < xs + run && x + 16u <= rng_bytes) {
+                    uint32_t base0, base1;      // shared-memory address of target byte p: base + p
+                    if (LONG_DST) {
+                        const uint32_t rr = fdiv(k, g.gl_m);
+                        const uint32_t jj = k - rr * m;
+                        const bool wrap = jj + 1u == m;
+                        base0 = segbase[r * m + jj] + rr * run - xs;
+                        base1 = segbase[r * m + (wrap ? 0u : jj + 1u)] + (wrap ? rr + 1u : rr) * run - (xs + run);
+                    } else {
+                        base0 = sb + k * (m - 1u) * run;    // segbase[r] + (k * m + j) * run - xs
+                        base1 = base0 + (m - 1u) * run;
+                    }
+                    union {
+                        uint4 v;
+                        T t[kPer];
+                    } u;
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        const uint32_t p = x + uint32_t(i * sizeof(T));
+                        u.t[i] = *reinterpret_cast<const T *>(tile + ((p >= xs + run ? base1 : base0) + p));
+                    }
+                    for (uint32_t f = 0; f < fanout; ++f) {
+                        char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                        st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
+                    }
+                }
+            }
+        }
+    } else if (g.zip_cpr.d != 0) {
         // runs of 32 bytes and more (same branch for every thread): slot = (run k of the range, i-th
         // target-aligned chunk that starts inside the run).  Such a chunk takes its units from run k and,
         // past its end, from run k + 1 -- two base addresses and a compare per unit, no division.

@@ -68,9 +68,10 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= seg + 30
         assert G["stage_pitch"] == G["zip_seg_pitch"] * nseg and G["stage_pitch"] * rpi <= 38 * 1024
         if G["zip_cpr"]:
+            assert G["zip_by_range"] == (1 if G["zip_slots"] >= 256 else 0)
             assert run >= 16 and unit < 16 and G["zip_cpr"] == -(-run // 16) and G["zip_slots"] == rpb * (m if long_dst else 1) * G["zip_cpr"]
         else:
-            assert G["zip_slots"] >= rpb * (m * run if long_dst else run) // 16
+            assert G["zip_by_range"] == 0 and G["zip_slots"] >= rpb * (m * run if long_dst else run) // 16
         assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
