@@ -276,6 +276,29 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.zip_seg_pitch = uint32_t(seg_pitch);
         G.zip_tile_fastest = !long_dst && run_bytes <= 16 ? 1u : 0u;
         G.stage_pitch = uint32_t(seg_pitch * nseg);
+        {
+            // periodic walk: a table row must give every thread several chunks, and the period must leave most
+            // threads of a block busy
+            static const i64 kZipPeriodic = [] {
+                const char *v = std::getenv("REDIST_ZIP_PERIODIC");   // tuning knob: fewest chunks per table row for the periodic walk (0: never)
+                return i64(v ? std::atoi(v) : 512);
+            }();
+            const i64 L = long_dst ? row_bytes : run_bytes;         // bytes after which the target pattern repeats, up to alignment
+            const i64 gc = std::gcd<i64>(16, L);
+            const i64 pc = L / gc;
+            G.zip_period = FastDiv{0, 0, 0};
+            G.zip_period_rows = 0;
+            static const i64 kZipPc = [] {
+                const char *v = std::getenv("REDIST_ZIP_PC");   // tuning knob: longest period, in chunks
+                return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 64);
+            }();
+            // (with long source rows of runs up to 16 bytes a thread stays with one of the m target tiles)
+            const i64 lanes_needed = !long_dst && run_bytes <= 16 ? pc * m : pc;
+            if (kZipPeriodic > 0 && rpb * row_bytes / 16 >= kZipPeriodic && lanes_needed <= kZipPc) {
+                G.zip_period = make_div(uint32_t(pc));
+                G.zip_period_rows = uint32_t(16 / gc);
+            }
+        }
         static const i64 kZipPerRun = [] {
             const char *v = std::getenv("REDIST_ZIP_PER_RUN");   // tuning knob: shortest run whose chunks are numbered per run (0: never)
             return i64(v ? std::atoi(v) : 32);

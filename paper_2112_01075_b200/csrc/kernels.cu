@@ -899,7 +899,49 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
     // whole chunks of the target ranges
     const uint32_t slots = g.zip_slots.d;
     const uint32_t total = nr * nrng * slots;
-    if (g.zip_cpr.d != 0 && g.zip_by_range != 0) {
+    if (g.zip_period.d != 0) {
+        // long ranges (same branch for every thread): the map from a target chunk to the shared-memory
+        // places of its units repeats every zip_period chunks, shifted by a whole number of rows.  A thread
+        // decodes the units of its first chunk once per table row and then strides through the range -- and,
+        // with long source rows, through the m target tiles -- in steps of S chunks, a multiple of the
+        // period: every further chunk costs one add per unit, the unit reads and the stores.
+        // Long source rows of very short runs: a thread stays with one target tile (tid mod m), so that
+        // neighbouring lanes read neighbouring units of the staged long row; otherwise it takes the tiles in turn.
+        uint32_t tl = tid, width = nthreads, jb = 0, jn = nrng;
+        if (!LONG_DST && g.zip_tile_fastest) {
+            tl = fdiv(tid, g.gl_m);
+            jb = tid - tl * m;
+            jn = 1;
+            width = fdiv(nthreads, g.gl_m);
+        }
+        const uint32_t S = fdiv(width, g.zip_period) * g.zip_period.d;
+        const uint32_t step = fdiv(S, g.zip_period) * g.zip_period_rows * (LONG_DST ? run : run * m);
+        for (uint32_t r = 0; r < nr && tl < S; ++r) {
+            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+            uint32_t head, chunks;
+            split_run(rng_bytes, d0, head, chunks);
+            uint32_t at[kPer];
+#pragma unroll
+            for (int i = 0; i < kPer; ++i)
+                at[i] = uint32_t(reinterpret_cast<const unsigned char *>(zip_src<LONG_DST, T, NT>(
+                                     g, tile, segbase, r, jb, head + (tl << 4) + uint32_t(i * sizeof(T)))) - tile);
+            for (uint32_t j = jb; j < jb + jn; ++j) {
+                uint32_t o = (j - jb) * run;
+                for (uint32_t c = tl; c < chunks; c += S, o += step) {
+                    union {
+                        uint4 v;
+                        T t[kPer];
+                    } u;
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) u.t[i] = *reinterpret_cast<const T *>(tile + (at[i] + o));
+                    for (uint32_t f = 0; f < fanout; ++f) {
+                        char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                        st_stream(reinterpret_cast<uint4 *>(dbase + d0 + head + (c << 4)), u.v);
+                    }
+                }
+            }
+        }
+    } else if (g.zip_cpr.d != 0 && g.zip_by_range != 0) {
         // long ranges of runs of 32 bytes and more (same branch for every thread): the block goes through
         // the ranges one after the other; a thread keeps its chunk number inside a run (ci) and walks down
         // the runs k, k + kstep, ... of the range, so everything that depends on the range is computed

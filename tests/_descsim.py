@@ -67,6 +67,11 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         seg = rpb * (run if long_dst else m * run)
         assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= seg + 30
         assert G["stage_pitch"] == G["zip_seg_pitch"] * nseg and G["stage_pitch"] * rpi <= 38 * 1024
+        if G["zip_period"]:
+            import math
+            lb = m * run if long_dst else run
+            assert G["zip_period"] == lb // math.gcd(16, lb) and G["zip_period_rows"] == 16 // math.gcd(16, lb)
+            assert rpb * m * run // 16 >= 512 and G["zip_period"] * (m if not long_dst and run <= 16 else 1) <= 64
         if G["zip_cpr"]:
             assert G["zip_by_range"] == (1 if G["zip_slots"] >= 256 else 0)
             assert run >= 16 and unit < 16 and G["zip_cpr"] == -(-run // 16) and G["zip_slots"] == rpb * (m if long_dst else 1) * G["zip_cpr"]
