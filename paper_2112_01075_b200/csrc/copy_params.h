@@ -97,10 +97,10 @@ struct CopyGeometry {
     FastDiv gl_m;                    // kModeGather, kModeZip: pieces per long row
     uint32_t zip_seg_pitch;          // kModeZip: shared-memory bytes reserved per source segment
     FastDiv zip_slots;               // kModeZip: chunk slots per target range of an item
-    FastDiv zip_cpr;                 // kModeZip: chunk slots per run when slots are numbered (run, chunk in run); d = 0: flat
+    FastDiv zip_cpr;                 // kModeZip: chunk slots per run in the by-range walk; d = 0: walk not used
     FastDiv zip_period;              // kModeZip: chunks after which the chunk -> units map repeats (d = 0: path not used)
     uint32_t zip_period_rows;        // kModeZip: rows of the zipped digit that one period spans
-    uint32_t zip_by_range;           // kModeZip with zip_cpr: 1 = ranges are long enough to be walked one after the other
+    uint32_t zip_lut_units;          // kModeZip: units of the longest range when their places are tabulated in shared memory (0: not)
     uint32_t zip_tile_fastest;       // kModeZip, long source rows: 1 = neighbouring lanes write to neighbouring target tiles
     FastDiv gl_n[kMaxGatherLevels];  // kModeGather: extents of those row digits, innermost first
     int64_t gl_b1[kMaxGatherLevels]; // kModeGather: their source byte strides

@@ -299,25 +299,38 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                 G.zip_period_rows = uint32_t(16 / gc);
             }
         }
+        // By-range walk: for runs of 32 bytes and more of 4-byte units (64 and more of 8-byte units; nothing
+        // to gain with 16-byte units) the chunk slots of a range are numbered (run, i-th target-aligned chunk
+        // that starts in the run) -- such a chunk takes its units from that run and, past its end, from the
+        // next one, no division per unit -- and a range with 256 slots or more is walked by the whole block.
         static const i64 kZipPerRun = [] {
-            const char *v = std::getenv("REDIST_ZIP_PER_RUN");   // tuning knob: shortest run whose chunks are numbered per run (0: never)
+            const char *v = std::getenv("REDIST_ZIP_PER_RUN");   // tuning knob: shortest run (of 4-byte units) for the by-range walk (0: never)
             return i64(v ? std::atoi(v) : 32);
         }();
-        // measured: pays from 32-byte runs of 4-byte units (four divisions per chunk saved), from 64-byte
-        // runs of 8-byte units; nothing to gain with 16-byte units
-        if (kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16) {
-            const i64 cpr = (run_bytes + 15) / 16;
-            static const i64 kZipByRange = [] {
-                const char *v = std::getenv("REDIST_ZIP_BY_RANGE");   // tuning knob: fewest chunk slots of a range walked on its own (0: never)
-                return i64(v ? std::atoi(v) : 256);
-            }();
+        static const i64 kZipByRange = [] {
+            const char *v = std::getenv("REDIST_ZIP_BY_RANGE");   // tuning knob: fewest chunk slots of a range for the by-range walk
+            return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 256);
+        }();
+        const i64 cpr = (run_bytes + 15) / 16;
+        if (G.zip_period.d == 0 && kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16 &&
+            rpb * (long_dst ? m : 1) * cpr >= kZipByRange) {
             G.zip_cpr = make_div(uint32_t(cpr));
             G.zip_slots = make_div(uint32_t(rpb * (long_dst ? m : 1) * cpr));
-            G.zip_by_range = kZipByRange > 0 && rpb * (long_dst ? m : 1) * cpr >= kZipByRange ? 1u : 0u;
         } else {
             G.zip_cpr = FastDiv{0, 0, 0};
-            G.zip_by_range = 0;
             G.zip_slots = make_div(uint32_t(rpb * (long_dst ? row_bytes : run_bytes) / 16 + 1));
+        }
+        {
+            // short ranges (neither walk above applies): the place of every unit of a range is tabulated in shared
+            // memory; the chunk slots are then numbered flat
+            static const i64 kZipLut = [] {
+                const char *v = std::getenv("REDIST_ZIP_LUT");   // tuning knob: longest range, in units, whose unit places are tabulated (0: never)
+                return i64(v ? std::atoi(v) : 2048);
+            }();
+            const i64 units = rpb * (long_dst ? row_bytes : run_bytes) / vec;
+            G.zip_lut_units = 0;
+            if (G.zip_period.d == 0 && G.zip_cpr.d == 0 && units <= kZipLut && seg_pitch * nseg * rpi + units * 4 <= 42 * 1024)
+                G.zip_lut_units = uint32_t(units);
         }
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     } else if (g_levels >= 0) {

@@ -890,6 +890,19 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
                      ::"r"(smem_addr(tile) + slot), "l"(src - mis), "r"(bytes), "r"(mbar)
                      : "memory");
     }
+    // short ranges: while the copies are in flight, tabulate for every unit position of a range where
+    // the unit sits -- which segment of its table row (upper bits) and at which byte of it (lower 20 bits)
+    uint32_t *lut = reinterpret_cast<uint32_t *>(tile + size_t(g.stage_pitch) * g.rows_per_item);
+    for (uint32_t u = tid; u < g.zip_lut_units; u += nthreads) {
+        const uint32_t k = fdiv(u, g.units_per_run);
+        const uint32_t w = (u - k * g.units_per_run.d) * uint32_t(sizeof(T));
+        if (LONG_DST) {
+            const uint32_t rr = fdiv(k, g.gl_m);
+            lut[u] = ((k - rr * m) << 20) | (rr * run + w);
+        } else {
+            lut[u] = k * m * run + w;
+        }
+    }
     __syncthreads();
     if (!mbar_wait_bounded(mbar, 0, 1u << 18)) {
         if (tid == 0) atomicAdd(&g_bulk_timeouts, 1u);
@@ -899,6 +912,49 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
     // whole chunks of the target ranges
     const uint32_t slots = g.zip_slots.d;
     const uint32_t total = nr * nrng * slots;
+    if (g.zip_lut_units != 0) {
+        // flat walk over (range, chunk); a unit costs a table read, the read of its segment's base and the
+        // read of the unit itself
+        for (uint32_t idx = tid; idx < total; idx += nthreads) {
+            uint32_t r, c, j = 0;
+            if (LONG_DST) {
+                r = fdiv(idx, g.zip_slots);
+                c = idx - r * slots;
+            } else if (g.zip_tile_fastest) {
+                const uint32_t t = fdiv(idx, g.gl_m);
+                j = idx - t * m;
+                r = fdiv(t, g.zip_slots);
+                c = t - r * slots;
+            } else {
+                const uint32_t q = fdiv(idx, g.zip_slots);
+                c = idx - q * slots;
+                r = fdiv(q, g.gl_m);
+                j = q - r * m;
+            }
+            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
+            uint32_t head, chunks;
+            split_run(rng_bytes, d0, head, chunks);
+            if (c < chunks) {
+                const uint32_t x = head + (c << 4);
+                const uint32_t u0 = x / uint32_t(sizeof(T));
+                const uint32_t sb = LONG_DST ? 0u : segbase[r] + j * run;
+                union {
+                    uint4 v;
+                    T t[kPer];
+                } u;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    const uint32_t e = lut[u0 + uint32_t(i)];
+                    const uint32_t at = LONG_DST ? segbase[r * m + (e >> 20)] + (e & 0xfffffu) : sb + e;
+                    u.t[i] = *reinterpret_cast<const T *>(tile + at);
+                }
+                for (uint32_t f = 0; f < fanout; ++f) {
+                    char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
+                    st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
+                }
+            }
+        }
+    } else
     if (g.zip_period.d != 0) {
         // long ranges (same branch for every thread): the map from a target chunk to the shared-memory
         // places of its units repeats every zip_period chunks, shifted by a whole number of rows.  A thread
@@ -941,7 +997,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
                 }
             }
         }
-    } else if (g.zip_cpr.d != 0 && g.zip_by_range != 0) {
+    } else if (g.zip_cpr.d != 0) {
         // long ranges of runs of 32 bytes and more (same branch for every thread): the block goes through
         // the ranges one after the other; a thread keeps its chunk number inside a run (ci) and walks down
         // the runs k, k + kstep, ... of the range, so everything that depends on the range is computed
@@ -985,49 +1041,6 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
                         char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
                         st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
                     }
-                }
-            }
-        }
-    } else if (g.zip_cpr.d != 0) {
-        // runs of 32 bytes and more (same branch for every thread): slot = (run k of the range, i-th
-        // target-aligned chunk that starts inside the run).  Such a chunk takes its units from run k and,
-        // past its end, from run k + 1 -- two base addresses and a compare per unit, no division.
-        const uint32_t cpr = g.zip_cpr.d;
-        const uint32_t nruns = cnt * (LONG_DST ? m : 1u);
-        for (uint32_t idx = tid; idx < total; idx += nthreads) {
-            const uint32_t q = fdiv(idx, g.zip_slots);
-            const uint32_t rem = idx - q * slots;
-            const uint32_t k = fdiv(rem, g.zip_cpr);
-            const uint32_t ci = rem - k * cpr;
-            const uint32_t r = LONG_DST ? q : fdiv(q, g.gl_m);
-            const uint32_t j = LONG_DST ? 0u : q - r * m;
-            const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
-            const uint32_t xs = k * run;
-            const uint32_t x = xs + ((16u - ((uint32_t(d0) + xs) & 15u)) & 15u) + (ci << 4);
-            if (k < nruns && x < xs + run && x + 16u <= rng_bytes) {
-                uint32_t base0, base1;      // shared-memory address of target byte p: base + p
-                if (LONG_DST) {
-                    const uint32_t rr = fdiv(k, g.gl_m);
-                    const uint32_t jj = k - rr * m;
-                    const bool wrap = jj + 1u == m;
-                    base0 = segbase[r * m + jj] + rr * run - xs;
-                    base1 = segbase[r * m + (wrap ? 0u : jj + 1u)] + (wrap ? rr + 1u : rr) * run - (xs + run);
-                } else {
-                    base0 = segbase[r] + (k * m + j) * run - xs;
-                    base1 = base0 + (m - 1u) * run;
-                }
-                union {
-                    uint4 v;
-                    T t[kPer];
-                } u;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    const uint32_t p = x + uint32_t(i * sizeof(T));
-                    u.t[i] = *reinterpret_cast<const T *>(tile + ((p >= xs + run ? base1 : base0) + p));
-                }
-                for (uint32_t f = 0; f < fanout; ++f) {
-                    char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
-                    st_stream(reinterpret_cast<uint4 *>(dbase + d0 + x), u.v);
                 }
             }
         }
@@ -1244,7 +1257,7 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
         // +4..12 %); large items, and items whose chunks are stored many times, keep 256
         const bool small = size_t(geo.stage_pitch) * geo.rows_per_item <= kZipSmallTile && geo.fanout <= 2;
         cfg.blockDim = dim3(small ? kBlockThreads / 2 : kBlockThreads);
-        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item;
+        cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item + size_t(geo.zip_lut_units) * 4;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -73,10 +73,13 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             assert G["zip_period"] == lb // math.gcd(16, lb) and G["zip_period_rows"] == 16 // math.gcd(16, lb)
             assert rpb * m * run // 16 >= 512 and G["zip_period"] * (m if not long_dst and run <= 16 else 1) <= 64
         if G["zip_cpr"]:
-            assert G["zip_by_range"] == (1 if G["zip_slots"] >= 256 else 0)
-            assert run >= 16 and unit < 16 and G["zip_cpr"] == -(-run // 16) and G["zip_slots"] == rpb * (m if long_dst else 1) * G["zip_cpr"]
+            assert not G["zip_period"] and not G["zip_lut_units"] and run >= 32 and unit < 16
+            assert G["zip_cpr"] == -(-run // 16) and G["zip_slots"] == rpb * (m if long_dst else 1) * G["zip_cpr"] >= 256
         else:
-            assert G["zip_by_range"] == 0 and G["zip_slots"] >= rpb * (m * run if long_dst else run) // 16
+            assert G["zip_slots"] >= rpb * (m * run if long_dst else run) // 16
+        if G["zip_lut_units"]:
+            assert not G["zip_period"] and G["zip_lut_units"] == rpb * (m * run if long_dst else run) // unit <= 2048
+            assert G["stage_pitch"] * rpi + 4 * G["zip_lut_units"] <= 42 * 1024
         assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
