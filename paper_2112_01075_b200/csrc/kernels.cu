@@ -824,6 +824,9 @@ __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
 // the covering 16-byte blocks; segbase[] remembers where byte 0 of the segment sits in shared memory.
 // Then the target ranges -- one per table row, or one per (table row, target tile) -- are written in
 // target-aligned 16-byte chunks assembled unit by unit from shared memory, ends in single units.
+// The kernel is bound by instruction issue, so the map from a chunk to the places of its units is made
+// cheap in one of three ways picked on the host (periodic walk, by-range walk, tabulated places; see
+// the branches of zip_body), with a flat walk of two divisions per unit as the fallback.
 template <bool LONG_DST, typename T, int NT>
 __device__ __forceinline__ const T *zip_src(const CopyGeometry &g, const unsigned char *tile, const uint32_t *segbase,
                                             uint32_t r, uint32_t j, uint32_t x)
