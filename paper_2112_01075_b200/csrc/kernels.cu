@@ -986,6 +986,10 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
                                      g, tile, segbase, r, jb, head + (tl << 4) + uint32_t(i * sizeof(T)))) - tile);
             for (uint32_t j = jb; j < jb + jn; ++j) {
                 uint32_t o = (j - jb) * run;
+                // fan-out 1: the target address is kept in a register (the pointer tables are read through
+                // generic loads, which the stores of the loop would otherwise order behind them)
+                char *const *dt = LONG_DST ? b.dtab : &P.dst[(b.t2 + j * g.gl_ts) * fanout];
+                char *d_first = dt[0] + d0 + head;
                 for (uint32_t c = tl; c < chunks; c += S, o += step) {
                     union {
                         uint4 v;
@@ -993,9 +997,11 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
                     } u;
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) u.t[i] = *reinterpret_cast<const T *>(tile + (at[i] + o));
-                    for (uint32_t f = 0; f < fanout; ++f) {
-                        char *dbase = LONG_DST ? b.dtab[f] : P.dst[(b.t2 + j * g.gl_ts) * fanout + f];
-                        st_stream(reinterpret_cast<uint4 *>(dbase + d0 + head + (c << 4)), u.v);
+                    if (fanout == 1) {
+                        st_stream(reinterpret_cast<uint4 *>(d_first + (c << 4)), u.v);
+                    } else {
+                        for (uint32_t f = 0; f < fanout; ++f)
+                            st_stream(reinterpret_cast<uint4 *>(dt[f] + d0 + head + (c << 4)), u.v);
                     }
                 }
             }
