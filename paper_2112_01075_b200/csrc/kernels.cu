@@ -777,6 +777,9 @@ __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
         return;
     }
     const uint32_t total = nr * cpb;
+    // fan-out 1: the target tile's address is kept in a register (the pointer table is read through
+    // generic loads, which the stores of the loop would otherwise order behind them)
+    char *const d_only = b.dtab[0] + b.o2;
     for (uint32_t idx = tid; idx < total; idx += kBlockThreads) {
         const uint32_t r = fdiv(idx, g.per_block_div);
         const uint32_t j = c0 + (idx - r * cpb);
@@ -784,8 +787,12 @@ __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
         if (j < ri.chunks) {
             const uint32_t x = ri.head + (j << 4);
             const uint4 v = lds_shifted(tile, ri.base + x);
-            const int64_t doff = b.o2 + rowtab[r].s2 + x;
-            for (uint32_t f = 0; f < fanout; ++f) st_stream(reinterpret_cast<uint4 *>(b.dtab[f] + doff), v);
+            if (fanout == 1) {
+                st_stream(reinterpret_cast<uint4 *>(d_only + rowtab[r].s2 + x), v);
+            } else {
+                const int64_t doff = b.o2 + rowtab[r].s2 + x;
+                for (uint32_t f = 0; f < fanout; ++f) st_stream(reinterpret_cast<uint4 *>(b.dtab[f] + doff), v);
+            }
         }
     }
     // ragged ends out of shared memory: head with the first column block, tail with the last
