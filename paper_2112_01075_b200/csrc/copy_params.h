@@ -100,6 +100,7 @@ struct CopyGeometry {
     FastDiv zip_cpr;                 // kModeZip: chunk slots per run in the by-range walk; d = 0: walk not used
     FastDiv zip_period;              // kModeZip: chunks after which the chunk -> units map repeats (d = 0: path not used)
     uint32_t zip_period_rows;        // kModeZip: rows of the zipped digit that one period spans
+    uint32_t zip_width;              // kModeZip: lanes that walk one table row together (a multiple of zip_period)
     uint32_t zip_lut_units;          // kModeZip: units of the longest range when their places are tabulated in shared memory (0: not)
     uint32_t zip_tile_fastest;       // kModeZip, long source rows: 1 = neighbouring lanes write to neighbouring target tiles
     FastDiv gl_n[kMaxGatherLevels];  // kModeGather: extents of those row digits, innermost first

@@ -281,22 +281,32 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             // threads of a block busy
             static const i64 kZipPeriodic = [] {
                 const char *v = std::getenv("REDIST_ZIP_PERIODIC");   // tuning knob: fewest chunks per table row for the periodic walk (0: never)
-                return i64(v ? std::atoi(v) : 512);
+                return i64(v ? std::atoi(v) : 1);
             }();
             const i64 L = long_dst ? row_bytes : run_bytes;         // bytes after which the target pattern repeats, up to alignment
             const i64 gc = std::gcd<i64>(16, L);
             const i64 pc = L / gc;
             G.zip_period = FastDiv{0, 0, 0};
             G.zip_period_rows = 0;
+            G.zip_width = 0;
             static const i64 kZipPc = [] {
                 const char *v = std::getenv("REDIST_ZIP_PC");   // tuning knob: longest period, in chunks
                 return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 64);
             }();
             // (with long source rows of runs up to 16 bytes a thread stays with one of the m target tiles)
             const i64 lanes_needed = !long_dst && run_bytes <= 16 ? pc * m : pc;
-            if (kZipPeriodic > 0 && rpb * row_bytes / 16 >= kZipPeriodic && lanes_needed <= kZipPc) {
+            const i64 range_chunks = rpb * L / 16;                  // chunks of one target range, at most
+            if (kZipPeriodic > 0 && rpb * row_bytes / 16 >= kZipPeriodic && lanes_needed <= kZipPc && range_chunks >= 2 * pc) {
                 G.zip_period = make_div(uint32_t(pc));
                 G.zip_period_rows = uint32_t(16 / gc);
+                // lanes per table row: about kZipLaneChunks chunks of a range for each, so that the decode of a
+                // lane's first chunk is shared by several chunks while short ranges still fill the block
+                static const i64 kZipLaneChunks = [] {
+                    const char *v = std::getenv("REDIST_ZIP_LANE_CHUNKS");   // tuning knob
+                    return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 4);
+                }();
+                const i64 want = std::max<i64>(1, (range_chunks + kZipLaneChunks * pc - 1) / (kZipLaneChunks * pc));
+                G.zip_width = uint32_t(std::min<i64>(want * pc, kBlockThreads / pc * pc));
             }
         }
         // By-range walk: for runs of 32 bytes and more of 4-byte units (64 and more of 8-byte units; nothing

@@ -966,7 +966,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
         }
     } else
     if (g.zip_period.d != 0) {
-        // long ranges (same branch for every thread): the map from a target chunk to the shared-memory
+        // periodic walk (same branch for every thread): the map from a target chunk to the shared-memory
         // places of its units repeats every zip_period chunks, shifted by a whole number of rows.  A thread
         // decodes the units of its first chunk once per table row and then strides through the range -- and,
         // with long source rows, through the m target tiles -- in steps of S chunks, a multiple of the
@@ -980,9 +980,14 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
             jn = 1;
             width = fdiv(nthreads, g.gl_m);
         }
-        const uint32_t S = fdiv(width, g.zip_period) * g.zip_period.d;
+        // The lanes are split into groups of S (a multiple of the period, at most zip_width: a few chunks of
+        // a range per lane); the groups share out the table rows of the item.
+        const uint32_t S = min(fdiv(width, g.zip_period) * g.zip_period.d, g.zip_width);
         const uint32_t step = fdiv(S, g.zip_period) * g.zip_period_rows * (LONG_DST ? run : run * m);
-        for (uint32_t r = 0; r < nr && tl < S; ++r) {
+        const uint32_t n_groups = width / S;
+        const uint32_t grp = tl / S;
+        tl -= grp * S;
+        for (uint32_t r = grp; r < nr && grp < n_groups; r += n_groups) {
             const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
             uint32_t head, chunks;
             split_run(rng_bytes, d0, head, chunks);
