@@ -223,8 +223,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const char *v = std::getenv("REDIST_ZIP_RUN");   // tuning knob: runs below this many bytes may take the zip kernels
         return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 2048);
     }();
-    // measured: aligned runs of 512 bytes and more are faster as plain bulk copies
-    const bool zip_run_ok = run_bytes < (G.aligned ? std::min<i64>(512, kZipRun) : kZipRun);
+    // measured: from 2 KiB the plain bulk copy (aligned runs) and the ragged chunk walk are faster
+    const bool zip_run_ok = run_bytes < kZipRun;
     i64 zip_n = 0;
     if (kZip > 0 && kBulk && (kZip >= 2 || g_levels < 0) && vec >= 4 && zip_run_ok && G.inner_digit != 0xffffffffu &&
         (m1[kp] == 1 || m2[kp] == 1) && !rows.empty()) {

@@ -56,7 +56,6 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         long_dst = G["gl_long_dst"] == 1
         m = max(m1, m2)
         assert unit >= 4 and run < 2048 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 16
-        assert run < 512 or unit < 16
         assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
         assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
         n = G["row_n"][-1]
