@@ -290,9 +290,10 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             G.zip_period_rows = 0;
             G.zip_width = 0;
             static const i64 kZipPc = [] {
-                // tuning knob: longest period, in chunks (at most 128: a block may have only 128 threads)
+                // tuning knob: longest period, in chunks (the lanes of one block must span it; above 128 the
+                // launch uses 256 threads)
                 const char *v = std::getenv("REDIST_ZIP_PC");
-                return i64(v && std::atoi(v) > 0 ? std::min(std::atoi(v), kBlockThreads / 2) : kBlockThreads / 2);
+                return i64(v && std::atoi(v) > 0 ? std::min(std::atoi(v), kBlockThreads - 1) : kBlockThreads - 1);
             }();
             // (with long source rows of runs up to 16 bytes a thread stays with one of the m target tiles)
             const i64 lanes_needed = !long_dst && run_bytes <= 16 ? pc * m : pc;

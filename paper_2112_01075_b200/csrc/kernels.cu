@@ -1276,7 +1276,8 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
         // small items stored to one or two replicas: eight and more blocks fit an SM, and half as many threads
         // per block means half as many threads that decode the item and wait for its copies (measured
         // +4..12 %); large items, and items whose chunks are stored many times, keep 256
-        const bool small = size_t(geo.stage_pitch) * geo.rows_per_item <= kZipSmallTile && geo.fanout <= 2;
+        const bool small = size_t(geo.stage_pitch) * geo.rows_per_item <= kZipSmallTile && geo.fanout <= 2 &&
+                           geo.zip_period.d * (geo.gl_long_dst == 0 && geo.zip_tile_fastest ? geo.gl_m.d : 1u) <= kBlockThreads / 2;
         cfg.blockDim = dim3(small ? kBlockThreads / 2 : kBlockThreads);
         cfg.dynamicSmemBytes = size_t(geo.stage_pitch) * geo.rows_per_item + size_t(geo.zip_lut_units) * 4;
         cfg.stream = stream;

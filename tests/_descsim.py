@@ -70,7 +70,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             import math
             lb = m * run if long_dst else run
             assert G["zip_period"] == lb // math.gcd(16, lb) and G["zip_period_rows"] == 16 // math.gcd(16, lb)
-            assert G["zip_period"] * (m if not long_dst and run <= 16 else 1) <= 128 and rpb * lb // 16 >= 2 * G["zip_period"]
+            assert G["zip_period"] * (m if not long_dst and run <= 16 else 1) <= 255 and rpb * lb // 16 >= 2 * G["zip_period"]
             assert G["zip_width"] % G["zip_period"] == 0 and G["zip_period"] <= G["zip_width"] <= 256
         if G["zip_cpr"]:
             assert not G["zip_period"] and not G["zip_lut_units"] and run >= 32 and unit < 16
