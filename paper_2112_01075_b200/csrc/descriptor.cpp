@@ -418,6 +418,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             rpi = std::max<i64>(1, std::min<i64>(rpi, std::min<i64>(kRaggedBulkRows, kRaggedKb * 1024 / pitch)));
             ragged_bulk = true;
             G.stage_pitch = uint32_t(pitch);
+            // lanes that walk one row together: about four chunks each, a whole number of warps
+            // (and no more groups than rows)
+            i64 w = 32;
+            while (w < kBlockThreads && (w * 4 < cpb || (kBlockThreads / w) > rpi)) w *= 2;
+            G.lanes = uint32_t(w);
         }
         G.mode = units ? kModeUnits : kModeChunks;
         G.rows = uint32_t(tab_rows);
