@@ -152,6 +152,17 @@ def test_register_kernels_behind_the_tuning_knobs():
     _random_problems_in_a_fresh_process({"REDIST_BULK": "0", "REDIST_GATHER": "0"}, 300, "v == {0, 1, 2, 3}")
 
 
+@pytest.mark.parametrize("env", [
+    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_LUT": "0", "REDIST_ZIP_PER_RUN": "0"},     # flat walk only
+    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_LUT": "0", "REDIST_ZIP_BY_RANGE": "1"},    # by-range walk, else flat
+    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_PER_RUN": "0"},                            # tabulated places, else flat
+], ids=["flat", "by_range", "tabulated"])
+def test_zip_kernels_with_each_chunk_map(env):
+    """The zip kernels pick one of several ways to map a target chunk to its units; the knobs force the
+    ones that the default choice (periodic walk) seldom leaves work for."""
+    _random_problems_in_a_fresh_process(env, 400, "7 in v")
+
+
 def test_gather_walk_wherever_it_applies():
     """REDIST_GATHER=2 sends every eligible launch through the gather walk, including long source rows
     that are scattered into several target tiles and 16-byte units (not chosen by default)."""
