@@ -35,7 +35,8 @@
 //                on both sides: source segments staged in shared memory by bulk copies (zip_body).
 // Index decoding uses multiply-shift division by host-computed constants; the per-item decode (box ->
 // tiles and base offsets) is amortised over ~32 KiB of data.  Every kernel starts with
-// griddepcontrol.wait / launch_dependents (programmatic dependent launch).
+// griddepcontrol.launch_dependents and places griddepcontrol.wait after the decode of its first work
+// item, just before its first access to global memory (programmatic dependent launch).
 #include <cuda_runtime.h>
 
 #include <cstdlib>
@@ -56,6 +57,11 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv &f)
 {
     return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
 }
+
+// Programmatic dependent launch: a kernel may start while the previous kernel of the stream still runs;
+// it must not touch global memory before this wait (kernel parameters and shared memory are free), so
+// every body decodes its first work item first and waits just before its first load.
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // streaming accesses: the data is touched once
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
@@ -211,6 +217,7 @@ __device__ __forceinline__ void rows_body(const CopyParams<NT> &P)
     const bool active = ty < rpp;
     for (uint32_t item = blockIdx.x; item < g.n_items; item += gridDim.x) {
         const BoxBase b = decode_box(P, item);
+        if (item == blockIdx.x) wait_for_previous_kernel();
         const char *sb = b.sbase + int64_t(tx) * 16;
         const int64_t dcol = b.o2 + int64_t(tx) * 16;
         const uint32_t row0 = b.part * g.rows_per_item;
@@ -269,6 +276,7 @@ __device__ __forceinline__ void chunks_body(const CopyParams<NT> &P, RowEntry *r
         const uint32_t group = fdiv(b.part, g.col_blocks);
         const uint32_t cb = b.part - group * g.col_blocks.d;
         const uint32_t nr = fill_rowtab(g, rowtab, group);
+        if (item == blockIdx.x) wait_for_previous_kernel();
         const uint32_t total = nr * cpb;
         const uint32_t c0 = cb * cpb;
         for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
@@ -343,6 +351,7 @@ __device__ __forceinline__ void units_walk(const CopyParams<NT> &P, RowEntry *ro
         const uint32_t group = fdiv(b.part, g.col_blocks);
         const uint32_t cb = b.part - group * g.col_blocks.d;
         const uint32_t nr = fill_rowtab(g, rowtab, group);
+        if (item == blockIdx.x) wait_for_previous_kernel();
         const uint32_t total = nr * cpb;
         const uint32_t c0 = cb * cpb;
         for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
@@ -404,7 +413,6 @@ __device__ __forceinline__ void copy_body(const CopyParams<NT> &P)
     // on the stream drains; nothing is read or written before that kernel has completed and its
     // stores are visible.  The next kernel is released to do the same as soon as every block of this
     // grid has started.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (VARIANT == 0) {
         rows_body<NT>(P);
@@ -473,6 +481,7 @@ __device__ __forceinline__ void gather_body(const CopyParams<NT> &P, RowEntry *r
         const uint32_t group = fdiv(b.part, g.col_blocks);
         const uint32_t cb = b.part - group * g.col_blocks.d;
         const uint32_t nr = fill_rowtab(g, rowtab, group);
+        if (item == blockIdx.x) wait_for_previous_kernel();
         const uint32_t total = nr * ns * cpb;
         const uint32_t c0 = cb * cpb;
         for (uint32_t base = tid; base < total; base += kBlockThreads * kU) {
@@ -555,7 +564,6 @@ __device__ __forceinline__ void gather_dispatch(const CopyParams<NT> &P)
     template <bool LONG_DST, int NT>                                                                 \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
-        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         gather_dispatch<LONG_DST, NT>(P);                                                            \
     }
@@ -608,8 +616,9 @@ __device__ __forceinline__ void bulk_body(const CopyParams<NT> &P)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // (the wait for the previous kernel of the stream comes just before the first access to global
+    // memory: decoding the item only reads kernel parameters)
     const uint32_t item = blockIdx.x;
     if (item >= g.n_items) return;
     const BoxBase b = decode_box(P, item);
@@ -635,8 +644,9 @@ __device__ __forceinline__ void bulk_body(const CopyParams<NT> &P)
     int64_t s1 = 0, s2 = 0;
     const bool mine = tid < nr;          // at most one row per thread (the host guarantees nr <= kBulkThreads)
     const uint32_t slot = smem_addr(stage) + tid * bytes;
+    if (mine) row_offsets(g, row0 + tid, s1, s2, int(g.n_row));
+    wait_for_previous_kernel();
     if (mine) {
-        row_offsets(g, row0 + tid, s1, s2, int(g.n_row));
         const char *src = b.sbase + s1 + int64_t(seg_off);
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(slot), "l"(src), "r"(bytes), "r"(mbar)
@@ -743,6 +753,7 @@ __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    wait_for_previous_kernel();
     for (uint32_t r = tid; r < nr; r += kBlockThreads) {
         RowEntry e;
         row_offsets(g, row0 + r, e.s1, e.s2, int(g.n_row_tab));
@@ -921,6 +932,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    wait_for_previous_kernel();
     for (uint32_t t = tid; t < nr * nseg; t += nthreads) {
         const uint32_t r = fdiv(t, g.gl_m);
         const uint32_t j = LONG_DST ? t - r * m : 0u;
@@ -1177,7 +1189,6 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
         __shared__ RowEntry rowtab[kZipSegments];                                                    \
         __shared__ uint32_t segbase[kZipSegments];                                                   \
         __shared__ __align__(8) unsigned long long mbar_storage;                                     \
-        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         const uint32_t mbar = smem_addr(&mbar_storage);                                              \
         switch (P.g.unit_bytes) {                                                                    \
@@ -1197,7 +1208,6 @@ REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
     template <int NT>                                                                                \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
-        asm volatile("griddepcontrol.wait;" ::: "memory");                                           \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         ragged_bulk_body<NT>(P);                                                                     \
     }
