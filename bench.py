@@ -335,7 +335,8 @@ def run_ours(args):
             "value": round(world * step_bytes / (other_ms / n_side * 1e-3) / 1e9, 1), "unit": UNIT,
             "ms_per_step": round(other_ms / n_side, 5), "steps": n_side,
             "note": "same steps, " + ("plain redist_execute calls" if args.graph else
-                                      "replayed from CUDA graphs of captured redist_execute calls")},
+                                      "replayed from CUDA graphs of captured redist_execute calls, one step per "
+                                      "graph (no dependent-launch overlap from one graph launch to the next)")},
         "legs": [{"name": l.w.name, "steps": l.plan.step_kinds(), "kernels": l.plan.launch_kernels(),
                   "gbs": round(l.eff_bytes / (statistics.mean(per[q]) * 1e-3) / 1e9, 1),
                   "us": round(statistics.mean(per[q]) * 1e3, 2)} for q, l in enumerate(legs)],
