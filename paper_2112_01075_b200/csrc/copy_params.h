@@ -14,7 +14,8 @@
 // Item numbering: the pieces of one long row (the m1*m2 units of the last differing dimension that
 // share a source or target tile row) are consecutive items, so blocks that run at the same time fill
 // the same memory sectors and partial-sector writes merge in L2 instead of being written back alone;
-// then come the row groups of a box, then the boxes.
+// then come the boxes of the other unit digits whose units share cache lines (fast_boxes of them), then
+// the row groups of a box, then the remaining boxes.
 //
 // Aligned items whose row segments are at least 512 bytes (`bulk == 1`) are moved by TMA bulk copies
 // through shared memory instead of by the register kernels; the item geometry is the same.
@@ -85,6 +86,7 @@ struct CopyGeometry {
     FastDiv per_block_div;           // flat walk: division by per_block
     FastDiv col_blocks;              // flat walk: column blocks per row (1 in kModeRows)
     FastDiv items_per_box;
+    FastDiv fast_boxes;              // boxes of the trailing unit digits that vary faster than the row groups of a box (1: none)
     FastDiv inner_n;                 // pieces of one long row that consecutive items handle (1: none, or all in one item)
     uint32_t inner_digit;            // unit digit those pieces belong to
     uint32_t inner_span;             // units of that digit per long row (m1 * m2)

@@ -101,6 +101,45 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.unit_n[u] = make_div(uint32_t(nq[kp] / inner));
         n_boxes /= inner;
     }
+    // Unit digits whose units sit side by side within a few cache lines of a tile (m > 1 and a byte stride
+    // below kFastStride on that side) are moved to the end of the digit list: they become the fastest
+    // part of the box number, and -- see decode_box -- vary faster than the row groups of a box, so that the
+    // blocks which share those lines run at the same time and partial sectors merge in L2.
+    static const i64 kFastStride = [] {
+        const char *v = std::getenv("REDIST_FAST_STRIDE");   // tuning knob: 0 switches the reordering off
+        return i64(v ? std::atoi(v) : 16384);
+    }();
+    G.fast_boxes = make_div(1);
+    {
+        std::vector<uint32_t> slow, fast;
+        for (uint32_t u = 0; u < nu; ++u) {
+            const bool f = u != G.inner_digit && G.unit_n[u].d > 1 &&
+                           ((G.unit_m2[u].d > 1 && G.unit_b2[u] < kFastStride) || (G.unit_m1[u].d > 1 && G.unit_b1[u] < kFastStride));
+            (f ? fast : slow).push_back(u);
+        }
+        if (!fast.empty()) {
+            CopyGeometry T = G;
+            uint32_t pos = 0;
+            i64 nfast = 1;
+            auto put = [&](uint32_t u) {
+                G.unit_n[pos] = T.unit_n[u];
+                G.unit_m1[pos] = T.unit_m1[u];
+                G.unit_m2[pos] = T.unit_m2[u];
+                G.unit_ts1[pos] = T.unit_ts1[u];
+                G.unit_ts2[pos] = T.unit_ts2[u];
+                G.unit_b1[pos] = T.unit_b1[u];
+                G.unit_b2[pos] = T.unit_b2[u];
+                if (u == T.inner_digit) G.inner_digit = pos;
+                ++pos;
+            };
+            for (uint32_t u : slow) put(u);
+            for (uint32_t u : fast) {
+                nfast *= T.unit_n[u].d;
+                put(u);
+            }
+            G.fast_boxes = make_div(uint32_t(nfast));
+        }
+    }
     // row digits inside a box: the dimensions before kp, merged where both sides stay contiguous
     std::vector<RowDigit> rows;
     for (int k = 0; k < kp; ++k) {

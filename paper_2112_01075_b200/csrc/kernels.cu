@@ -175,10 +175,12 @@ template <int NT>
 __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t item)
 {
     const CopyGeometry &g = P.g;
+    // item = ((slow boxes * items_per_box + part) * fast_boxes + fast box) * inner_n + piece
     const uint32_t outer = fdiv(item, g.inner_n);
     const uint32_t piece = item - outer * g.inner_n.d;
-    const uint32_t box = fdiv(outer, g.items_per_box);
-    uint32_t t1 = 0, t2 = 0, rem = box;
+    const uint32_t rest = fdiv(outer, g.fast_boxes);
+    const uint32_t slow = fdiv(rest, g.items_per_box);
+    uint32_t t1 = 0, t2 = 0, rem = slow * g.fast_boxes.d + (outer - rest * g.fast_boxes.d);
     int64_t o1 = 0, o2 = 0;
     for (int u = int(g.n_unit) - 1; u >= 0; --u) {
         const uint32_t nxt = fdiv(rem, g.unit_n[u]);
@@ -199,7 +201,7 @@ __device__ __forceinline__ BoxBase decode_box(const CopyParams<NT> &P, uint32_t 
     b.o2 = o2;
     b.t1 = t1;
     b.t2 = t2;
-    b.part = outer - box * g.items_per_box.d;
+    b.part = rest - slow * g.items_per_box.d;
     return b;
 }
 
