@@ -200,6 +200,12 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         fan = p.n_devices / nt;
     }
     const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
+    // items of the plain bulk-copy kernels at fan-out 1: measured best at 20 KiB once the kernels wait for
+    // their predecessor only after decoding the item (finer tail, more blocks ready behind the wait)
+    static const i64 kBulkItemKb = [] {
+        const char *v = std::getenv("REDIST_BULK_ITEM_KB");   // tuning knob: KiB per item of the bulk-copy kernels at fan-out 1
+        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 20);
+    }();
     // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
     // thread, the item staged in at most 47 KiB of shared memory)
     static const bool kBulk = [] {
@@ -212,6 +218,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }();
     const i64 max_chunks = run_bytes / 16;           // whole 16-byte chunks a run can hold
     if (max_chunks >= (1ll << 31)) return REDIST_EUNSUPPORTED;
+    const i64 bulk_item_bytes =
+        kItemKb == 0 && kBulk && G.aligned && fan == 1 && run_bytes >= kBulkMin ? kBulkItemKb * 1024 : kItemBytes;
     i64 ipb;
     G.lanes = kBlockThreads;
     G.rows_per_pass = 1;
@@ -420,6 +428,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         ipb = (tab_rows + rpi - 1) / rpi * ncb;
     } else if (G.aligned && max_chunks <= kBlockThreads) {
         // aligned short runs: `lanes` threads per row, one chunk each
+        const i64 kItemBytes = bulk_item_bytes;
         const i64 lanes = max_chunks;
         G.mode = kModeRows;
         G.lanes = uint32_t(lanes);
@@ -433,6 +442,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     } else {
         // flat walk over (row, chunk) -- or, for short ragged runs, over (table row, unit piece) where a
         // table row carries all the runs of the innermost row digit
+        const i64 kItemBytes = bulk_item_bytes;
         const bool units = run_bytes < 256;
         i64 tab_inner = 1, tab_rows = n_rows;
         if (units && run_bytes <= 16 && !rows.empty() && rows.back().n * (run_bytes / vec) < (1ll << 30)) {
