@@ -200,10 +200,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         fan = p.n_devices / nt;
     }
     const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
-    // items of the plain bulk-copy kernels at fan-out 1: measured best at 20 KiB once the kernels wait for
-    // their predecessor only after decoding the item (finer tail, more blocks ready behind the wait)
+    // Items of the plain bulk-copy kernels: measured best at 20 KiB (12 / 6 KiB for fan-out >= 2 / >= 4) once
+    // the kernels wait for their predecessor only after decoding the item -- finer tail, more blocks ready
+    // behind the wait.
     static const i64 kBulkItemKb = [] {
-        const char *v = std::getenv("REDIST_BULK_ITEM_KB");   // tuning knob: KiB per item of the bulk-copy kernels at fan-out 1
+        const char *v = std::getenv("REDIST_BULK_ITEM_KB");   // tuning knob: KiB per item of the bulk-copy kernels at fan-out 1 (2-3: 0.6x, 4 and more: 0.3x)
         return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 20);
     }();
     // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
@@ -218,8 +219,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }();
     const i64 max_chunks = run_bytes / 16;           // whole 16-byte chunks a run can hold
     if (max_chunks >= (1ll << 31)) return REDIST_EUNSUPPORTED;
-    const i64 bulk_item_bytes =
-        kItemKb == 0 && kBulk && G.aligned && fan == 1 && run_bytes >= kBulkMin ? kBulkItemKb * 1024 : kItemBytes;
+    const i64 bulk_item_bytes = kItemKb == 0 && kBulk && G.aligned && run_bytes >= kBulkMin
+                                    ? (fan >= 4 ? kBulkItemKb * 3 / 10 : fan >= 2 ? kBulkItemKb * 6 / 10 : kBulkItemKb) * 1024
+                                    : kItemBytes;
     i64 ipb;
     G.lanes = kBlockThreads;
     G.rows_per_pass = 1;
