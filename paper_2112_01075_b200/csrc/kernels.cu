@@ -1234,6 +1234,14 @@ REDIST_DEFINE_KERNEL(redist_allgather_kernel)
 REDIST_DEFINE_KERNEL(redist_allpermute_kernel)
 REDIST_DEFINE_KERNEL(redist_fused_kernel)
 
+// Launch attribute of every kernel: programmatic stream serialization (the kernel may start before its
+// predecessor in the stream has finished; see wait_for_previous_kernel).
+static int pdl_allowed()
+{
+    static const bool kSerialize = std::getenv("REDIST_NO_PDL") != nullptr;   // tuning knob: plain stream order
+    return kSerialize ? 0 : 1;
+}
+
 template <int VARIANT, int NT>
 cudaError_t launch_one(int kernel, const CopyParams<NT> &P, int grid, cudaStream_t stream)
 {
@@ -1245,7 +1253,6 @@ cudaError_t launch_one(int kernel, const CopyParams<NT> &P, int grid, cudaStream
     case 3: case 4: fn = redist_allpermute_kernel<VARIANT, NT>; break;
     default: fn = redist_fused_kernel<VARIANT, NT>; break;
     }
-    static const bool kSerialize = std::getenv("REDIST_NO_PDL") != nullptr;   // tuning knob
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(grid));
     cfg.blockDim = dim3(kBlockThreads);
@@ -1253,7 +1260,7 @@ cudaError_t launch_one(int kernel, const CopyParams<NT> &P, int grid, cudaStream
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = kSerialize ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, P);
@@ -1283,7 +1290,7 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, fn, P);
@@ -1306,7 +1313,7 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
             cfg.stream = stream;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             return cudaLaunchKernelEx(&cfg, fn, P);
@@ -1334,7 +1341,7 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, fn, P);
@@ -1355,7 +1362,7 @@ cudaError_t launch_nt(int kernel, const CopyGeometry &geo, const char *const *sr
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, fn, P);
