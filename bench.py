@@ -255,6 +255,8 @@ def run_ours(args):
     gen.manual_seed(2112010752 + rank)
     ws = legs_of(args.workload)
     flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
+    if args.cost_permute:
+        flags |= api.COST_PERMUTE
     legs = [DeviceLeg(w, flags, torch, api, gen) for w in ws]
     step_bytes = sum(l.eff_bytes for l in legs)
 
@@ -477,6 +479,8 @@ def run_sweep(args):
         pairs, label = wl.evaluation_like_problems(args.pairs), \
             "eval: %d random problems shaped like the paper's evaluation sample (3 mesh axes, <= 6-D, 64-800 MB)"
     flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
+    if args.cost_permute:
+        flags |= api.COST_PERMUTE
     G = None
     stream = torch.cuda.current_stream()
     rows = []
@@ -519,13 +523,14 @@ def run_sweep(args):
                      "launches": plan.num_launches, "run_bytes": min(i.run_bytes for i in li),
                      "fanout": max(i.fanout for i in li), "eff_bytes": eff, "us": round(ms * 1e3, 1),
                      "gbs": round(eff / (ms * 1e-3) / 1e9, 1),
-                     "scratch_per_device": plan.scratch_bytes_per_device})
+                     "scratch_per_device": plan.scratch_bytes_per_device, "plan_cost_elems": plan.cost})
         del src, dst, owned, scratch, call, plan
         torch.cuda.empty_cache()
     g = [r["gbs"] for r in rows]
     peak, how = measured_peak()
     line = {"metric": METRIC, "workload": label % len(rows),
-            "fuse": args.fuse, "geomean_gbs": round(math.exp(sum(math.log(x) for x in g) / len(g)), 1),
+            "fuse": args.fuse, "cost_permute": bool(args.cost_permute),
+            "plan_cost_elems_total": sum(r["plan_cost_elems"] for r in rows), "geomean_gbs": round(math.exp(sum(math.log(x) for x in g) / len(g)), 1),
             "min_gbs": min(g), "max_gbs": max(g), "median_gbs": statistics.median(g),
             "total_gbs": round(sum(r["eff_bytes"] for r in rows) / sum(r["us"] * 1e-6 for r in rows) / 1e9, 1),
             "peak": peak, "peak_source": how, "pairs_below_70pct_of_peak": sum(x < 0.7 * peak for x in g)}
@@ -636,6 +641,8 @@ def main():
     ap.add_argument("--only", default="", help="sweeps: comma-separated problem names to run")
     ap.add_argument("--dump", default="", help="sweeps: write the per-problem table to this JSON file")
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
+    ap.add_argument("--cost-permute", action="store_true",
+                    help="plan with REDIST_COST_PERMUTE (the final permutation counted when choosing the sequence)")
     ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")
     ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays instead of plain stream launches")
     ap.add_argument("--no-graph", action="store_true", help=argparse.SUPPRESS)   # accepted, the default

@@ -60,7 +60,8 @@ typedef struct redist_type {
 
 typedef struct redist_plan_s redist_plan_t;   /* opaque, host memory, immutable once created */
 
-/* plan flags: exactly one execution mode, optionally or-ed with REDIST_NO_OVERPARTITION */
+/* plan flags: exactly one execution mode, optionally or-ed with REDIST_NO_OVERPARTITION and/or
+   REDIST_COST_PERMUTE */
 enum {
     REDIST_FUSE_ADJACENT = 0,    /* default: adjacent steps of the sequence run as one kernel wherever
                                     the fused copy keeps contiguous runs of at least 64 bytes         */
@@ -70,8 +71,16 @@ enum {
     REDIST_NAIVE = 3,            /* comparison baseline only: gather the whole global array, then
                                     slice (the "easy" redistribution, Section 4.3)                    */
     REDIST_MODE_MASK = 3,
-    REDIST_NO_OVERPARTITION = 16 /* forbid dynslice steps that partition the array over more mesh
+    REDIST_NO_OVERPARTITION = 16,/* forbid dynslice steps that partition the array over more mesh
                                     axes than the target type uses (over-partitioning, Section 7.2)  */
+    REDIST_COST_PERMUTE = 32     /* count the final allpermute when choosing the sequence.  The search
+                                    of Section 7.3 weighs only dynslice / alltoall / allgather (the
+                                    permutation "is not a graph edge") and appends the permutation
+                                    afterwards; with this flag the sequences whose own cost lies below
+                                    that plan's total are lowered too and the cheapest total (sequence
+                                    plus permutation, cost model of Section 6.2) is kept.  The result
+                                    never costs more than the default plan and obeys the same memory
+                                    bound; planning takes longer.                                     */
 };
 
 enum { REDIST_MAX_RANK = 8, REDIST_MAX_MESH_AXES = 16, REDIST_MAX_DEVICES = 1024 };

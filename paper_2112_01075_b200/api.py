@@ -20,6 +20,7 @@ LIB_PATH = os.environ.get("REDIST_LIB") or os.path.join(HERE, "libredist_b200.so
 
 FUSE_ADJACENT, FUSE_NONE, FUSE_ALL, NAIVE = 0, 1, 2, 3
 NO_OVERPARTITION = 16
+COST_PERMUTE = 32
 MAX_RANK = 8
 STATIC_SCRATCH_BYTES = 8 << 20
 

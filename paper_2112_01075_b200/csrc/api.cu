@@ -135,7 +135,7 @@ redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const 
         return REDIST_EINVAL;
     if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4 && elem_bytes != 8 && elem_bytes != 16)
         return REDIST_EINVAL;
-    if (flags & ~uint32_t(REDIST_MODE_MASK | REDIST_NO_OVERPARTITION)) return REDIST_EINVAL;
+    if (flags & ~uint32_t(REDIST_MODE_MASK | REDIST_NO_OVERPARTITION | REDIST_COST_PERMUTE)) return REDIST_EINVAL;
     i64 N = 1;
     for (int a = 0; a < n_mesh_axes; ++a) {
         if (mesh_shape[a] < 1) return REDIST_EINVAL;

@@ -9,6 +9,7 @@
 // allpermute is appended and moved before any trailing allgathers (Section 7.3).
 #include <algorithm>
 #include <cstring>
+#include <limits>
 #include <map>
 #include <queue>
 
@@ -114,6 +115,79 @@ struct Search {
         }
     }
 
+    // Every weak collective that applies to the weak type `key` (its last entry is the phase of the
+    // normal form: 0 = dynslices still allowed, 1 = alltoalls, 2 = allgathers only), reported as
+    // relax(successor, weight, step).
+    template <class R>
+    void expand(const std::vector<uint8_t> &key, bool no_over, R relax) const
+    {
+        using Key = std::vector<uint8_t>;
+        const int phase = key[r * np];
+        std::vector<i64> c(r);
+        i64 L = 1;
+        std::vector<int> used(np, 0);
+        for (int k = 0; k < r; ++k) {
+            c[k] = p.global_shape[k] / shard_factor(key, k);
+            L *= c[k];
+            for (int q = 0; q < np; ++q) used[q] += key[k * np + q];
+        }
+        // dynslice(i, m): m from unused primes, m | c_i, weight 0 (phase 0 only: normal form)
+        if (phase == 0) {
+            std::vector<int> caps(np);
+            for (int q = 0; q < np; ++q) caps[q] = mesh_cnt[q] - used[q];
+            for (int i = 0; i < r; ++i)
+                for_each_factor(caps, [&](const std::vector<int> &e) {
+                    i64 m = pow_of(e);
+                    if (c[i] % m) return;
+                    if (no_over)
+                        for (int q = 0; q < np; ++q) {
+                            if (e[q] == 0) continue;
+                            int tgt_used = 0;
+                            for (int k = 0; k < r; ++k) tgt_used += tgt_exps[k * np + q];
+                            if (key[i * np + q] + e[q] > tgt_exps[i * np + q] || used[q] + e[q] > tgt_used)
+                                return;
+                        }
+                    Key nk = key;
+                    for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] + e[q]);
+                    relax(nk, 0, WeakStep{REDIST_STEP_DYNSLICE, i, -1, e, m});
+                });
+        }
+        // alltoall(i -> j, m): m from the primes on dim i, m | c_j, weight localsize (phases 0, 1)
+        if (phase <= 1) {
+            for (int i = 0; i < r; ++i) {
+                std::vector<int> caps(np);
+                for (int q = 0; q < np; ++q) caps[q] = key[i * np + q];
+                for (int j = 0; j < r; ++j) {
+                    if (j == i) continue;
+                    for_each_factor(caps, [&](const std::vector<int> &e) {
+                        i64 m = pow_of(e);
+                        if (c[j] % m) return;
+                        Key nk = key;
+                        for (int q = 0; q < np; ++q) {
+                            nk[i * np + q] = uint8_t(nk[i * np + q] - e[q]);
+                            nk[j * np + q] = uint8_t(nk[j * np + q] + e[q]);
+                        }
+                        nk[r * np] = 1;
+                        relax(nk, L, WeakStep{REDIST_STEP_ALLTOALL, i, j, e, m});
+                    });
+                }
+            }
+        }
+        // allgather(i, m): m from the primes on dim i, weight = new localsize <= M
+        for (int i = 0; i < r; ++i) {
+            std::vector<int> caps(np);
+            for (int q = 0; q < np; ++q) caps[q] = key[i * np + q];
+            for_each_factor(caps, [&](const std::vector<int> &e) {
+                i64 m = pow_of(e);
+                if (L > M / m) return;   // L * m <= M, overflow-safe
+                Key nk = key;
+                for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] - e[q]);
+                nk[r * np] = 2;
+                relax(nk, L * m, WeakStep{REDIST_STEP_ALLGATHER, i, -1, e, m});
+            });
+        }
+    }
+
     // All shortest paths (minimal cost, then minimal number of steps), up to `max_paths` of them:
     // the weak graph cannot tell them apart, the lowering can (one may need no final permutation).
     bool run(std::vector<std::vector<WeakStep>> &paths, size_t max_paths)
@@ -174,15 +248,6 @@ struct Search {
                 continue;
             }
             const Key &key = cur.key;
-            const int phase = key[r * np];
-            std::vector<i64> c(r);
-            i64 L = 1;
-            std::vector<int> used(np, 0);
-            for (int k = 0; k < r; ++k) {
-                c[k] = p.global_shape[k] / shard_factor(key, k);
-                L *= c[k];
-                for (int q = 0; q < np; ++q) used[q] += key[k * np + q];
-            }
             auto relax = [&](const Key &nk, i64 w, const WeakStep &ws) {
                 i64 nc = cur.cost + w;
                 int ns = cur.nsteps + 1;
@@ -198,61 +263,7 @@ struct Search {
                 info[nk] = Info{nc, ns, {{key, ws}}, false};
                 pq.push(QE{nc, ns, seq++, nk});
             };
-            // dynslice(i, m): m from unused primes, m | c_i, weight 0 (phase 0 only: normal form)
-            if (phase == 0) {
-                std::vector<int> caps(np);
-                for (int q = 0; q < np; ++q) caps[q] = mesh_cnt[q] - used[q];
-                for (int i = 0; i < r; ++i)
-                    for_each_factor(caps, [&](const std::vector<int> &e) {
-                        i64 m = pow_of(e);
-                        if (c[i] % m) return;
-                        if (no_over)
-                            for (int q = 0; q < np; ++q) {
-                                if (e[q] == 0) continue;
-                                int tgt_used = 0;
-                                for (int k = 0; k < r; ++k) tgt_used += tgt_exps[k * np + q];
-                                if (key[i * np + q] + e[q] > tgt_exps[i * np + q] || used[q] + e[q] > tgt_used)
-                                    return;
-                            }
-                        Key nk = key;
-                        for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] + e[q]);
-                        relax(nk, 0, WeakStep{REDIST_STEP_DYNSLICE, i, -1, e, m});
-                    });
-            }
-            // alltoall(i -> j, m): m from the primes on dim i, m | c_j, weight localsize (phases 0, 1)
-            if (phase <= 1) {
-                for (int i = 0; i < r; ++i) {
-                    std::vector<int> caps(np);
-                    for (int q = 0; q < np; ++q) caps[q] = key[i * np + q];
-                    for (int j = 0; j < r; ++j) {
-                        if (j == i) continue;
-                        for_each_factor(caps, [&](const std::vector<int> &e) {
-                            i64 m = pow_of(e);
-                            if (c[j] % m) return;
-                            Key nk = key;
-                            for (int q = 0; q < np; ++q) {
-                                nk[i * np + q] = uint8_t(nk[i * np + q] - e[q]);
-                                nk[j * np + q] = uint8_t(nk[j * np + q] + e[q]);
-                            }
-                            nk[r * np] = 1;
-                            relax(nk, L, WeakStep{REDIST_STEP_ALLTOALL, i, j, e, m});
-                        });
-                    }
-                }
-            }
-            // allgather(i, m): m from the primes on dim i, weight = new localsize <= M
-            for (int i = 0; i < r; ++i) {
-                std::vector<int> caps(np);
-                for (int q = 0; q < np; ++q) caps[q] = key[i * np + q];
-                for_each_factor(caps, [&](const std::vector<int> &e) {
-                    i64 m = pow_of(e);
-                    if (L > M / m) return;   // L * m <= M, overflow-safe
-                    Key nk = key;
-                    for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] - e[q]);
-                    nk[r * np] = 2;
-                    relax(nk, L * m, WeakStep{REDIST_STEP_ALLGATHER, i, -1, e, m});
-                });
-            }
+            expand(key, no_over, relax);
         }
         if (found.empty()) return false;
         paths.clear();
@@ -284,6 +295,114 @@ struct Search {
             }
         }
         return !paths.empty();
+    }
+    // Sequences of weak cost strictly below `bound` and of at most `max_steps` steps, those with the
+    // cheapest continuation first, at most `max_paths` of them.  The search of Section 7.3 leaves the
+    // final permutation out of the edge weights ("not a graph edge"), so a sequence that is not a
+    // shortest path can still be the cheaper plan once its permutation -- or the lack of one -- is
+    // counted.  Call after run().
+    void near(i64 bound, int max_steps, size_t max_paths, std::vector<std::vector<WeakStep>> &paths) const
+    {
+        using Key = std::vector<uint8_t>;
+        const bool no_over = (p.flags & REDIST_NO_OVERPARTITION) != 0 && !allow_over;
+        const Key start = key_of(p.src_pax, 0);
+        struct Edge {
+            int to;
+            i64 w;
+            WeakStep ws;
+        };
+        const i64 INF = std::numeric_limits<i64>::max();
+        std::map<Key, int> id;
+        std::vector<Key> keys;
+        std::vector<std::vector<Edge>> out;
+        std::vector<i64> from_start;
+        auto node = [&](const Key &k) {
+            auto it = id.find(k);
+            if (it != id.end()) return it->second;
+            int v = int(keys.size());
+            id.emplace(k, v);
+            keys.push_back(k);
+            out.emplace_back();
+            from_start.push_back(INF);
+            return v;
+        };
+        // 1. every weak type within the bound, with its out-edges (Dijkstra order from the source type)
+        using QE = std::pair<i64, int>;
+        std::priority_queue<QE, std::vector<QE>, std::greater<QE>> pq;
+        from_start[node(start)] = 0;
+        pq.push({0, 0});
+        std::vector<char> expanded;
+        while (!pq.empty()) {
+            auto [dv, v] = pq.top();
+            pq.pop();
+            if (expanded.size() < keys.size()) expanded.resize(keys.size(), 0);
+            if (expanded[v] || dv != from_start[v]) continue;
+            expanded[v] = 1;
+            const Key key = keys[v];
+            expand(key, no_over, [&](const Key &nk, i64 w, const WeakStep &ws) {
+                if (dv + w >= bound) return;
+                int u = node(nk);
+                out[v].push_back(Edge{u, w, ws});
+                if (dv + w < from_start[u]) {
+                    from_start[u] = dv + w;
+                    pq.push({dv + w, u});
+                }
+            });
+        }
+        // 2. cheapest continuation to the target local type, whatever the phase
+        const int V = int(keys.size());
+        std::vector<std::vector<std::pair<int, i64>>> in(V);
+        for (int v = 0; v < V; ++v)
+            for (const Edge &e : out[v]) in[e.to].push_back({v, e.w});
+        std::vector<i64> to_goal(V, INF);
+        std::vector<char> is_goal(V, 0);
+        for (int v = 0; v < V; ++v)
+            if (std::equal(tgt_exps.begin(), tgt_exps.end(), keys[v].begin())) {
+                is_goal[v] = 1;
+                to_goal[v] = 0;
+                pq.push({0, v});
+            }
+        while (!pq.empty()) {
+            auto [dv, v] = pq.top();
+            pq.pop();
+            if (dv != to_goal[v]) continue;
+            for (auto [u, w] : in[v])
+                if (dv + w < to_goal[u]) {
+                    to_goal[u] = dv + w;
+                    pq.push({dv + w, u});
+                }
+        }
+        for (int v = 0; v < V; ++v)
+            std::stable_sort(out[v].begin(), out[v].end(), [&](const Edge &a, const Edge &b) {
+                i64 ca = to_goal[a.to] == INF ? INF : a.w + to_goal[a.to];
+                i64 cb = to_goal[b.to] == INF ? INF : b.w + to_goal[b.to];
+                return ca < cb;
+            });
+        // 3. depth-first enumeration under the bound (dynslices only add axes and every other step
+        //    costs at least one element, so no walk is endless); the visit budget keeps planning fast
+        struct Frame {
+            int v;
+            size_t next;
+            i64 cost;
+        };
+        std::vector<Frame> stack{Frame{0, 0, 0}};
+        std::vector<WeakStep> cur;
+        size_t visits = 0;
+        while (!stack.empty() && paths.size() < max_paths && visits < 20000) {
+            Frame &f = stack.back();
+            if (f.next == 0 && is_goal[f.v] && !cur.empty()) paths.push_back(cur);
+            if (is_goal[f.v] || f.next >= out[f.v].size() || int(stack.size()) > max_steps) {
+                stack.pop_back();
+                if (!cur.empty()) cur.pop_back();
+                continue;
+            }
+            const Edge &e = out[f.v][f.next++];
+            ++visits;
+            if (to_goal[e.to] == INF || f.cost + e.w + to_goal[e.to] >= bound) continue;
+            cur.push_back(e.ws);
+            const i64 nc = f.cost + e.w;
+            stack.push_back(Frame{e.to, 0, nc});
+        }
     }
 };
 
@@ -626,85 +745,114 @@ redist_status synthesize(Plan &p)
     }
     if (!have) return REDIST_EINTERNAL;
 
-    // 4. at most one allpermute, placed before the trailing allgathers
-    if (!same_assignment(p, end, target)) {
-        size_t g0 = steps.size();
-        while (g0 > 0 && steps[g0 - 1].kind == REDIST_STEP_ALLGATHER) --g0;
-        ConcreteState pre_gather = g0 < steps.size() ? steps[g0].pre : end;
-        if (g0 < steps.size()) pre_gather = (g0 == 0) ? p.initial : steps[g0 - 1].post;
-        // target type extended by the gathered axes (taken from axes the target leaves unused)
-        ConcreteState ext = target;
-        std::vector<char> busy(A, 0);
-        for (const auto &l : p.dst_pax)
-            for (int a : l) busy[a] = 1;
-        std::vector<std::vector<int>> blocks;
-        std::vector<std::vector<int>> extra(p.rank);
-        for (size_t t = g0; t < steps.size(); ++t) {
-            std::vector<int> blk;
-            for (int a : steps[t].acting) {
-                int pickd = -1;
-                if (!busy[a]) pickd = a;
-                for (int b = 0; b < A && pickd < 0; ++b)
-                    if (!busy[b] && p.primes[b].size == p.primes[a].size) pickd = b;
-                if (pickd < 0) return REDIST_EINTERNAL;
-                busy[pickd] = 1;
-                blk.push_back(pickd);
+    // 4. at most one allpermute, placed before the trailing allgathers; 5. costs and height
+    auto finish = [&](std::vector<Step> &steps, ConcreteState &end, i64 &cost, i64 &height) -> redist_status {
+        if (!same_assignment(p, end, target)) {
+            size_t g0 = steps.size();
+            while (g0 > 0 && steps[g0 - 1].kind == REDIST_STEP_ALLGATHER) --g0;
+            ConcreteState pre_gather = g0 < steps.size() ? steps[g0].pre : end;
+            if (g0 < steps.size()) pre_gather = (g0 == 0) ? p.initial : steps[g0 - 1].post;
+            // target type extended by the gathered axes (taken from axes the target leaves unused)
+            ConcreteState ext = target;
+            std::vector<char> busy(A, 0);
+            for (const auto &l : p.dst_pax)
+                for (int a : l) busy[a] = 1;
+            std::vector<std::vector<int>> blocks;
+            std::vector<std::vector<int>> extra(p.rank);
+            for (size_t t = g0; t < steps.size(); ++t) {
+                std::vector<int> blk;
+                for (int a : steps[t].acting) {
+                    int pickd = -1;
+                    if (!busy[a]) pickd = a;
+                    for (int b = 0; b < A && pickd < 0; ++b)
+                        if (!busy[b] && p.primes[b].size == p.primes[a].size) pickd = b;
+                    if (pickd < 0) return REDIST_EINTERNAL;
+                    busy[pickd] = 1;
+                    blk.push_back(pickd);
+                }
+                blocks.push_back(blk);
+                extra[steps[t].dim_i].insert(extra[steps[t].dim_i].end(), blk.begin(), blk.end());
             }
-            blocks.push_back(blk);
-            extra[steps[t].dim_i].insert(extra[steps[t].dim_i].end(), blk.begin(), blk.end());
+            for (int k = 0; k < p.rank; ++k) {
+                std::vector<int> nl = extra[k];
+                nl.insert(nl.end(), p.dst_pax[k].begin(), p.dst_pax[k].end());
+                ext.ax[k] = nl;
+            }
+            std::vector<Step> tail(steps.begin() + g0, steps.end());
+            steps.resize(g0);
+            if (!same_assignment(p, pre_gather, ext)) {
+                Step pm;
+                pm.kind = REDIST_STEP_ALLPERMUTE;
+                pm.pre = pre_gather;
+                pm.post = ext;
+                pm.local_before = localtype_of(p, pre_gather);
+                pm.local_after = localtype_of(p, ext);
+                if (pm.local_before != pm.local_after) return REDIST_EINTERNAL;
+                if (!make_permutation(p, pre_gather, ext, pm.source_of)) return REDIST_EINTERNAL;
+                steps.push_back(pm);
+            }
+            ConcreteState cur = ext;
+            for (size_t t = 0; t < tail.size(); ++t) {
+                Step g = tail[t];
+                g.acting = blocks[t];
+                g.pre = cur;
+                g.local_before = localtype_of(p, cur);
+                const int i = g.dim_i;
+                // the block is minor-most in ext by construction
+                for (size_t q = 0; q < g.acting.size(); ++q)
+                    if (cur.ax[i].size() <= q || cur.ax[i][q] != g.acting[q]) return REDIST_EINTERNAL;
+                cur.ax[i].erase(cur.ax[i].begin(), cur.ax[i].begin() + g.acting.size());
+                g.post = cur;
+                g.local_after = localtype_of(p, cur);
+                steps.push_back(g);
+            }
+            end = cur;
         }
-        for (int k = 0; k < p.rank; ++k) {
-            std::vector<int> nl = extra[k];
-            nl.insert(nl.end(), p.dst_pax[k].begin(), p.dst_pax[k].end());
-            ext.ax[k] = nl;
-        }
-        std::vector<Step> tail(steps.begin() + g0, steps.end());
-        steps.resize(g0);
-        if (!same_assignment(p, pre_gather, ext)) {
-            Step pm;
-            pm.kind = REDIST_STEP_ALLPERMUTE;
-            pm.pre = pre_gather;
-            pm.post = ext;
-            pm.local_before = localtype_of(p, pre_gather);
-            pm.local_after = localtype_of(p, ext);
-            if (pm.local_before != pm.local_after) return REDIST_EINTERNAL;
-            if (!make_permutation(p, pre_gather, ext, pm.source_of)) return REDIST_EINTERNAL;
-            steps.push_back(pm);
-        }
-        ConcreteState cur = ext;
-        for (size_t t = 0; t < tail.size(); ++t) {
-            Step g = tail[t];
-            g.acting = blocks[t];
-            g.pre = cur;
-            g.local_before = localtype_of(p, cur);
-            const int i = g.dim_i;
-            // the block is minor-most in ext by construction
-            for (size_t q = 0; q < g.acting.size(); ++q)
-                if (cur.ax[i].size() <= q || cur.ax[i][q] != g.acting[q]) return REDIST_EINTERNAL;
-            cur.ax[i].erase(cur.ax[i].begin(), cur.ax[i].begin() + g.acting.size());
-            g.post = cur;
-            g.local_after = localtype_of(p, cur);
-            steps.push_back(g);
-        }
-        end = cur;
-    }
 
-    // 5. costs, height, end-state check
-    p.height = p.local_src;
-    p.cost = 0;
-    for (Step &s : steps) {
-        i64 before = product(s.local_before), after = product(s.local_after);
-        s.localsize_after = after;
-        switch (s.kind) {
-        case REDIST_STEP_DYNSLICE: s.cost = 0; break;
-        case REDIST_STEP_ALLGATHER: s.cost = after; break;
-        default: s.cost = before; break;   // alltoall, allpermute
+        height = p.local_src;
+        cost = 0;
+        for (Step &s : steps) {
+            i64 before = product(s.local_before), after = product(s.local_after);
+            s.localsize_after = after;
+            switch (s.kind) {
+            case REDIST_STEP_DYNSLICE: s.cost = 0; break;
+            case REDIST_STEP_ALLGATHER: s.cost = after; break;
+            default: s.cost = before; break;   // alltoall, allpermute
+            }
+            cost += s.cost;
+            height = std::max(height, after);
         }
-        p.cost += s.cost;
-        p.height = std::max(p.height, after);
+        if (!same_assignment(p, end, target)) return REDIST_EINTERNAL;
+        if (height > std::max(p.local_src, p.local_dst)) return REDIST_EINTERNAL;
+        return REDIST_OK;
+    };
+    redist_status rc = finish(steps, end, p.cost, p.height);
+    if (rc != REDIST_OK) return rc;
+
+    // 6. optionally count the permutation: try the sequences whose own cost lies below the total
+    //    of the plan found so far, and keep the cheapest total (then the fewest steps)
+    if (p.flags & REDIST_COST_PERMUTE) {
+        std::vector<std::vector<WeakStep>> near;
+        S.near(p.cost, int(steps.size()) + 3, 256, near);
+        for (const auto &cand : near) {
+            i64 weak = 0;
+            std::vector<Step> st;
+            ConcreteState e;
+            if (!L.lower(cand, st, e)) continue;
+            for (const Step &s : st)
+                weak += s.kind == REDIST_STEP_DYNSLICE    ? 0
+                        : s.kind == REDIST_STEP_ALLGATHER ? product(s.local_after)
+                                                          : product(s.local_before);
+            if (weak >= p.cost) continue;
+            i64 cost = 0, height = 0;
+            if (finish(st, e, cost, height) != REDIST_OK) continue;
+            if (cost < p.cost || (cost == p.cost && st.size() < steps.size())) {
+                steps = st;
+                p.cost = cost;
+                p.height = height;
+            }
+        }
     }
-    if (!same_assignment(p, end, target)) return REDIST_EINTERNAL;
-    if (p.height > std::max(p.local_src, p.local_dst)) return REDIST_EINTERNAL;
     p.steps = steps;
     return REDIST_OK;
 }

@@ -84,7 +84,7 @@ def test_random_sweep_reduced_shape(mode):
         assert_same(got, want, w.name + " " + w.src.notation(w.mesh_shape) + "->" + w.dst.notation(w.mesh_shape))
 
 
-def random_problems_small_and_odd(n_problems):
+def random_problems_small_and_odd(n_problems, extra_flags=0):
     """Odd primes, all element sizes, element-sized runs, several steps with scratch ping-pong.
     Returns the set of kernel variants that ran."""
     rng = np.random.default_rng(2112)
@@ -117,7 +117,7 @@ def random_problems_small_and_odd(n_problems):
         src, dst = (gshape, a1), (gshape, a2)
         src_tiles = oracle.reslice(mesh, src, G)
         want = oracle.redistribute(mesh, src, dst, src_tiles)
-        mode = MODES[t % 4]
+        mode = MODES[t % 4] | extra_flags
         plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
         n_multi += plan.num_launches >= 3
         variants.update(plan.launch_info(q).variant for q in range(plan.num_launches))
@@ -129,6 +129,12 @@ def random_problems_small_and_odd(n_problems):
 def test_random_problems_small_and_odd():
     variants = random_problems_small_and_odd(600)
     assert variants >= {0, 3, 4, 5, 6, 7}   # rows, units, bulk, gather, ragged bulk and zip kernels all ran
+
+
+def test_random_problems_with_the_permutation_counted():
+    """Plans chosen with the final permutation in the cost (other sequences than the default ones,
+    e.g. an extra leading dynslice) in every execution mode."""
+    random_problems_small_and_odd(300, api.COST_PERMUTE)
 
 
 def _random_problems_in_a_fresh_process(env, n_problems, expect):

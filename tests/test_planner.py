@@ -327,6 +327,48 @@ def test_near_optimality_against_brute_force(mesh):
         p.close()
 
 
+def test_counting_the_permutation_example():
+    """Mesh {a:2, b:2, c:3}, [2{c,a}12] -> [4{c}12].  The shortest weak path is a single allgather; lowered, it
+    needs a permutation in front and costs 6 in total.  Slicing over the idle axis b first halves the
+    tiles the permutation moves: 5 in total, the optimum over all sequences of the four typing rules.  Both plans are checked step by step against the rules and the oracle."""
+    mesh, src, dst = (2, 2, 3), ((12,), ((2, 0),)), ((12,), ((2,),))
+    d0 = check_plan(mesh, src, dst, 4)
+    d1 = check_plan(mesh, src, dst, 4, api.COST_PERMUTE)
+    assert (d0["cost"], d1["cost"]) == (6, 5)
+    assert brute_force_optimum(mesh, src[0], src[1], dst[1]) == 5
+    assert [s["kind"] for s in d1["steps"]] == ["dynslice", "allpermute", "allgather"]
+
+
+@pytest.mark.parametrize("mesh", [(2, 2), (2, 3), (4, 6), (2, 4, 2), (6, 2), (2, 2, 3), (2, 2, 2, 2)])
+def test_counting_the_permutation_never_costs_more(mesh):
+    """REDIST_COST_PERMUTE: every plan is still a typed normal-form sequence inside the memory bound
+    that ends in the oracle's tiles (check_plan), and its total cost is at most the default plan's."""
+    rng = np.random.default_rng(sum(mesh) * 17 + len(mesh))
+    for t in range(16):
+        src, dst = random_problem(rng, mesh)
+        e = int(rng.choice([1, 2, 4, 8, 16]))
+        p0 = api.Plan(mesh, src, dst, e)
+        d1 = check_plan(mesh, src, dst, e, api.COST_PERMUTE | MODES[t % 4], seed=t)
+        assert d1["cost"] <= p0.cost
+        p0.close()
+
+
+def test_counting_the_permutation_on_evaluation_shaped_problems():
+    """On problems of the evaluation's shape some plans get cheaper (a permutation avoided or moved to
+    smaller tiles), none gets dearer, and the memory bound still holds."""
+    better = 0
+    for w in wl.evaluation_like_problems(200):
+        p0 = api.Plan(w.mesh_shape, w.src, w.dst, 4)
+        p1 = api.Plan(w.mesh_shape, w.src, w.dst, 4, api.COST_PERMUTE)
+        assert p1.cost <= p0.cost
+        assert p1.height <= max(p1.local_elems(0), p1.local_elems(1))
+        assert p1.step_kinds().count("allpermute") <= 1
+        better += p1.cost < p0.cost
+        p0.close()
+        p1.close()
+    assert better > 0
+
+
 def test_planner_throughput_on_evaluation_shaped_problems():
     """Section 8 reports synthesis in under a second per problem (unoptimised Python); the host planner
     here must stay far below that on 300 problems of the same shape (3 mesh axes, up to 6-D)."""
