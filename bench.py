@@ -1,21 +1,29 @@
 #!/usr/bin/env python
 """Benchmark: effective HBM GB/s of executing a synthesized redistribution on one B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl ours|reference]
 
-A *step* is one pass of the workload: for ``c2`` (the default: bf16 [8,2048,4096], mesh 4x2, 8 virtual
-devices) the forward redistribution {d0:x, d2:y} -> {d1:(x,y)} followed by the reverse, i.e. two
-plans and two fused kernel launches.  Metric: effective bytes (every global element read once plus
-every destination byte written once) per second, in GB/s.  Inputs are synthetic, seeded and
-resident in HBM before the timed region; four buffer sets rotate so that no buffer is re-read
-within 1 GiB of traffic (L2 is 126 MB).  The timed region calls ``redist_execute`` once per
-redistribution on one stream (kernels use programmatic dependent launch, so consecutive launches
-overlap their ramp-up with the previous kernel's tail); ``--graph`` times CUDA-graph replays instead.  ``e2e`` is the same step through ``redist_execute_host``
-with pinned host tiles, host<->device copies inside the timed region.
+A *step* is one pass of the workload.  The default is ``c5`` -- the largest configuration: bf16
+[32768, 32768] (2 GiB) on a 4x4x4 mesh of 64 virtual devices -- and a step runs its two
+redistributions, {d0:(x,y), d1:z} -> {d0:(y,x), d1:z} (an allpermute) and {d0:(x,y), d1:z} ->
+{d0:z, d1:(y,x)} (alltoall + allpermute fused into one kernel): two launches of 2 GiB read + 2 GiB
+written each.  Metric: effective bytes (every global element read once plus every destination byte
+written once) per second, in GB/s.  Inputs are synthetic, seeded and resident in HBM before the
+timed region; buffer sets rotate, and every launch moves far more than the 126 MB L2 holds.  The
+timed region calls ``redist_execute`` once per redistribution on one stream (kernels use
+programmatic dependent launch, so consecutive launches overlap their ramp-up with the previous
+kernel's tail); ``--graph`` times CUDA-graph replays instead.  ``e2e`` is the same step through
+``redist_execute_host`` with pinned host tiles, host<->device copies inside the timed region.
 
-With ``--gpus N`` (launched by torchrun, one rank per GPU) every rank runs an independent replica:
-the method has no inter-GPU step here (virtual devices share one GPU), so there is no collective on
-the data path; only the timing is reduced (max over ranks).
+The same JSON line carries a ``configs`` block: every benchmark configuration (c1, c2, c3a, c3b, c3c,
+c5a, c5b and a fixed subset of the c4 sweep) timed in its own event-bracketed region, with GB/s,
+microseconds per launch (back to back and for one launch alone), fraction of the measured copy
+bandwidth, launches and scratch per virtual device.
+
+With ``--gpus N`` every rank runs an independent replica: the method has no inter-GPU step here
+(virtual devices share one GPU), so there is no collective on the data path; only the timing is
+reduced (max over ranks).  Started without a launcher (``WORLD_SIZE`` unset) the script re-executes
+itself under ``torch.distributed.run`` with N ranks on 127.0.0.1.
 
 ``--impl reference`` times the CPU oracle (``oracle/``) on the host cores for the same metric.
 """
@@ -148,15 +156,23 @@ def ncu_traffic(workload: str):
 
 # ---------------------------------------------------------------------------------------- ours
 
-class DeviceLeg:
-    """One redistribution with N_SETS rotating sets of device tiles."""
+def sets_for(eff_bytes: int) -> int:
+    """Buffer sets that rotate: a launch that moves at least 1 GB streams far more than the L2 holds
+    and two sets suffice; smaller workloads get four."""
+    return 2 if eff_bytes >= (1 << 30) else N_SETS
 
-    def __init__(self, w, flags, torch, api, gen, sets=N_SETS, alias_replicas=True):
+
+class DeviceLeg:
+    """One redistribution with rotating sets of device tiles."""
+
+    def __init__(self, w, flags, torch, api, gen, sets=None, alias_replicas=True):
         self.w = w
         self.plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, flags)
         p = self.plan
         self.n = p.n_devices
-        sb, db = p.local_elems(0) * w.elem_bytes, p.local_elems(1) * w.elem_bytes
+        self.eff_bytes = effective_bytes(w)
+        sets = sets or sets_for(self.eff_bytes)
+        db = p.local_elems(1) * w.elem_bytes
         G = torch.randint(0, 256, tuple(w.src.global_shape) + (w.elem_bytes,), dtype=torch.uint8, device="cuda",
                           generator=gen)
         self.src, self.dst = [], []
@@ -170,11 +186,11 @@ class DeviceLeg:
                 key = o if alias_replicas else d
                 if key not in owned:
                     owned[key] = tiles[d].clone()
+            del tiles
             self.src.append([owned[o if alias_replicas else d] for d, o in enumerate(offs)])
             self.dst.append([torch.empty(db, dtype=torch.uint8, device="cuda") for _ in range(self.n)])
         del G
         self.scratch = p.alloc_scratch()
-        self.eff_bytes = effective_bytes(w)
         self.launches = p.num_launches
         sp = self.scratch.data_ptr() if self.scratch is not None else 0
         sn = self.scratch.numel() if self.scratch is not None else 0
@@ -236,6 +252,47 @@ def time_legs(torch, legs, steps, warmup, per_launch=False, graphs=None):
     return t0.elapsed_time(t1), [[a.elapsed_time(b) for a, b in ev[k]] for k in range(len(legs))]
 
 
+def kernel_name(api, li) -> str:
+    kname = {"naive_gather": "allgather", "naive_slice": "dynslice", "copy": "allpermute"}.get(
+        api.KERNELS[li.kernel], api.KERNELS[li.kernel])
+    return f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk', 7: '_zip'}.get(li.variant, '') }_kernel"
+
+
+def spawn_ranks(n: int):
+    """Started without a launcher: run this script again under torch.distributed.run, one rank per GPU."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    os.execv(sys.executable, cmd)
+
+
+def run_standin(args):
+    """The launch plumbing of an N-rank run with a CPU stand-in for the timed body (gloo, no CUDA):
+    used by the tests of the multi-process path.  Every rank 'processes' a fixed number of bytes in a
+    rank-dependent time; the line is built by the same reduce / aggregate code as the real run."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    mine_ms = 10.0 + 5.0 * rank
+    worst = reduce_max(dist if world > 1 else None, mine_ms, device="cpu")
+    step_bytes = 512 << 20
+    line = {"metric": METRIC, "value": round(aggregate_value(world, step_bytes, worst / args.steps), 3),
+            "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": worst / args.steps, "higher_is_better": True, "scaling": "weak",
+            "config": {"workload": "stand-in"}, "standin": True}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     from paper_2112_01075_b200 import api
@@ -257,7 +314,8 @@ def run_ours(args):
     flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
     if args.cost_permute:
         flags |= api.COST_PERMUTE
-    legs = [DeviceLeg(w, flags, torch, api, gen) for w in ws]
+    legs = [DeviceLeg(w, flags, torch, api, gen, sets=args.sets or None) for w in ws]
+    n_sets = len(legs[0].calls)
     step_bytes = sum(l.eff_bytes for l in legs)
 
     def barrier():
@@ -278,8 +336,8 @@ def run_ours(args):
         t_end = time.perf_counter() + 0.35
         extra = 0
         while time.perf_counter() < t_end:
-            time_legs(torch, legs, 50, 0, graphs=graphs)
-            extra += 50
+            time_legs(torch, legs, 20, 0, graphs=graphs)
+            extra += 20
         window = f"warm-up, timed region and {extra} further untimed steps of the same workload"
     clocks = sampler.stop()
     clocks["window"] = window
@@ -292,16 +350,20 @@ def run_ours(args):
     # used plain launches, and vice versa), and once more with an event pair around every launch
     # (per-leg numbers; the events themselves cost a few microseconds and break launch overlap)
     n_side = max(3, min(args.steps, 200))
-    other_graphs = None if args.graph else capture_graphs(torch, legs)
-    other_ms, _ = time_legs(torch, legs, n_side, 3, graphs=other_graphs)
+    other_ms = None
+    if not args.lean:
+        other_graphs = None if args.graph else capture_graphs(torch, legs)
+        other_ms, _ = time_legs(torch, legs, n_side, 3, graphs=other_graphs)
+        del other_graphs
     _, per = time_legs(torch, legs, n_side, 3, per_launch=True)
 
-    # roofline of the dominant kernel.  When every launch of the step runs the same kernel on the
-    # same number of bytes (the default workload), its average duration is the timed region divided
-    # by the number of launches; otherwise the per-launch event pairs decide.
+    # Roofline of the dominant kernel (the leg that takes longest).  When every launch of the step runs the
+    # same kernel on the same number of bytes, its average duration is the timed region divided by the
+    # number of launches; otherwise the event pair around each of its launches decides.
     infos = [l.plan.launch_info(0) for l in legs]
     n_launch = sum(l.launches for l in legs)
-    same = all(l.launches == 1 for l in legs) and len({(i.kernel, i.bytes_read + i.bytes_written) for i in infos}) == 1
+    same = all(l.launches == 1 for l in legs) and \
+        len({(kernel_name(api, i), i.bytes_read + i.bytes_written) for i in infos}) == 1
     sums = [sum(p) for p in per]
     k = max(range(len(legs)), key=lambda q: sums[q])
     dom, li = legs[k], infos[k]
@@ -309,66 +371,124 @@ def run_ours(args):
     avg_ms = (total_ms / (args.steps * n_launch)) if same else statistics.mean(per[k]) / dom.launches
     peak, how = measured_peak()
     achieved = alg / (avg_ms * 1e-3) / 1e9
-    kname = {"naive_gather": "allgather", "naive_slice": "dynslice", "copy": "allpermute"}.get(
-        api.KERNELS[li.kernel], api.KERNELS[li.kernel])
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "traffic": ncu_traffic(args.workload),
-                "kernel": f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk', 7: '_zip'}.get(li.variant, '') }_kernel",
+                "frac": round(achieved / peak, 4), "traffic": ncu_traffic(dom.w.name),
+                "kernel": kernel_name(api, li), "workload_leg": dom.w.name,
                 "algorithmic_bytes_per_launch": alg,
                 "avg_launch_us": round(avg_ms * 1e3, 2),
-                "avg_from": "timed region / launches" if same else "event pair around each launch",
+                "avg_from": "timed region / launches" if same else
+                            f"event pair around each of its {len(per[k])} launches (a region of the same steps right after the headline region)",
+                "timed_region_us_per_launch_all_kernels": round(total_ms / (args.steps * n_launch) * 1e3, 2),
                 "peak_source": how + " copy bandwidth", "frac_of_8TBs_nominal": round(achieved / 8000.0, 4)}
 
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": describe_workload(args.workload, ws), "fuse": args.fuse,
-                   "launch": "CUDA graph replay of captured redist_execute calls (one graph per buffer set)"
-                   if args.graph else "redist_execute called once per redistribution on the stream",
-                   "cache": f"{N_SETS} rotating buffer sets, no buffer re-read within 1 GiB of traffic",
-                   "parallelism": "replicas only" if world > 1 else "single GPU, virtual devices"},
+        "config": {"workload": describe_workload(args.workload, ws)},
+        "run": {"fuse": args.fuse,
+                "launch": "CUDA graph replay of captured redist_execute calls (one graph per buffer set)"
+                if args.graph else "redist_execute called once per redistribution on the stream",
+                "cache": f"{n_sets} rotating buffer sets; one launch moves {legs[0].eff_bytes >> 20} MiB "
+                         f"(L2: 126 MB)",
+                "parallelism": "replicas only" if world > 1 else "single GPU, virtual devices",
+                "timed_region_ms": round(total_ms, 3)},
         "gpu_launches": args.steps * sum(l.launches for l in legs),
         "clocks": clocks, "roofline": roofline,
         "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in legs),
         "memory_bound_bytes_per_virtual_device": max(max(l.plan.local_elems(0), l.plan.local_elems(1)) *
                                                      l.w.elem_bytes for l in legs),
-        ("stream_launch" if args.graph else "graph_replay"): {
-            "value": round(world * step_bytes / (other_ms / n_side * 1e-3) / 1e9, 1), "unit": UNIT,
-            "ms_per_step": round(other_ms / n_side, 5), "steps": n_side,
-            "note": "same steps, " + ("plain redist_execute calls" if args.graph else
-                                      "replayed from CUDA graphs of captured redist_execute calls, one step per "
-                                      "graph (no dependent-launch overlap from one graph launch to the next)")},
         "legs": [{"name": l.w.name, "steps": l.plan.step_kinds(), "kernels": l.plan.launch_kernels(),
                   "gbs": round(l.eff_bytes / (statistics.mean(per[q]) * 1e-3) / 1e9, 1),
                   "us": round(statistics.mean(per[q]) * 1e3, 2)} for q, l in enumerate(legs)],
     }
+    if other_ms is not None:
+        line["stream_launch" if args.graph else "graph_replay"] = {
+            "value": round(world * step_bytes / (other_ms / n_side * 1e-3) / 1e9, 1), "unit": UNIT,
+            "ms_per_step": round(other_ms / n_side, 5), "steps": n_side,
+            "note": "same steps, " + ("plain redist_execute calls" if args.graph else
+                                      "replayed from CUDA graphs of captured redist_execute calls, one step per "
+                                      "graph (no dependent-launch overlap from one graph launch to the next)")}
+    del legs, graphs
+    torch.cuda.empty_cache()
+    e2e_steps = max(3, min(args.steps, 10))
     if rank == 0 and not args.no_e2e:
-        line["e2e"] = run_e2e(torch, api, ws, flags, max(3, min(args.steps, 10)), world, dist)
+        line["e2e"] = run_e2e(torch, api, ws, flags, e2e_steps, world, dist)
     elif dist is not None and not args.no_e2e:
-        run_e2e(torch, api, ws, flags, max(3, min(args.steps, 10)), world, dist)
+        run_e2e(torch, api, ws, flags, e2e_steps, world, dist)
+    torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(ws)
-    if rank == 0 and world == 1 and args.fuse == "adjacent":
+    if rank == 0 and world == 1 and args.fuse == "adjacent" and not args.lean:
         # comparison points on the same workload (short runs, outside the headline region): the
         # sequence run collective by collective through scratch, and the naive gather-then-slice method
-        del legs
-        torch.cuda.empty_cache()
         for key, fl in (("unfused", api.FUSE_NONE), ("naive_gpu_baseline", api.NAIVE)):
-            cmp_legs = [DeviceLeg(w, fl, torch, api, gen) for w in ws]
-            ms, _ = time_legs(torch, cmp_legs, 50, 3)
-            line[key] = {"value": round(step_bytes / (ms / 50 * 1e-3) / 1e9, 1), "unit": UNIT,
+            cmp_legs = [DeviceLeg(w, fl, torch, api, gen, sets=args.sets or None) for w in ws]
+            reps = 20
+            ms, _ = time_legs(torch, cmp_legs, reps, 3)
+            line[key] = {"value": round(step_bytes / (ms / reps * 1e-3) / 1e9, 1), "unit": UNIT,
                          "launches_per_step": sum(l.launches for l in cmp_legs),
                          "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in cmp_legs)}
             del cmp_legs
             torch.cuda.empty_cache()
-    if rank == 0 and world == 1 and args.others:
-        line["others"] = run_others(torch, api, gen, args)
+    if rank == 0 and world == 1 and args.fuse == "adjacent" and not args.lean and not args.no_configs:
+        line["configs"] = run_configs(torch, api, gen)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+CONFIG_ENTRIES = [("c1", ["c1", "c1_back"]), ("c2", ["c2", "c2_back"]), ("c3a", ["c3a"]), ("c3b", ["c3b"]),
+                  ("c3c", ["c3c"]), ("c5a", ["c5a"]), ("c5b", ["c5b"])]
+C4_SUBSET = list(range(0, 100, 8))      # the fixed subset of the 100 seeded pairs: every eighth
+
+
+def run_configs(torch, api, gen, reps: int = 30):
+    """Every benchmark configuration in its own event-bracketed region of `reps` steps (default mode):
+    back-to-back launches on one stream (`gbs`, `us_per_launch`) and one launch alone between two
+    events (`isolated_us`), with the fraction of the measured copy bandwidth, the number of kernel
+    launches per step and the scratch per virtual device.  c1 moves 512 KiB per step and stays in L2:
+    it measures launch latency.  c4 is a fixed subset of the sweep (every eighth pair)."""
+    from paper_2112_01075_b200 import workloads as wl
+    peak, _ = measured_peak()
+    b = wl.bench_workloads()
+    out = {}
+    for name, parts in CONFIG_ENTRIES:
+        legs = [DeviceLeg(b[p], api.FUSE_ADJACENT, torch, api, gen) for p in parts]
+        eff = sum(l.eff_bytes for l in legs)
+        n_launch = sum(l.launches for l in legs)
+        r = max(reps, 20)
+        ms, _ = time_legs(torch, legs, r, 5)
+        _, per = time_legs(torch, legs, r, 3, per_launch=True)
+        iso = statistics.median([sum(per[q][i] for q in range(len(legs))) for i in range(r)]) / n_launch
+        gbs = eff / (ms / r * 1e-3) / 1e9
+        out[name] = {"gbs": round(gbs, 1), "us_per_launch": round(ms / r / n_launch * 1e3, 2),
+                     "frac": round(gbs / peak, 4), "frac_of_8TBs_nominal": round(gbs / 8000.0, 4),
+                     "isolated_us": round(iso * 1e3, 2),
+                     "isolated_gbs": round(eff / n_launch / (iso * 1e-3) / 1e9, 1),
+                     "launches_per_step": n_launch, "bytes_per_launch": eff // n_launch, "reps": r,
+                     "steps": [l.plan.step_kinds() for l in legs],
+                     "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in legs),
+                     "memory_bound_bytes_per_virtual_device": max(
+                         max(l.plan.local_elems(0), l.plan.local_elems(1)) * l.w.elem_bytes for l in legs)}
+        del legs
+        torch.cuda.empty_cache()
+    rows = sweep_rows(torch, api, [wl.config4()[i] for i in C4_SUBSET], api.FUSE_ADJACENT, wl.CONFIG4_FILL_SEED)
+    g = [r["gbs"] for r in rows]
+    out["c4"] = {"pairs": [r["name"] for r in rows], "geomean_gbs": round(geomean(g), 1), "min_gbs": min(g),
+                 "max_gbs": max(g), "frac_geomean": round(geomean(g) / peak, 4), "frac_min": round(min(g) / peak, 4),
+                 "launches_max": max(r["launches"] for r in rows),
+                 "scratch_bytes_per_virtual_device_max": max(r["scratch_per_device"] for r in rows),
+                 "note": "every eighth of the 100 seeded pairs, each planned, executed and timed on its own "
+                         "(global array 4 GiB; 5 timed repetitions per pair after 2 warm-up launches)"}
+    return out
+
+
+def geomean(v):
+    import math
+    return math.exp(sum(math.log(x) for x in v) / len(v))
 
 
 def describe_workload(name, ws):
@@ -438,8 +558,7 @@ def run_others(torch, api, gen, args):
             if fuse != "adjacent" and name in ("c1",):
                 continue
             try:
-                sets = 2 if name.startswith(("c3c", "c5")) else N_SETS
-                legs = [DeviceLeg(w, flags, torch, api, gen, sets=sets) for w in ws]
+                legs = [DeviceLeg(w, flags, torch, api, gen) for w in ws]
                 total, per = time_legs(torch, legs, 10, 3, per_launch=True)
                 eff = sum(l.eff_bytes for l in legs)
                 med = statistics.median([sum(per[q][i] for q in range(len(legs))) for i in range(10)])
@@ -460,33 +579,15 @@ def run_others(torch, api, gen, args):
     return out
 
 
-def run_sweep(args):
-    """Config 4: the 100 seeded random (source, target) pairs on f32 [64,128,256,512], mesh 2x4x2.
-    Every pair is planned, executed and timed on its own (global array 4 GiB, far above L2, so no
-    buffer rotation is needed); replicated source tiles share one buffer per distinct tile."""
-    import math
-    import torch
-    from paper_2112_01075_b200 import api, workloads as wl
-
-    torch.cuda.set_device(0)
+def sweep_rows(torch, api, pairs, flags, fill_seed):
+    """Plan, execute and time every problem of `pairs` on its own.  Global arrays are far larger than
+    the L2, so no buffer rotation is needed; replicated source tiles share one buffer per distinct tile."""
     gen = torch.Generator(device="cuda")
-    gen.manual_seed(wl.CONFIG4_FILL_SEED)
-    if args.workload == "c4":
-        pairs, label = wl.config4(), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
-    elif args.workload == "adv":
-        pairs, label = wl.adversarial_problems(), "adv: the %d problems of the paper's table of largest slow-downs"
-    else:
-        pairs, label = wl.evaluation_like_problems(args.pairs), \
-            "eval: %d random problems shaped like the paper's evaluation sample (3 mesh axes, <= 6-D, 64-800 MB)"
-    flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
-    if args.cost_permute:
-        flags |= api.COST_PERMUTE
+    gen.manual_seed(fill_seed)
     G = None
     stream = torch.cuda.current_stream()
     rows = []
-    if args.only:
-        pairs = [w for w in pairs if w.name in args.only.split(",")]
-    for w in pairs[: args.pairs]:
+    for w in pairs:
         if G is None or tuple(G.shape[:-1]) != tuple(w.src.global_shape):
             G = None
             G = torch.randint(0, 256, tuple(w.src.global_shape) + (4,), dtype=torch.uint8, device="cuda",
@@ -521,16 +622,40 @@ def run_sweep(args):
         rows.append({"name": w.name, "src": w.src.notation(w.mesh_shape, w.axis_names),
                      "dst": w.dst.notation(w.mesh_shape, w.axis_names), "steps": plan.step_kinds(),
                      "launches": plan.num_launches, "run_bytes": min(i.run_bytes for i in li),
+                     "variants": [i.variant for i in li],
                      "fanout": max(i.fanout for i in li), "eff_bytes": eff, "us": round(ms * 1e3, 1),
                      "gbs": round(eff / (ms * 1e-3) / 1e9, 1),
                      "scratch_per_device": plan.scratch_bytes_per_device, "plan_cost_elems": plan.cost})
         del src, dst, owned, scratch, call, plan
         torch.cuda.empty_cache()
+    return rows
+
+
+def run_sweep(args):
+    """Config 4: the 100 seeded random (source, target) pairs on f32 [64,128,256,512], mesh 2x4x2 -- or the
+    paper's P1-P4 (`adv`), or random problems shaped like the paper's evaluation sample (`eval`)."""
+    import torch
+    from paper_2112_01075_b200 import api, workloads as wl
+
+    torch.cuda.set_device(0)
+    if args.workload == "c4":
+        pairs, label = wl.config4(), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
+    elif args.workload == "adv":
+        pairs, label = wl.adversarial_problems(), "adv: the %d problems of the paper's table of largest slow-downs"
+    else:
+        pairs, label = wl.evaluation_like_problems(args.pairs), \
+            "eval: %d random problems shaped like the paper's evaluation sample (3 mesh axes, <= 6-D, 64-800 MB)"
+    flags = {"adjacent": api.FUSE_ADJACENT, "none": api.FUSE_NONE, "all": api.FUSE_ALL, "naive": api.NAIVE}[args.fuse]
+    if args.cost_permute:
+        flags |= api.COST_PERMUTE
+    if args.only:
+        pairs = [w for w in pairs if w.name in args.only.split(",")]
+    rows = sweep_rows(torch, api, pairs[: args.pairs], flags, wl.CONFIG4_FILL_SEED)
     g = [r["gbs"] for r in rows]
     peak, how = measured_peak()
     line = {"metric": METRIC, "workload": label % len(rows),
             "fuse": args.fuse, "cost_permute": bool(args.cost_permute),
-            "plan_cost_elems_total": sum(r["plan_cost_elems"] for r in rows), "geomean_gbs": round(math.exp(sum(math.log(x) for x in g) / len(g)), 1),
+            "plan_cost_elems_total": sum(r["plan_cost_elems"] for r in rows), "geomean_gbs": round(geomean(g), 1),
             "min_gbs": min(g), "max_gbs": max(g), "median_gbs": statistics.median(g),
             "total_gbs": round(sum(r["eff_bytes"] for r in rows) / sum(r["us"] * 1e-6 for r in rows) / 1e9, 1),
             "peak": peak, "peak_source": how, "pairs_below_70pct_of_peak": sum(x < 0.7 * peak for x in g)}
@@ -623,7 +748,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-            "config": {"workload": describe_workload(args.workload, ws), "fuse": "n/a (CPU oracle)"},
+            "config": {"workload": describe_workload(args.workload, ws)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -632,10 +757,10 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2",
+    ap.add_argument("--workload", default="c5",
                     choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval"])
     ap.add_argument("--pairs", type=int, default=100, help="sweeps: how many problems to run")
     ap.add_argument("--only", default="", help="sweeps: comma-separated problem names to run")
@@ -643,14 +768,25 @@ def main():
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
     ap.add_argument("--cost-permute", action="store_true",
                     help="plan with REDIST_COST_PERMUTE (the final permutation counted when choosing the sequence)")
-    ap.add_argument("--others", action="store_true", help="also measure the other configurations briefly")
+    ap.add_argument("--others", action="store_true", help="also measure every configuration unfused and naive")
     ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays instead of plain stream launches")
     ap.add_argument("--no-graph", action="store_true", help=argparse.SUPPRESS)   # accepted, the default
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="leave out the per-configuration block")
+    ap.add_argument("--lean", action="store_true",
+                    help="headline region and per-launch events only (no graph replay, comparison modes or "
+                         "per-configuration block): the small command for profiler captures")
+    ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0: chosen from the workload size)")
+    ap.add_argument("--standin", action="store_true",
+                    help="CPU stand-in for the timed body (gloo, no CUDA): tests the N-rank launch plumbing")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
-    if args.workload in ("c4", "adv", "eval"):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.workload not in ("c4", "adv", "eval"):
+        spawn_ranks(args.gpus)      # does not return
+    if args.standin:
+        run_standin(args)
+    elif args.workload in ("c4", "adv", "eval"):
         if args.impl == "reference":
             raise SystemExit("the sweeps (c4, adv, eval) are GPU-side measurements; use another workload for --impl reference")
         run_sweep(args)

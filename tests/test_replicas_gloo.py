@@ -44,3 +44,21 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.reduce_max(None, 3.5) == 3.5
     assert abs(bench.aggregate_value(1, 10**9, 1.0) - 1000.0) < 1e-9
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` without WORLD_SIZE re-executes itself under torch.distributed.run; with
+    the CPU stand-in for the timed body the printed line must come from two ranks: n_gpus 2, the slower
+    rank's time, both ranks' bytes."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--standin", "--steps", "5"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                      # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["steps"] == 5
+    assert abs(line["ms_per_step"] - 15.0 / 5) < 1e-9          # max over ranks (10 ms and 15 ms)
+    assert abs(line["value"] - 2 * (512 << 20) / (3.0e-3) / 1e9) < 1e-2
