@@ -386,7 +386,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": describe_workload(args.workload, ws)},
-        "run": {"fuse": args.fuse,
+        "run": {"fuse": args.fuse, "tune": args.tune,
                 "launch": "CUDA graph replay of captured redist_execute calls (one graph per buffer set)"
                 if args.graph else "redist_execute called once per redistribution on the stream",
                 "cache": f"{n_sets} rotating buffer sets; one launch moves {legs[0].eff_bytes >> 20} MiB "
@@ -473,6 +473,18 @@ def run_configs(torch, api, gen, reps: int = 30):
                      "scratch_bytes_per_virtual_device": max(l.plan.scratch_bytes_per_device for l in legs),
                      "memory_bound_bytes_per_virtual_device": max(
                          max(l.plan.local_elems(0), l.plan.local_elems(1)) * l.w.elem_bytes for l in legs)}
+        if name in ("c1", "c2"):
+            # host time of one bound call (redist_bound_execute through ctypes): launches queued without waiting
+            sp = torch.cuda.current_stream().cuda_stream
+            torch.cuda.synchronize()
+            calls = 500
+            t0 = time.perf_counter()
+            for i in range(calls):
+                for l in legs:
+                    l.run(i, sp)
+            host = (time.perf_counter() - t0) / (calls * len(legs))
+            torch.cuda.synchronize()
+            out[name]["host_us_per_bound_call"] = round(host * 1e6, 2)
         del legs
         torch.cuda.empty_cache()
     rows = sweep_rows(torch, api, [wl.config4()[i] for i in C4_SUBSET], api.FUSE_ADJACENT, wl.CONFIG4_FILL_SEED)
@@ -778,12 +790,18 @@ def main():
                     help="headline region and per-launch events only (no graph replay, comparison modes or "
                          "per-configuration block): the small command for profiler captures")
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0: chosen from the workload size)")
+    ap.add_argument("--tune", default="", help="tuning values for the plans, e.g. pdl=0,item_kb=16 (redist_tuning_set)")
     ap.add_argument("--standin", action="store_true",
                     help="CPU stand-in for the timed body (gloo, no CUDA): tests the N-rank launch plumbing")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.workload not in ("c4", "adv", "eval"):
         spawn_ranks(args.gpus)      # does not return
+    if args.tune and args.impl == "ours" and not args.standin:
+        from paper_2112_01075_b200 import api
+        for kv in args.tune.split(","):
+            k, v = kv.split("=")
+            api.tuning_set(k.strip(), int(v))
     if args.standin:
         run_standin(args)
     elif args.workload in ("c4", "adv", "eval"):

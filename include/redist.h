@@ -11,7 +11,7 @@
  *
  * Conventions
  *   - A distributed type lists, per array dimension, the mesh axes that partition it, ordered
- *     minor-to-major: the first listed axis varies fastest (Section 2.2, "Distributed array
+ *     minor-to-major: the first listed axis varies fastest (Section 2.1, "Distributed array
  *     types").  Tile size = global size / product of the listed axis sizes; it must divide
  *     (rule wf-dim).  Axes a type does not list replicate the data.
  *   - Virtual device id = row-major index of the device's mesh coordinates over mesh_shape
@@ -60,8 +60,8 @@ typedef struct redist_type {
 
 typedef struct redist_plan_s redist_plan_t;   /* opaque, host memory, immutable once created */
 
-/* plan flags: exactly one execution mode, optionally or-ed with REDIST_NO_OVERPARTITION and/or
-   REDIST_COST_PERMUTE */
+/* plan flags: exactly one execution mode, optionally or-ed with REDIST_NO_OVERPARTITION,
+   REDIST_COST_PERMUTE and/or REDIST_NO_CACHE */
 enum {
     REDIST_FUSE_ADJACENT = 0,    /* default: adjacent steps of the sequence run as one kernel wherever
                                     the fused copy keeps contiguous runs of at least 64 bytes         */
@@ -73,14 +73,15 @@ enum {
     REDIST_MODE_MASK = 3,
     REDIST_NO_OVERPARTITION = 16,/* forbid dynslice steps that partition the array over more mesh
                                     axes than the target type uses (over-partitioning, Section 7.2)  */
-    REDIST_COST_PERMUTE = 32     /* count the final allpermute when choosing the sequence.  The search
+    REDIST_COST_PERMUTE = 32,    /* count the final allpermute when choosing the sequence.  The search
                                     of Section 7.3 weighs only dynslice / alltoall / allgather (the
-                                    permutation "is not a graph edge") and appends the permutation
-                                    afterwards; with this flag the sequences whose own cost lies below
-                                    that plan's total are lowered too and the cheapest total (sequence
-                                    plus permutation, cost model of Section 6.2) is kept.  The result
-                                    never costs more than the default plan and obeys the same memory
-                                    bound; planning takes longer.                                     */
+                                    permutation carries no edge weight there) and appends the
+                                    permutation afterwards; with this flag the sequences whose own cost
+                                    lies below that plan's total are lowered too and the cheapest total
+                                    (sequence plus permutation, cost model of Section 6.2) is kept.  The
+                                    result never costs more than the default plan and obeys the same
+                                    memory bound; planning takes longer.                              */
+    REDIST_NO_CACHE = 64         /* synthesize afresh instead of consulting the plan cache             */
 };
 
 enum { REDIST_MAX_RANK = 8, REDIST_MAX_MESH_AXES = 16, REDIST_MAX_DEVICES = 1024 };
@@ -137,12 +138,47 @@ typedef struct redist_launch_info {
  *   flags                                  see above
  *   out                                    host; receives the plan, owned by the caller until
  *                                          redist_plan_destroy
+ * Plans are cached (the evaluation of Section 8 asks how long synthesis takes; a runtime asks for the
+ * same few redistributions over and over): a second request for the same mesh, types, element size,
+ * flags and tuning values returns a handle to the same immutable plan without searching again.  The
+ * cache keeps the 256 most recently created plans; every handle must still be destroyed.
  * Errors: EINVAL, EILLFORMED, ENOTDIV, EGLOBAL, EUNSUPPORTED, ENOMEM, EINTERNAL.
  */
 redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *src,
                           const redist_type *dst, int32_t elem_bytes, uint32_t flags, redist_plan_t **out);
 
 void redist_plan_destroy(redist_plan_t *plan);
+
+/* Plan cache counters since the library was loaded or the cache was last cleared (any may be NULL). */
+void redist_plan_cache_stats(int64_t *hits, int64_t *misses, int64_t *entries);
+void redist_plan_cache_clear(void);
+
+/*
+ * Tuning values -- process-wide, copied into every plan created afterwards (existing plans keep theirs).
+ * Defaults are the measured optima.  Names and ranges:
+ *   "bulk"               0/1    1: aligned runs of 512 bytes and more move by TMA bulk copies (default);
+ *                               0: register kernels only
+ *   "gather"             0..2   gather walk: never / where measured faster (default 1) / wherever it applies
+ *   "zip"                0..2   zip kernels: never / only where the gather walk is not chosen / wherever
+ *                               they apply (default 2)
+ *   "zip_walks"          0..7   chunk-to-unit maps the zip kernels may use: 1 periodic + 2 by range +
+ *                               4 tabulated (default 7; the flat walk is always available)
+ *   "zip_by_range_slots" >= 1   fewest chunk slots of a range for the by-range walk (default 256)
+ *   "item_kb"            0..1024 KiB read per work item; 0 (default) = 32 / 16 / 8 by fan-out, and 20 / 12 / 6
+ *                               in the bulk-copy kernels
+ *   "pdl"                0/1    1: kernels use programmatic dependent launch (default); 0: plain stream order
+ *   "step_latency"       >= 0   elements added to the cost of every collective while searching: small
+ *                               transfers are bound by per-step latency, not by bytes (Section 8, the
+ *                               third research question); 0 (default) is the paper's cost model
+ *   "wait_polls"         >= 1   mbarrier polls before a bulk-copy block gives up (default 2^18)
+ *   "test_extra_tx"      >= 0   test only: makes every bounded wait run out (see redist_bulk_timeouts)
+ *   "test_shrink_tiles"  >= 0   test only: the checked build takes every tile to be that many bytes shorter
+ *                               (see redist_debug_bounds_report); no effect on the normal build
+ * Errors: EINVAL for an unknown name or a value out of range.
+ */
+redist_status redist_tuning_set(const char *name, int64_t value);
+redist_status redist_tuning_get(const char *name, int64_t *value);
+void redist_tuning_reset(void);
 
 /*
  * redist_execute -- run the plan on the GPU (asynchronous on `stream`).
@@ -153,16 +189,21 @@ void redist_plan_destroy(redist_plan_t *plan);
  *
  *   src_shards[N]   host array of DEVICE pointers; src_shards[d] holds localsize(src)*elem_bytes
  *                   bytes.  Devices that replicate a tile must hold identical bytes (not checked);
- *                   source pointers may alias each other.  Read only.
+ *                   source pointers may alias each other.  Read only.  When the tile size is not a
+ *                   multiple of 16 bytes the kernels may read (never write) up to the next 16-byte
+ *                   boundary past the tile's end -- always inside the allocation granule of any
+ *                   CUDA allocator, and, as tiles start on 16-byte boundaries, never a byte of
+ *                   another tile.
  *   dst_shards[N]   host array of DEVICE pointers; dst_shards[d] receives localsize(dst)*elem_bytes
  *                   bytes.  Every destination is written completely.
  *   scratch         DEVICE pointer to at least redist_plan_scratch_bytes(plan) bytes, or NULL when
  *                   that is 0.  Contents are undefined afterwards.
  *   cuda_stream     a cudaStream_t (NULL = default stream) on the current device
- * Ownership: all buffers and the stream belong to the caller.  The call allocates no device memory
- * (only small host-side tables), copies no table to the device (tables travel as kernel parameters)
- * and does not synchronize; ENOMEM is returned if a host table cannot be allocated.  A plan
- * may be executed from several host threads at once on different streams and buffers.
+ * Ownership: all buffers and the stream belong to the caller.  The call allocates nothing, on the
+ * host or on the device (pointer tables and the kernel parameter block live on the call's stack,
+ * about 100 KiB), copies no table to the device (tables travel as kernel parameters) and does not
+ * synchronize.  A plan may be executed from several host threads at once on different streams and
+ * buffers.
  * Errors: EINVAL, ESCRATCH, EALIGN (pointers must be multiples of redist_plan_alignment),
  * EOVERLAP (destination and scratch ranges must be disjoint from each other and from every
  * source; checked on the host), ECUDA (launch error; see redist_last_cuda_error).
@@ -170,6 +211,26 @@ void redist_plan_destroy(redist_plan_t *plan);
 redist_status redist_execute(const redist_plan_t *plan, const void *const *src_shards,
                              void *const *dst_shards, void *scratch, size_t scratch_bytes,
                              void *cuda_stream);
+
+/*
+ * redist_bind / redist_bound_execute -- the same execution split in two for callers that run one
+ * redistribution on the same buffers many times (every step of a training loop): binding validates
+ * the buffers exactly as redist_execute does and prepares every kernel launch once (entry point,
+ * launch shape, parameter block with both pointer tables); executing the bound plan is then the
+ * kernel launches and nothing else -- no checks, no table building, no allocation.
+ *
+ *   redist_bind            arguments as redist_execute; *out receives the bound plan (host memory,
+ *                          owned by the caller until redist_bound_destroy; it keeps the plan alive).
+ *                          The buffers must stay valid and in place while the bound plan is used.
+ *   redist_bound_execute   asynchronous on `cuda_stream`; may be called from several threads at once
+ *                          (but the launches of all calls write the same buffers: order them)
+ * Errors: redist_bind as redist_execute plus ENOMEM; redist_bound_execute EINVAL, ECUDA.
+ */
+typedef struct redist_bound_s redist_bound_t;
+redist_status redist_bind(const redist_plan_t *plan, const void *const *src_shards, void *const *dst_shards,
+                          void *scratch, size_t scratch_bytes, redist_bound_t **out);
+redist_status redist_bound_execute(const redist_bound_t *bound, void *cuda_stream);
+void redist_bound_destroy(redist_bound_t *bound);
 
 /*
  * redist_execute_host -- the same redistribution for tiles that live in HOST memory.
@@ -203,7 +264,8 @@ redist_status redist_execute_host(const redist_plan_t *plan, const void *const *
  *                   a larger plan is refused with REDIST_ESCRATCH and nothing runs
  *   src_shards[N], dst_shards[N], cuda_stream    exactly as for redist_execute
  * Set-up: the first call on each device (with that device current) looks up the device address of
- * the built-in array; make that first call before any stream capture begins.
+ * the built-in array; make that first call before any stream capture begins.  The address is kept
+ * for the life of the process: it does not survive a cudaDeviceReset.
  * Sharing: all calls on a device use the same array.  It keeps whatever the previous call left;
  * nothing in it has to start at zero, because every byte a step reads from it was written by an
  * earlier step of the same call.  Two calls whose kernels may overlap on the GPU (different
@@ -258,13 +320,28 @@ int32_t redist_last_cuda_error(void);
 
 /*
  * redist_bulk_timeouts -- health counter of the bulk-copy kernels (not part of the paper's method).
- * Aligned runs are moved by TMA bulk copies whose completion a thread block awaits on an mbarrier
- * with a bounded number of polls; a block whose wait runs out skips its stores, counts itself here
- * and returns, so a faulty copy engine shows up as a non-zero count and wrong output instead of a
- * hang.  Returns the count for the current device since the library was loaded (0 in a healthy run),
- * or -1 on a CUDA error.  Synchronizes the device.
+ * Runs are staged in shared memory by TMA bulk copies whose completion a thread block awaits on an
+ * mbarrier with a bounded number of polls ("wait_polls").  A block whose wait runs out stores
+ * nothing, counts itself here, keeps polling (sleeping up to 256 ns between polls) for as many polls
+ * again so that copies still in flight can land in shared memory it still owns, and returns: a
+ * faulty copy engine shows up as a non-zero count and unwritten output instead of a hang.  Returns
+ * the count for the current device since the library was loaded (0 in a healthy run), or -1 on a
+ * CUDA error.  Synchronizes the device.  A non-zero count means the outputs of the run are invalid.
+ * The tuning value "test_extra_tx" exists to test this path: it makes every block announce that
+ * many bytes more than its copies deliver, so every copy lands but no wait ever completes.
  */
 int64_t redist_bulk_timeouts(void);
+
+/*
+ * redist_debug_bounds_report -- checked build only (the library compiled with -DREDIST_BOUNDS, which
+ * the tests load in place of the normal one).  There every global access of the kernels is tested
+ * against the tiles of the launch and every dynamic shared-memory access against the launch's
+ * shared-memory size; a failing access is skipped, not performed.  out[0] = number of failed tests
+ * since the last call, out[1..4] = source line, thread block, side (1 read, 2 write, 3 shared memory)
+ * and distance from the nearest tile base of the first one.  The call resets the record.
+ * Synchronizes the device.  The normal build returns EUNSUPPORTED.
+ */
+redist_status redist_debug_bounds_report(int64_t out[5]);
 
 #ifdef __cplusplus
 }

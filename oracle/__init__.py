@@ -17,4 +17,5 @@ from .reference import (  # noqa: F401
     redistribute,
     reslice,
     set_threads,
+    tile_of,
 )

@@ -136,6 +136,16 @@ def reslice(mesh_shape, dtype, G: np.ndarray, out: List[np.ndarray] | None = Non
     return out
 
 
+def tile_of(mesh_shape, dtype, G: np.ndarray, device: int) -> np.ndarray:
+    """One device's tile of the global array ``G`` under ``dtype``: the block of ``G`` that starts at the
+    device's base offset T[[tau]](d) and has the local tile shape (the same definition as ``reslice``,
+    for callers that cannot hold every tile at once).  Returns a view into ``G``."""
+    tile, off = base_offsets(mesh_shape, dtype)
+    if tuple(G.shape[:-1]) != tuple(int(s) for s in dtype[0]):
+        raise ValueError("global array shape does not match the type")
+    return G[tuple(slice(int(o), int(o) + int(c)) for o, c in zip(off[device], tile))]
+
+
 def redistribute(mesh_shape, src_type, dst_type, shards: Sequence[np.ndarray], check: bool = True) -> List[np.ndarray]:
     """The definition: assemble the global array under ``src_type``, slice it under ``dst_type``.
 

@@ -6,10 +6,11 @@ not been built, loading fails with an error that says how to build it.
 
 A distributed type is ``(global_shape, axes)`` -- or any object with ``global_shape`` and ``axes``
 attributes -- where ``axes[k]`` lists the mesh axes (indices into ``mesh_shape``) that partition
-dimension ``k``, minor-to-major (Section 2.2 of the paper).
+dimension ``k``, minor-to-major (Section 2.1 of the paper).
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import json
 import os
@@ -21,6 +22,7 @@ LIB_PATH = os.environ.get("REDIST_LIB") or os.path.join(HERE, "libredist_b200.so
 FUSE_ADJACENT, FUSE_NONE, FUSE_ALL, NAIVE = 0, 1, 2, 3
 NO_OVERPARTITION = 16
 COST_PERMUTE = 32
+NO_CACHE = 64
 MAX_RANK = 8
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -29,6 +31,9 @@ KERNELS = ("dynslice", "alltoall", "allgather", "allpermute", "copy", "fused", "
 
 EXPORTS = (
     "redist_plan", "redist_plan_destroy", "redist_execute", "redist_execute_host", "redist_execute_static",
+    "redist_bind", "redist_bound_execute", "redist_bound_destroy",
+    "redist_plan_cache_stats", "redist_plan_cache_clear",
+    "redist_tuning_set", "redist_tuning_get", "redist_tuning_reset", "redist_debug_bounds_report",
     "redist_plan_num_devices", "redist_plan_rank", "redist_plan_local_elems", "redist_plan_scratch_bytes",
     "redist_plan_scratch_bytes_per_device", "redist_plan_staging_bytes", "redist_plan_alignment",
     "redist_plan_height", "redist_plan_cost", "redist_plan_num_steps", "redist_plan_num_launches",
@@ -113,6 +118,24 @@ def load() -> ctypes.CDLL:
     lib.redist_last_cuda_error.restype = i32
     lib.redist_bulk_timeouts.argtypes = []
     lib.redist_bulk_timeouts.restype = i64
+    lib.redist_bind.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, sz, ctypes.POINTER(vp)]
+    lib.redist_bind.restype = i32
+    lib.redist_bound_execute.argtypes = [vp, vp]
+    lib.redist_bound_execute.restype = i32
+    lib.redist_bound_destroy.argtypes = [vp]
+    lib.redist_bound_destroy.restype = None
+    lib.redist_plan_cache_stats.argtypes = [ctypes.POINTER(i64)] * 3
+    lib.redist_plan_cache_stats.restype = None
+    lib.redist_plan_cache_clear.argtypes = []
+    lib.redist_plan_cache_clear.restype = None
+    lib.redist_tuning_set.argtypes = [ctypes.c_char_p, i64]
+    lib.redist_tuning_set.restype = i32
+    lib.redist_tuning_get.argtypes = [ctypes.c_char_p, ctypes.POINTER(i64)]
+    lib.redist_tuning_get.restype = i32
+    lib.redist_tuning_reset.argtypes = []
+    lib.redist_tuning_reset.restype = None
+    lib.redist_debug_bounds_report.argtypes = [ctypes.POINTER(i64)]
+    lib.redist_debug_bounds_report.restype = i32
     _lib = lib
     return lib
 
@@ -320,30 +343,34 @@ class Plan:
 
     def bind(self, src_ptrs: Sequence[int], dst_ptrs: Sequence[int], scratch_ptr: int = 0,
              scratch_bytes: int = 0):
-        """Marshal the pointer tables once; the returned callable runs ``redist_execute`` on a stream
-        (``call(stream_ptr)``) with no per-call Python work beyond the foreign call itself."""
+        """``redist_bind``: validate the buffers and prepare every launch once; the returned callable runs
+        ``redist_bound_execute`` on a stream (``call(stream_ptr)``) -- the kernel launches and nothing else.
+        The buffers must stay alive and in place as long as the callable is used."""
+        if len(src_ptrs) != self.n_devices or len(dst_ptrs) != self.n_devices:
+            raise RedistError(1, "one tile per virtual device is required")
         s = (ctypes.c_void_p * len(src_ptrs))(*src_ptrs)
         d = (ctypes.c_void_p * len(dst_ptrs))(*dst_ptrs)
-        sp, sn, h, fn = ctypes.c_void_p(scratch_ptr or None), ctypes.c_size_t(scratch_bytes), self._h, \
-            self._lib.redist_execute
+        h = ctypes.c_void_p()
+        rc = self._lib.redist_bind(self._h, s, d, ctypes.c_void_p(scratch_ptr or None), scratch_bytes, ctypes.byref(h))
+        if rc:
+            raise RedistError(rc, "redist_bind")
+        return _Bound(self, h)
 
-        def call(stream_ptr: int = 0):
-            rc = fn(h, s, d, sp, sn, ctypes.c_void_p(stream_ptr or None))
-            if rc:
-                raise RedistError(rc, "redist_execute")
-
-        return call
+    def _check_tiles(self, src_shards, dst_shards, cuda: bool = True) -> None:
+        """What the C entry points cannot know: one tile per virtual device, each a contiguous tensor in
+        the right memory holding exactly localsize*elem_bytes bytes."""
+        if len(src_shards) != self.n_devices or len(dst_shards) != self.n_devices:
+            raise RedistError(1, "one tile per virtual device is required")
+        sb, db = self.local_elems(0) * self.elem_bytes, self.local_elems(1) * self.elem_bytes
+        for t, need in [(x, sb) for x in src_shards] + [(x, db) for x in dst_shards]:
+            if t.is_cuda != cuda or not t.is_contiguous() or t.numel() * t.element_size() != need:
+                raise RedistError(1, "tiles must be contiguous %s tensors of the local size" % ("CUDA" if cuda else "host"))
 
     def execute(self, src_shards, dst_shards, scratch=None, stream=None) -> None:
         """``redist_execute`` on lists of CUDA tensors (one per virtual device), asynchronous."""
         import torch
 
-        if len(src_shards) != self.n_devices or len(dst_shards) != self.n_devices:
-            raise RedistError(1, "one tile per virtual device is required")
-        sb, db = self.local_elems(0) * self.elem_bytes, self.local_elems(1) * self.elem_bytes
-        for t, need in [(x, sb) for x in src_shards] + [(x, db) for x in dst_shards]:
-            if not t.is_cuda or not t.is_contiguous() or t.numel() * t.element_size() != need:
-                raise RedistError(1, "tiles must be contiguous CUDA tensors of the local size")
+        self._check_tiles(src_shards, dst_shards)
         if stream is None:
             stream = torch.cuda.current_stream()
         sp = scratch.data_ptr() if scratch is not None else 0
@@ -357,6 +384,7 @@ class Plan:
         (plans needing more than ``STATIC_SCRATCH_BYTES`` are refused)."""
         import torch
 
+        self._check_tiles(src_shards, dst_shards)
         if stream is None:
             stream = torch.cuda.current_stream()
         n = self.n_devices
@@ -370,6 +398,7 @@ class Plan:
         """``redist_execute_host``: host tiles in, host tiles out, staged through ``dev_src``/``dev_dst``."""
         import torch
 
+        self._check_tiles(src_host, dst_host, cuda=False)
         if stream is None:
             stream = torch.cuda.current_stream()
         n = self.n_devices
@@ -390,6 +419,76 @@ class Plan:
 
         n = self.scratch_bytes
         return torch.empty(n, dtype=torch.uint8, device=device) if n else None
+
+
+class _Bound:
+    """A plan bound to one set of buffers (``redist_bind``); calling it launches the kernels on a stream."""
+
+    def __init__(self, plan: Plan, handle):
+        self._plan, self._h = plan, handle          # the plan object stays alive with its bound form
+        self._fn, self._destroy = plan._lib.redist_bound_execute, plan._lib.redist_bound_destroy
+
+    def __call__(self, stream_ptr: int = 0) -> None:
+        rc = self._fn(self._h, ctypes.c_void_p(stream_ptr or None))
+        if rc:
+            raise RedistError(rc, "redist_bound_execute")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+
+def tuning_set(name: str, value: int) -> None:
+    """``redist_tuning_set``: change a tuning value for the plans created from now on."""
+    rc = load().redist_tuning_set(name.encode(), int(value))
+    if rc:
+        raise RedistError(rc, f"redist_tuning_set({name!r}, {value})")
+
+
+def tuning_get(name: str) -> int:
+    out = ctypes.c_int64()
+    rc = load().redist_tuning_get(name.encode(), ctypes.byref(out))
+    if rc:
+        raise RedistError(rc, f"redist_tuning_get({name!r})")
+    return int(out.value)
+
+
+def tuning_reset() -> None:
+    load().redist_tuning_reset()
+
+
+@contextlib.contextmanager
+def tuning(**values):
+    """``with tuning(bulk=0, gather=0): plan = Plan(...)`` -- plans created inside get these values."""
+    try:
+        for k, v in values.items():
+            tuning_set(k, v)
+        yield
+    finally:
+        tuning_reset()
+
+
+def plan_cache_stats():
+    """``(hits, misses, entries)`` of the plan cache."""
+    h, m, e = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    load().redist_plan_cache_stats(ctypes.byref(h), ctypes.byref(m), ctypes.byref(e))
+    return int(h.value), int(m.value), int(e.value)
+
+
+def plan_cache_clear() -> None:
+    load().redist_plan_cache_clear()
+
+
+def debug_bounds_report():
+    """Checked build only: ``(violations, line, block, side, distance)`` since the last call."""
+    out = (ctypes.c_int64 * 5)()
+    rc = load().redist_debug_bounds_report(out)
+    if rc:
+        raise RedistError(rc, "redist_debug_bounds_report")
+    return tuple(int(v) for v in out)
 
 
 def redist_bulk_timeouts() -> int:

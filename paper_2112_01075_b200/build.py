@@ -1,21 +1,32 @@
 """Build step: compile the CUDA library for sm_100a with nvcc, in-tree.
 
-``python -m paper_2112_01075_b200.build`` (or ``build()``) produces ``libredist_b200.so`` next to this
-file.  nvcc cross-compiles without a GPU.  The CUDA runtime is linked statically, so the library
-loads (and its host-only entry points work) on a machine without a driver.
+``python -m paper_2112_01075_b200.build`` (or ``build()``) produces, next to this file,
+
+* ``libredist_b200.so`` -- the library, and
+* ``libredist_b200_bounds.so`` -- the same sources with the kernels compiled with ``-DREDIST_BOUNDS``:
+  every global and shared-memory access is tested against the launch's tiles and skipped if it fails,
+  the first failure is recorded (``redist_debug_bounds_report``).  Only the tests load it.
+
+nvcc cross-compiles without a GPU.  The CUDA runtime is linked statically, so the libraries load (and
+their host-only entry points work) on a machine without a driver.  Sources compile in parallel into
+``_obj/``; only what changed is recompiled.
 """
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_obj")
 LIB = os.path.join(HERE, "libredist_b200.so")
+LIB_BOUNDS = os.path.join(HERE, "libredist_b200_bounds.so")
 SOURCES = ["api.cu", "kernels.cu", "static_scratch.cu", "planner.cpp", "descriptor.cpp", "describe.cpp"]
 HEADERS = ["plan.hpp", "copy_params.h", "kernels.h"]
+CHECKED = ["kernels.cu"]          # sources that differ in the checked build
 
 
 def _nvcc() -> str:
@@ -25,31 +36,60 @@ def _nvcc() -> str:
     return "nvcc"
 
 
+def _deps():
+    return [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.join(ROOT, "include", "redist.h"),
+                                                                   os.path.abspath(__file__)]
+
+
 def needs_build() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.join(ROOT, "include", "redist.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+    newest = max(os.path.getmtime(d) for d in _deps())
+    return any(not os.path.exists(lib) or os.path.getmtime(lib) < newest for lib in (LIB, LIB_BOUNDS))
+
+
+def _compile(src: str, obj: str, defines, verbose: bool) -> str:
+    cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+           "-Xcompiler", "-fPIC,-Wall,-Wno-unknown-pragmas", "-c",
+           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", obj] + [f"-D{d}" for d in defines]
+    if verbose:
+        cmd += ["-Xptxas", "-v"]
+    res = subprocess.run(cmd + [os.path.join(CSRC, src)], capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError(f"nvcc failed on {src}")
+    return res.stdout + res.stderr
+
+
+def _link(objs, lib: str) -> None:
+    tmp = lib + f".tmp{os.getpid()}"
+    res = subprocess.run([_nvcc(), "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
+                          "-o", tmp] + objs, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("link failed")
+    os.replace(tmp, lib)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-Xcompiler", "-fPIC,-Wall,-Wno-unknown-pragmas", "-shared", "-cudart", "static",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp]
+    os.makedirs(OBJ, exist_ok=True)
+    newest_header = max(os.path.getmtime(d) for d in _deps() if not d.endswith((".cu", ".cpp")))
+    jobs = []
+    for src in SOURCES:
+        variants = [("", [])] + ([("_bounds", ["REDIST_BOUNDS"])] if src in CHECKED else [])
+        for suffix, defines in variants:
+            obj = os.path.join(OBJ, os.path.splitext(src)[0] + suffix + ".o")
+            stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(
+                newest_header, os.path.getmtime(os.path.join(CSRC, src)))
+            jobs.append((src, obj, defines, stale))
+    with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
+        logs = list(pool.map(lambda j: _compile(j[0], j[1], j[2], verbose) if j[3] else "", jobs))
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, f) for f in SOURCES]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed")
-    if verbose:
-        sys.stderr.write(res.stdout + res.stderr)
-    os.replace(tmp, LIB)
+        sys.stderr.write("".join(logs))
+    plain = [os.path.join(OBJ, os.path.splitext(s)[0] + ".o") for s in SOURCES]
+    checked = [os.path.join(OBJ, os.path.splitext(s)[0] + ("_bounds" if s in CHECKED else "") + ".o") for s in SOURCES]
+    _link(plain, LIB)
+    _link(checked, LIB_BOUNDS)
     return LIB
 
 

@@ -1,10 +1,13 @@
-// The C boundary: plan creation, execution and queries.
+// The C boundary: plan creation (with the plan cache and the tuning values), execution and queries.
 #include <cuda_runtime.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <cstring>
+#include <deque>
+#include <mutex>
 #include <new>
+#include <string>
+#include <unordered_map>
 #include <vector>
 
 #include "kernels.h"
@@ -16,37 +19,29 @@ namespace redist {
 thread_local int tl_cuda_error = 0;
 }
 
-namespace {
+// A plan bound to one set of buffers: every launch prepared once (entry point, launch shape, parameter
+// block with both pointer tables), so that executing it is the kernel launches and nothing else.
+struct redist_bound_s {
+    std::shared_ptr<const redist::Plan> ref;
+    std::vector<redist::PreparedLaunch> launches;
+};
 
-// One thread block per work item by default: the hardware block scheduler balances the load and
-// keeps the tail to one item.  REDIST_GRID_MULT=k (tuning knob) switches to a grid-stride loop with
-// k blocks per SM.
-int grid_for(const CopyGeometry &g)
-{
-    static const long long cap = [] {
-        const char *m = std::getenv("REDIST_GRID_MULT");
-        if (!m || std::atoi(m) <= 0) return 0ll;
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-        return 1ll * n * std::atoi(m);
-    }();
-    return int(cap > 0 ? std::min<long long>(g.n_items, cap) : g.n_items);
-}
+namespace {
 
 struct Range {
     uintptr_t lo, hi;
     int kind;   // 0 source (may alias other sources), 1 written
 };
 
-bool overlaps(std::vector<Range> &r)
+// a written range may not intersect any other range; sources may intersect sources (sweep over the
+// ranges sorted by start; sorts `r` in place, allocates nothing)
+bool overlaps(Range *r, int n)
 {
-    std::sort(r.begin(), r.end(), [](const Range &a, const Range &b) { return a.lo < b.lo; });
-    // sweep: a written range may not intersect any other range; sources may intersect sources
+    std::sort(r, r + n, [](const Range &a, const Range &b) { return a.lo < b.lo; });
     uintptr_t max_hi_written = 0, max_hi_any = 0;
     bool have_w = false, have_any = false;
-    for (const Range &x : r) {
+    for (int i = 0; i < n; ++i) {
+        const Range &x = r[i];
         if (x.lo >= x.hi) continue;
         if (x.kind == 1) {
             if (have_any && x.lo < max_hi_any) return true;
@@ -63,7 +58,134 @@ bool overlaps(std::vector<Range> &r)
     return false;
 }
 
+// ---- tuning values and plan cache (process-wide, behind one mutex) ----------------------------
+std::mutex g_mutex;
+Tuning g_tuning;
+
+struct TuningName {
+    const char *name;
+    int64_t Tuning::*field;
+    int64_t lo, hi;
+};
+const TuningName kTuningNames[] = {
+    {"bulk", &Tuning::bulk, 0, 1},
+    {"gather", &Tuning::gather, 0, 2},
+    {"zip", &Tuning::zip, 0, 2},
+    {"zip_walks", &Tuning::zip_walks, 0, 7},
+    {"zip_by_range_slots", &Tuning::zip_by_range_slots, 1, 1 << 20},
+    {"item_kb", &Tuning::item_kb, 0, 1024},
+    {"pdl", &Tuning::pdl, 0, 1},
+    {"step_latency", &Tuning::step_latency, 0, int64_t(1) << 50},
+    {"wait_polls", &Tuning::wait_polls, 1, int64_t(1) << 30},
+    {"test_extra_tx", &Tuning::test_extra_tx, 0, 1 << 20},
+    {"test_shrink_tiles", &Tuning::test_shrink_tiles, 0, 1 << 20},
+};
+
+constexpr size_t kCacheEntries = 256;
+std::unordered_map<std::string, std::shared_ptr<const Plan>> g_cache;
+std::deque<std::string> g_cache_order;     // oldest first
+int64_t g_cache_hits = 0, g_cache_misses = 0;
+
+std::string cache_key(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *src, const redist_type *dst,
+                      int32_t elem_bytes, uint32_t flags, const Tuning &t)
+{
+    std::string k;
+    auto put = [&k](int64_t v) { k.append(reinterpret_cast<const char *>(&v), sizeof v); };
+    put(n_mesh_axes);
+    for (int a = 0; a < n_mesh_axes; ++a) put(mesh_shape[a]);
+    for (const redist_type *ty : {src, dst}) {
+        put(ty->rank);
+        for (int d = 0; d < ty->rank; ++d) {
+            put(ty->global_shape[d]);
+            put(ty->axes_off[d + 1] - ty->axes_off[d]);
+            for (int q = ty->axes_off[d]; q < ty->axes_off[d + 1]; ++q) put(ty->axes[q]);
+        }
+    }
+    put(elem_bytes);
+    put(flags);
+    for (const TuningName &n : kTuningNames) put(t.*(n.field));
+    return k;
+}
+
+// Buffer checks shared by every execute entry point: pointers present and aligned, destination and
+// scratch ranges disjoint from each other and from every source.  Allocates nothing.
+redist_status check_buffers(const Plan &p, const void *const *src_shards, void *const *dst_shards, const void *scratch,
+                            size_t scratch_range)
+{
+    const int N = p.n_devices;
+    const uintptr_t amask = uintptr_t(p.alignment) - 1;
+    const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
+    Range ranges[2 * REDIST_MAX_DEVICES + 1];
+    int n = 0;
+    for (int d = 0; d < N; ++d) {
+        if (!src_shards[d] || !dst_shards[d]) return REDIST_EINVAL;
+        const uintptr_t s = uintptr_t(src_shards[d]), t = uintptr_t(dst_shards[d]);
+        if ((s & amask) || (t & amask)) return REDIST_EALIGN;
+        ranges[n++] = Range{s, s + uintptr_t(sb), 0};
+        ranges[n++] = Range{t, t + uintptr_t(db), 1};
+    }
+    if (scratch_range > 0) {
+        if (uintptr_t(scratch) & 255) return REDIST_EALIGN;
+        ranges[n++] = Range{uintptr_t(scratch), uintptr_t(scratch) + uintptr_t(scratch_range), 1};
+    }
+    return overlaps(ranges, n) ? REDIST_EOVERLAP : REDIST_OK;
+}
+
+// Pointer tables of one launch from the caller's buffers, then the prepared launch.
+redist_status prepare_launch(const Plan &p, const Launch &L, const void *const *src_shards, void *const *dst_shards,
+                             char *scratch, PreparedLaunch &pl)
+{
+    const int N = p.n_devices;
+    auto buffer = [&](BufKind kind, int32_t dev) -> char * {
+        switch (kind) {
+        case BUF_SRC: return static_cast<char *>(const_cast<void *>(src_shards[dev]));
+        case BUF_DST: return static_cast<char *>(dst_shards[dev]);
+        case BUF_SCRATCH0: return scratch + i64(dev) * p.slot_bytes;
+        case BUF_SCRATCH1: return scratch + (i64(N) + dev) * p.slot_bytes;
+        default: return scratch;
+        }
+    };
+    const int ns = int(L.src_holder.size()), nd = int(L.dst_devs.size());
+    if (ns > REDIST_MAX_DEVICES || nd > REDIST_MAX_DEVICES) return REDIST_EUNSUPPORTED;
+    const char *stab[REDIST_MAX_DEVICES];
+    char *dtab[REDIST_MAX_DEVICES];
+    for (int t = 0; t < ns; ++t) stab[t] = buffer(L.from, L.src_holder[t] < 0 ? 0 : L.src_holder[t]);
+    for (int t = 0; t < nd; ++t) dtab[t] = buffer(L.to, L.dst_devs[t] < 0 ? 0 : L.dst_devs[t]);
+    cudaError_t ce = prepare_copy(L.kernel, L.geo, stab, ns, dtab, nd, int(p.tuning.pdl), pl);
+    if (ce != cudaSuccess) {
+        tl_cuda_error = int(ce);
+        return REDIST_ECUDA;
+    }
+    return REDIST_OK;
+}
+
 }  // namespace
+
+namespace redist {
+
+// Checks, then one kernel launch per entry of the plan's launch list.  Tables and the parameter block
+// live on this call's stack (about 100 KiB); nothing is allocated on the host or on the device.
+redist_status run_plan(const Plan &p, const void *const *src_shards, void *const *dst_shards, void *scratch,
+                       size_t scratch_range, void *cuda_stream)
+{
+    redist_status rc = check_buffers(p, src_shards, dst_shards, scratch, scratch_range);
+    if (rc != REDIST_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    PreparedLaunch pl;
+    for (const Launch &L : p.launches) {
+        if (L.geo.n_items == 0) continue;
+        rc = prepare_launch(p, L, src_shards, dst_shards, static_cast<char *>(scratch), pl);
+        if (rc != REDIST_OK) return rc;
+        cudaError_t ce = launch_prepared(pl, stream);
+        if (ce != cudaSuccess) {
+            tl_cuda_error = int(ce);
+            return REDIST_ECUDA;
+        }
+    }
+    return REDIST_OK;
+}
+
+}  // namespace redist
 
 extern "C" {
 
@@ -135,7 +257,8 @@ redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const 
         return REDIST_EINVAL;
     if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4 && elem_bytes != 8 && elem_bytes != 16)
         return REDIST_EINVAL;
-    if (flags & ~uint32_t(REDIST_MODE_MASK | REDIST_NO_OVERPARTITION | REDIST_COST_PERMUTE)) return REDIST_EINVAL;
+    if (flags & ~uint32_t(REDIST_MODE_MASK | REDIST_NO_OVERPARTITION | REDIST_COST_PERMUTE | REDIST_NO_CACHE))
+        return REDIST_EINVAL;
     i64 N = 1;
     for (int a = 0; a < n_mesh_axes; ++a) {
         if (mesh_shape[a] < 1) return REDIST_EINVAL;
@@ -155,10 +278,31 @@ redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const 
         if (gsize > (i64(1) << 56) / src->global_shape[k]) return REDIST_EUNSUPPORTED;
         gsize *= src->global_shape[k];
     }
-    redist_plan_s *h = new (std::nothrow) redist_plan_s();
-    if (!h) return REDIST_ENOMEM;
+    // plan cache: the same problem under the same tuning values gets the same (immutable) plan again
+    const bool cached = (flags & REDIST_NO_CACHE) == 0;
+    flags &= ~uint32_t(REDIST_NO_CACHE);
+    std::shared_ptr<Plan> fresh;
     try {
-        Plan &p = h->p;
+        Tuning tuning;
+        std::string key;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            tuning = g_tuning;
+            if (cached) {
+                key = cache_key(n_mesh_axes, mesh_shape, src, dst, elem_bytes, flags, tuning);
+                auto it = g_cache.find(key);
+                if (it != g_cache.end()) {
+                    ++g_cache_hits;
+                    redist_plan_s *h = new redist_plan_s(it->second);
+                    *out = h;
+                    return REDIST_OK;
+                }
+                ++g_cache_misses;
+            }
+        }
+        fresh = std::make_shared<Plan>();
+        Plan &p = *fresh;
+        p.tuning = tuning;
         p.n_mesh_axes = n_mesh_axes;
         p.rank = src->rank;
         p.elem_bytes = elem_bytes;
@@ -191,16 +335,85 @@ redist_status redist_plan(int32_t n_mesh_axes, const int64_t *mesh_shape, const 
             }
         }
         if (rc == REDIST_OK) describe(p);
+        if (rc != REDIST_OK) return rc;
+        redist_plan_s *h = new redist_plan_s(fresh);
+        if (cached) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            if (g_cache.emplace(key, fresh).second) {
+                g_cache_order.push_back(key);
+                if (g_cache_order.size() > kCacheEntries) {
+                    g_cache.erase(g_cache_order.front());
+                    g_cache_order.pop_front();
+                }
+            }
+        }
+        *out = h;
+        return REDIST_OK;
     } catch (const std::bad_alloc &) {
-        rc = REDIST_ENOMEM;
+        return REDIST_ENOMEM;
     } catch (...) {
-        rc = REDIST_EINTERNAL;
+        return REDIST_EINTERNAL;
     }
-    if (rc != REDIST_OK) {
-        delete h;
-        return rc;
+}
+
+void redist_plan_cache_stats(int64_t *hits, int64_t *misses, int64_t *entries)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (hits) *hits = g_cache_hits;
+    if (misses) *misses = g_cache_misses;
+    if (entries) *entries = int64_t(g_cache.size());
+}
+
+void redist_plan_cache_clear(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_cache.clear();
+    g_cache_order.clear();
+    g_cache_hits = g_cache_misses = 0;
+}
+
+redist_status redist_tuning_set(const char *name, int64_t value)
+{
+    if (!name) return REDIST_EINVAL;
+    for (const TuningName &n : kTuningNames)
+        if (std::strcmp(name, n.name) == 0) {
+            if (value < n.lo || value > n.hi) return REDIST_EINVAL;
+            std::lock_guard<std::mutex> lock(g_mutex);
+            g_tuning.*(n.field) = value;
+            return REDIST_OK;
+        }
+    return REDIST_EINVAL;
+}
+
+redist_status redist_tuning_get(const char *name, int64_t *value)
+{
+    if (!name || !value) return REDIST_EINVAL;
+    for (const TuningName &n : kTuningNames)
+        if (std::strcmp(name, n.name) == 0) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            *value = g_tuning.*(n.field);
+            return REDIST_OK;
+        }
+    return REDIST_EINVAL;
+}
+
+void redist_tuning_reset(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_tuning = Tuning();
+}
+
+redist_status redist_debug_bounds_report(int64_t out[5])
+{
+    if (!out) return REDIST_EINVAL;
+    long long r[5];
+    cudaError_t ce = read_bounds_report(r);
+    if (ce == cudaErrorNotSupported) return REDIST_EUNSUPPORTED;
+    if (ce != cudaSuccess) {
+        tl_cuda_error = int(ce);
+        return REDIST_ECUDA;
     }
-    *out = h;
+    for (int i = 0; i < 5; ++i) out[i] = r[i];
     return REDIST_OK;
 }
 
@@ -287,50 +500,34 @@ redist_status redist_execute(const redist_plan_t *plan, const void *const *src_s
     try {
         if (!plan || !src_shards || !dst_shards) return REDIST_EINVAL;
         const Plan &p = plan->p;
-        const int N = p.n_devices;
         if (p.scratch_bytes > 0 && (!scratch || scratch_bytes < size_t(p.scratch_bytes))) return REDIST_ESCRATCH;
-        const uintptr_t amask = uintptr_t(p.alignment) - 1;
-        const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
-        std::vector<Range> ranges;
-        ranges.reserve(size_t(2 * N + 1));
-        for (int d = 0; d < N; ++d) {
-            if (!src_shards[d] || !dst_shards[d]) return REDIST_EINVAL;
-            const uintptr_t s = uintptr_t(src_shards[d]), t = uintptr_t(dst_shards[d]);
-            if ((s & amask) || (t & amask)) return REDIST_EALIGN;
-            ranges.push_back(Range{s, s + uintptr_t(sb), 0});
-            ranges.push_back(Range{t, t + uintptr_t(db), 1});
-        }
-        if (p.scratch_bytes > 0) {
-            if (uintptr_t(scratch) & 255) return REDIST_EALIGN;
-            ranges.push_back(Range{uintptr_t(scratch), uintptr_t(scratch) + uintptr_t(p.scratch_bytes), 1});
-        }
-        if (overlaps(ranges)) return REDIST_EOVERLAP;
+        return run_plan(p, src_shards, dst_shards, scratch, size_t(p.scratch_bytes), cuda_stream);
+    } catch (...) {
+        return REDIST_EINTERNAL;
+    }
+}
 
-        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-        auto buffer = [&](BufKind kind, int32_t dev) -> char * {
-            switch (kind) {
-            case BUF_SRC: return static_cast<char *>(const_cast<void *>(src_shards[dev]));
-            case BUF_DST: return static_cast<char *>(dst_shards[dev]);
-            case BUF_SCRATCH0: return static_cast<char *>(scratch) + i64(dev) * p.slot_bytes;
-            case BUF_SCRATCH1: return static_cast<char *>(scratch) + (i64(N) + dev) * p.slot_bytes;
-            default: return static_cast<char *>(scratch);
-            }
-        };
-        std::vector<const char *> stab;
-        std::vector<char *> dtab;
+redist_status redist_bind(const redist_plan_t *plan, const void *const *src_shards, void *const *dst_shards,
+                          void *scratch, size_t scratch_bytes, redist_bound_t **out)
+{
+    if (!plan || !src_shards || !dst_shards || !out) return REDIST_EINVAL;
+    const Plan &p = plan->p;
+    if (p.scratch_bytes > 0 && (!scratch || scratch_bytes < size_t(p.scratch_bytes))) return REDIST_ESCRATCH;
+    redist_status rc = check_buffers(p, src_shards, dst_shards, scratch, size_t(p.scratch_bytes));
+    if (rc != REDIST_OK) return rc;
+    try {
+        std::unique_ptr<redist_bound_s> b(new redist_bound_s());
+        b->ref = plan->ref;
+        size_t n = 0;
+        for (const Launch &L : p.launches) n += L.geo.n_items != 0;
+        b->launches.resize(n);
+        size_t q = 0;
         for (const Launch &L : p.launches) {
-            stab.resize(L.src_holder.size());
-            dtab.resize(L.dst_devs.size());
-            for (size_t t = 0; t < stab.size(); ++t) stab[t] = buffer(L.from, L.src_holder[t] < 0 ? 0 : L.src_holder[t]);
-            for (size_t t = 0; t < dtab.size(); ++t) dtab[t] = buffer(L.to, L.dst_devs[t] < 0 ? 0 : L.dst_devs[t]);
             if (L.geo.n_items == 0) continue;
-            cudaError_t ce = launch_copy(L.kernel, L.geo, stab.data(), int(stab.size()), dtab.data(), int(dtab.size()),
-                                         grid_for(L.geo), stream);
-            if (ce != cudaSuccess) {
-                tl_cuda_error = int(ce);
-                return REDIST_ECUDA;
-            }
+            rc = prepare_launch(p, L, src_shards, dst_shards, static_cast<char *>(scratch), b->launches[q++]);
+            if (rc != REDIST_OK) return rc;
         }
+        *out = b.release();
         return REDIST_OK;
     } catch (const std::bad_alloc &) {
         return REDIST_ENOMEM;
@@ -338,6 +535,22 @@ redist_status redist_execute(const redist_plan_t *plan, const void *const *src_s
         return REDIST_EINTERNAL;
     }
 }
+
+redist_status redist_bound_execute(const redist_bound_t *bound, void *cuda_stream)
+{
+    if (!bound) return REDIST_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (const PreparedLaunch &pl : bound->launches) {
+        cudaError_t ce = launch_prepared(pl, stream);
+        if (ce != cudaSuccess) {
+            tl_cuda_error = int(ce);
+            return REDIST_ECUDA;
+        }
+    }
+    return REDIST_OK;
+}
+
+void redist_bound_destroy(redist_bound_t *bound) { delete bound; }
 
 redist_status redist_execute_host(const redist_plan_t *plan, const void *const *src_host, void *const *dst_host,
                                   void *dev_src, size_t dev_src_bytes, void *dev_dst, size_t dev_dst_bytes,
@@ -353,8 +566,8 @@ redist_status redist_execute_host(const redist_plan_t *plan, const void *const *
         const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
         const i64 sp = (sb + 255) / 256 * 256, dp = (db + 255) / 256 * 256;
         cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-        std::vector<const void *> s(N);
-        std::vector<void *> t(N);
+        const void *s[REDIST_MAX_DEVICES];
+        void *t[REDIST_MAX_DEVICES];
         for (int d = 0; d < N; ++d) {
             if (!src_host[d] || !dst_host[d]) return REDIST_EINVAL;
             s[d] = static_cast<char *>(dev_src) + d * sp;
@@ -367,7 +580,7 @@ redist_status redist_execute_host(const redist_plan_t *plan, const void *const *
                 return REDIST_ECUDA;
             }
         }
-        redist_status rc = redist_execute(plan, s.data(), t.data(), scratch, scratch_bytes, cuda_stream);
+        redist_status rc = redist_execute(plan, s, t, scratch, scratch_bytes, cuda_stream);
         if (rc != REDIST_OK) return rc;
         for (int d = 0; d < N; ++d) {
             cudaError_t ce = cudaMemcpyAsync(dst_host[d], t[d], size_t(db), cudaMemcpyDeviceToHost, stream);
@@ -377,8 +590,6 @@ redist_status redist_execute_host(const redist_plan_t *plan, const void *const *
             }
         }
         return REDIST_OK;
-    } catch (const std::bad_alloc &) {
-        return REDIST_ENOMEM;
     } catch (...) {
         return REDIST_EINTERNAL;
     }

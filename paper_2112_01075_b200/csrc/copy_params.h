@@ -121,6 +121,12 @@ struct CopyGeometry {
     FastDiv row_n[kMaxRowDigits];
     int64_t row_b1[kMaxRowDigits];       // byte stride of the row digit, source / target
     int64_t row_b2[kMaxRowDigits];
+    uint32_t wait_polls;             // bulk-copy kernels: mbarrier polls before a block gives up (bounded wait)
+    uint32_t test_extra_tx;          // test only: bytes announced on the mbarrier beyond what the copies deliver, so
+                                     // that every copy lands but the phase never completes (0 in every real plan)
+    uint32_t n_src_tab, n_dst_tab;   // entries of the two pointer tables
+    uint64_t src_tile_bytes;         // bytes of one source / target tile (the checked build tests every access
+    uint64_t dst_tile_bytes;         // against them; the kernels themselves do not need them)
 };
 
 template <int NT>

@@ -3,7 +3,6 @@
 // of adjacent collectives -- merging of adjacent operations, Section 7.1, taken one step further:
 // on one GPU any run of steps composes into a single strided copy).
 #include <algorithm>
-#include <cstdlib>
 #include <numeric>
 
 #include "plan.hpp"
@@ -86,10 +85,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     G.inner_span = 1;
     G.inner_mul = 1;
     i64 inner = 1;
-    static const i64 kInnerRun = [] {
-        const char *v = std::getenv("REDIST_INNER_RUN");   // tuning knob: runs below this many bytes get adjacent-piece item numbering
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 16384);
-    }();
+    const i64 kInnerRun = 16384;   // runs below this many bytes get adjacent-piece item numbering (measured)
     if (kp >= 0 && run_bytes < kInnerRun && nq[kp] > 1 && m1[kp] * m2[kp] > 1) {
         inner = m1[kp] * m2[kp];
         uint32_t u = 0;
@@ -105,10 +101,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // below kFastStride on that side) are moved to the end of the digit list: they become the fastest
     // part of the box number, and -- see decode_box -- vary faster than the row groups of a box, so that the
     // blocks which share those lines run at the same time and partial sectors merge in L2.
-    static const i64 kFastStride = [] {
-        const char *v = std::getenv("REDIST_FAST_STRIDE");   // tuning knob: 0 switches the reordering off
-        return i64(v ? std::atoi(v) : 16384);
-    }();
+    const i64 kFastStride = 16384;
     G.fast_boxes = make_div(1);
     {
         std::vector<uint32_t> slow, fast;
@@ -189,10 +182,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     G.rows = uint32_t(n_rows);
     // work items: about 32 KiB read each -- less when every byte read is stored to several
     // replicas, so that the bytes written per block stay comparable
-    static const i64 kItemKb = [] {
-        const char *v = std::getenv("REDIST_ITEM_KB");   // tuning knob: KiB read per work item
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 0);
-    }();
+    const Tuning &tune = p.tuning;
+    const i64 kItemKb = tune.item_kb > 0 ? tune.item_kb : 0;
     i64 fan = 1;
     if (!b.shared_global) {
         i64 nt = 1;
@@ -203,20 +194,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // Items of the plain bulk-copy kernels: measured best at 20 KiB (12 / 6 KiB for fan-out >= 2 / >= 4) once
     // the kernels wait for their predecessor only after decoding the item -- finer tail, more blocks ready
     // behind the wait.
-    static const i64 kBulkItemKb = [] {
-        const char *v = std::getenv("REDIST_BULK_ITEM_KB");   // tuning knob: KiB per item of the bulk-copy kernels at fan-out 1 (2-3: 0.6x, 4 and more: 0.3x)
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 20);
-    }();
+    const i64 kBulkItemKb = 20;
     // aligned segments of 512 bytes or more go through the bulk-copy kernels (at most one segment per
     // thread, the item staged in at most 47 KiB of shared memory)
-    static const bool kBulk = [] {
-        const char *v = std::getenv("REDIST_BULK");      // tuning knob: REDIST_BULK=0 keeps aligned runs on the register path
-        return !v || std::atoi(v) > 0;
-    }();
-    static const i64 kBulkMin = [] {
-        const char *v = std::getenv("REDIST_BULK_MIN");  // tuning knob: shortest segment moved by a bulk copy
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 512);
-    }();
+    const bool kBulk = tune.bulk > 0;     // 0 keeps every run on the register kernels
+    const i64 kBulkMin = 512;             // shortest segment moved by a bulk copy
     const i64 max_chunks = run_bytes / 16;           // whole 16-byte chunks a run can hold
     if (max_chunks >= (1ll << 31)) return REDIST_EUNSUPPORTED;
     const i64 bulk_item_bytes = kItemKb == 0 && kBulk && G.aligned && run_bytes >= kBulkMin
@@ -228,12 +210,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     bool ragged_bulk = false;
     // gather walk: short runs whose m pieces interleave on one side; the target bytes of a table row
     // (the stretch) are produced in whole 16-byte chunks
-    static const int kGather = [] {
-        // tuning knob: REDIST_GATHER=0 disables the gather walk, 2 uses it wherever it applies; the default
-        // (1) keeps it to the cases where it was measured faster than the walk over unit pieces
-        const char *v = std::getenv("REDIST_GATHER");
-        return v ? std::atoi(v) : 1;
-    }();
+    // 0 disables the gather walk, 2 uses it wherever it applies; the default (1) keeps it to the cases
+    // where it was measured faster than the walk over unit pieces
+    const int kGather = int(tune.gather);
     int g_levels = -1;
     i64 g_stretch = 0;
     if (kGather > 0 && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu && (m1[kp] == 1 || m2[kp] == 1)) {
@@ -257,21 +236,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }
     // zip: the same interleaving when the innermost row digit is contiguous on both sides -- the source
     // segments of an item are then long enough for bulk copies into shared memory
-    static const int kZip = [] {
-        // tuning knob: REDIST_ZIP=0 disables the zip kernels, 1 uses them only where the gather walk is
-        // not chosen; the default (2) wherever they apply (measured: within 0.3 % of the best choice per
-        // problem on the odd-shape sweep)
-        const char *v = std::getenv("REDIST_ZIP");
-        return v ? std::atoi(v) : 2;
-    }();
-    static const i64 kZipMinRange = [] {
-        const char *v = std::getenv("REDIST_ZIP_MIN");   // tuning knob: shortest target range of a table row for the zip kernels
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 128);
-    }();
-    static const i64 kZipRun = [] {
-        const char *v = std::getenv("REDIST_ZIP_RUN");   // tuning knob: runs below this many bytes may take the zip kernels
-        return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 2048);
-    }();
+    // 0 disables the zip kernels, 1 uses them only where the gather walk is not chosen; the default (2)
+    // wherever they apply (measured: within 0.3 % of the best choice per problem on the odd-shape sweep)
+    const int kZip = int(tune.zip);
+    const i64 kZipMinRange = 128;         // shortest target range of a table row
+    const i64 kZipRun = 2048;             // runs below this many bytes may take the zip kernels
     // measured: from 2 KiB the plain bulk copy (aligned runs) and the ragged chunk walk are faster
     const bool zip_run_ok = run_bytes < kZipRun;
     i64 zip_n = 0;
@@ -293,11 +262,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const i64 tab_rows = n_rows / zip_n;
         const i64 seg_row = long_dst ? run_bytes : row_bytes;   // bytes of one row in a source segment
         const i64 kTile = 38 * 1024;                            // shared-memory tile of an item, at most
-        static const i64 kZipKb = [] {
-            const char *v = std::getenv("REDIST_ZIP_KB");    // tuning knob: KiB read per zip item
-            return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 0);
-        }();
-        const i64 kZipBytes = kZipKb > 0 ? kZipKb * 1024 : kItemBytes;
+        const i64 kZipBytes = kItemBytes;
         i64 rpb = std::max<i64>(1, std::min<i64>(zip_n, kZipBytes / row_bytes));
         rpb = std::max<i64>(1, std::min<i64>(rpb, (kTile / nseg - 48) / seg_row));
         const i64 ncb = (zip_n + rpb - 1) / rpb;
@@ -328,22 +293,15 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         {
             // periodic walk: a table row must give every thread several chunks, and the period must leave most
             // threads of a block busy
-            static const i64 kZipPeriodic = [] {
-                const char *v = std::getenv("REDIST_ZIP_PERIODIC");   // tuning knob: fewest chunks per table row for the periodic walk (0: never)
-                return i64(v ? std::atoi(v) : 1);
-            }();
+            const i64 kZipPeriodic = (tune.zip_walks & 1) ? 1 : 0;
             const i64 L = long_dst ? row_bytes : run_bytes;         // bytes after which the target pattern repeats, up to alignment
             const i64 gc = std::gcd<i64>(16, L);
             const i64 pc = L / gc;
             G.zip_period = FastDiv{0, 0, 0};
             G.zip_period_rows = 0;
             G.zip_width = 0;
-            static const i64 kZipPc = [] {
-                // tuning knob: longest period, in chunks (the lanes of one block must span it; above 128 the
-                // launch uses 256 threads)
-                const char *v = std::getenv("REDIST_ZIP_PC");
-                return i64(v && std::atoi(v) > 0 ? std::min(std::atoi(v), kBlockThreads - 1) : kBlockThreads - 1);
-            }();
+            // longest period, in chunks (the lanes of one block must span it; above 128 the launch uses 256 threads)
+            const i64 kZipPc = kBlockThreads - 1;
             // (with long source rows of runs up to 16 bytes a thread stays with one of the m target tiles)
             const i64 lanes_needed = !long_dst && run_bytes <= 16 ? pc * m : pc;
             const i64 range_chunks = rpb * L / 16;                  // chunks of one target range, at most
@@ -352,10 +310,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                 G.zip_period_rows = uint32_t(16 / gc);
                 // lanes per table row: about kZipLaneChunks chunks of a range for each, so that the decode of a
                 // lane's first chunk is shared by several chunks while short ranges still fill the block
-                static const i64 kZipLaneChunks = [] {
-                    const char *v = std::getenv("REDIST_ZIP_LANE_CHUNKS");   // tuning knob
-                    return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 4);
-                }();
+                const i64 kZipLaneChunks = 4;
                 const i64 want = std::max<i64>(1, (range_chunks + kZipLaneChunks * pc - 1) / (kZipLaneChunks * pc));
                 G.zip_width = uint32_t(std::min<i64>(want * pc, kBlockThreads / pc * pc));
             }
@@ -364,14 +319,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         // to gain with 16-byte units) the chunk slots of a range are numbered (run, i-th target-aligned chunk
         // that starts in the run) -- such a chunk takes its units from that run and, past its end, from the
         // next one, no division per unit -- and a range with 256 slots or more is walked by the whole block.
-        static const i64 kZipPerRun = [] {
-            const char *v = std::getenv("REDIST_ZIP_PER_RUN");   // tuning knob: shortest run (of 4-byte units) for the by-range walk (0: never)
-            return i64(v ? std::atoi(v) : 32);
-        }();
-        static const i64 kZipByRange = [] {
-            const char *v = std::getenv("REDIST_ZIP_BY_RANGE");   // tuning knob: fewest chunk slots of a range for the by-range walk
-            return i64(v && std::atoi(v) > 0 ? std::atoi(v) : 256);
-        }();
+        const i64 kZipPerRun = (tune.zip_walks & 2) ? 32 : 0;   // shortest run (of 4-byte units) for the by-range walk
+        const i64 kZipByRange = std::max<i64>(1, tune.zip_by_range_slots);
         const i64 cpr = (run_bytes + 15) / 16;
         if (G.zip_period.d == 0 && kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16 &&
             rpb * (long_dst ? m : 1) * cpr >= kZipByRange) {
@@ -384,10 +333,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         {
             // short ranges (neither walk above applies): the place of every unit of a range is tabulated in shared
             // memory; the chunk slots are then numbered flat
-            static const i64 kZipLut = [] {
-                const char *v = std::getenv("REDIST_ZIP_LUT");   // tuning knob: longest range, in units, whose unit places are tabulated (0: never)
-                return i64(v ? std::atoi(v) : 2048);
-            }();
+            const i64 kZipLut = (tune.zip_walks & 4) ? 2048 : 0;   // longest range, in units, whose unit places are tabulated
             const i64 units = rpb * (long_dst ? row_bytes : run_bytes) / vec;
             G.zip_lut_units = 0;
             if (G.zip_period.d == 0 && G.zip_cpr.d == 0 && units <= kZipLut && seg_pitch * nseg * rpi + units * 4 <= 42 * 1024)
@@ -462,10 +408,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             // ragged rows: each row segment is loaded by one bulk copy of the 16-byte blocks that cover
             // it (up to 15 bytes before and after, plus the ragged head), then shifted out of shared memory
             const i64 pitch = cpb * 16 + 64;
-            static const i64 kRaggedKb = [] {
-                const char *v = std::getenv("REDIST_RBULK_KB");   // tuning knob: shared-memory tile of a ragged bulk item, KiB (at most 38)
-                return i64(v && std::atoi(v) > 0 ? std::min(std::atoi(v), 38) : 38);
-            }();
+            const i64 kRaggedKb = 38;      // shared-memory tile of a ragged bulk item, KiB
             rpi = std::max<i64>(1, std::min<i64>(rpi, std::min<i64>(kRaggedBulkRows, kRaggedKb * 1024 / pitch)));
             ragged_bulk = true;
             G.stage_pitch = uint32_t(pitch);
@@ -530,6 +473,14 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         l1 *= a.tile[k];
         l2 *= b.tile[k];
     }
+    G.wait_polls = uint32_t(std::max<i64>(1, std::min<i64>(tune.wait_polls, 1ll << 30)));
+    G.test_extra_tx = uint32_t(std::max<i64>(0, std::min<i64>(tune.test_extra_tx, 1 << 20)));
+    G.n_src_tab = uint32_t(out.src_holder.size());
+    G.n_dst_tab = uint32_t(out.dst_devs.size());
+    // (test_shrink_tiles, test only: the checked build is told shorter tiles, so that the last accesses of
+    // every tile fail their test, are skipped and are counted -- the positive control of that build)
+    G.src_tile_bytes = uint64_t(std::max<i64>(0, l1 * e - tune.test_shrink_tiles));
+    G.dst_tile_bytes = uint64_t(std::max<i64>(0, l2 * e - tune.test_shrink_tiles));
     out.run_bytes = run_bytes;
     out.src_tile_bytes = l1 * e;
     out.dst_tile_bytes = l2 * e;

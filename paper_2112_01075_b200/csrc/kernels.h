@@ -10,14 +10,32 @@ namespace redist {
 constexpr int kSmallTable = 64;     // pointer-table capacity of the small parameter block
 constexpr int kLargeTable = 1024;   // ... of the large one (REDIST_MAX_DEVICES)
 
-// kernel: 0 dynslice, 1 alltoall, 2 allgather, 3 allpermute, 4 copy, 5 fused, 6 naive gather,
-// 7 naive slice.  src_tab / dst_tab are HOST arrays of device pointers (copied into the kernel
-// parameters).  Asynchronous on `stream`.
-cudaError_t launch_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
-                        char *const *dst_tab, int n_dst, int grid, cudaStream_t stream);
+// One kernel launch, ready to go: entry point, launch shape and the complete parameter block (copy
+// descriptor plus both pointer tables).  Plain data, so it can sit on the stack of a call or in a
+// bound plan that is launched again and again.
+struct PreparedLaunch {
+    const void *fn = nullptr;
+    unsigned grid = 0, block = 0;
+    size_t smem = 0;
+    int pdl = 1;
+    alignas(16) unsigned char params[sizeof(CopyParams<kLargeTable>)];
+};
 
-// Work items of the bulk-copy kernel whose bounded wait ran out on the current device (0 in a healthy
+// kernel: 0 dynslice, 1 alltoall, 2 allgather, 3 allpermute, 4 copy, 5 fused, 6 naive gather,
+// 7 naive slice.  src_tab / dst_tab are HOST arrays of device pointers (copied into the parameter
+// block).  Host only; allocates nothing.
+cudaError_t prepare_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
+                         char *const *dst_tab, int n_dst, int pdl, PreparedLaunch &out);
+
+// Asynchronous on `stream`; the parameter block is read during the call.
+cudaError_t launch_prepared(const PreparedLaunch &pl, cudaStream_t stream);
+
+// Work items of the bulk-copy kernels whose bounded wait ran out on the current device (0 in a healthy
 // run).  Synchronizes the device.
 cudaError_t read_bulk_timeouts(unsigned int *out);
+
+// Checked build only: {violations, source line, block, side, distance} of the accesses that failed
+// their bounds test since the last call (and resets the record); cudaErrorNotSupported otherwise.
+cudaError_t read_bounds_report(long long out[5]);
 
 }  // namespace redist

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cstdint>
+#include <memory>
 #include <string>
 #include <vector>
 
@@ -49,6 +50,30 @@ struct Step {
     i64 localsize_after = 0;
 };
 
+// Tuning values, copied into a plan when it is created (redist_tuning_set changes the values later
+// plans get).  Defaults are the measured optima; the tests use them to force the kernel variants that
+// the default choice seldom leaves work for, the benchmark to show what a choice is worth.
+struct Tuning {
+    int64_t bulk = 1;                 // 0: no TMA bulk copies at all (register kernels only)
+    int64_t gather = 1;               // gather walk: 0 never, 1 where measured faster, 2 wherever it applies
+    int64_t zip = 2;                  // zip kernels: 0 never, 1 only where the gather walk is not chosen, 2 wherever they apply
+    int64_t zip_walks = 7;            // chunk -> units maps the zip kernels may use: 1 periodic, 2 by range, 4 tabulated
+    int64_t zip_by_range_slots = 256; // fewest chunk slots of a range for the by-range walk
+    int64_t item_kb = 0;              // KiB read per work item (0: 32 / 16 / 8 by fan-out, bulk copies 20 / 12 / 6)
+    int64_t pdl = 1;                  // 0: plain stream order instead of programmatic dependent launch
+    int64_t step_latency = 0;         // elements added to the cost of every collective when searching (Section 8, RQ3)
+    int64_t wait_polls = 1 << 18;     // mbarrier polls before a bulk-copy block gives up
+    int64_t test_extra_tx = 0;        // test only, see CopyGeometry::test_extra_tx
+    int64_t test_shrink_tiles = 0;    // test only: bytes by which the checked build believes every tile to be shorter
+    bool operator==(const Tuning &o) const
+    {
+        return bulk == o.bulk && gather == o.gather && zip == o.zip && zip_walks == o.zip_walks &&
+               zip_by_range_slots == o.zip_by_range_slots && item_kb == o.item_kb && pdl == o.pdl &&
+               step_latency == o.step_latency && wait_polls == o.wait_polls && test_extra_tx == o.test_extra_tx &&
+               test_shrink_tiles == o.test_shrink_tiles;
+    }
+};
+
 enum BufKind { BUF_SRC = 0, BUF_DST = 1, BUF_SCRATCH0 = 2, BUF_SCRATCH1 = 3, BUF_GLOBAL = 4 };
 
 struct Launch {
@@ -64,6 +89,7 @@ struct Launch {
 struct Plan {
     int n_mesh_axes = 0, rank = 0, elem_bytes = 0, n_devices = 0;
     uint32_t flags = 0;
+    Tuning tuning;
     std::vector<i64> mesh_shape, global_shape;
     std::vector<std::vector<int>> src_axes, dst_axes;      // original axes
     std::vector<PrimeAxis> primes;
@@ -81,15 +107,24 @@ struct Plan {
 
 }  // namespace redist
 
-// The opaque handle of the C boundary.
+// The opaque handle of the C boundary: a reference to an immutable plan, which the plan cache and
+// any number of handles may share.
 struct redist_plan_s {
-    redist::Plan p;
+    std::shared_ptr<const redist::Plan> ref;
+    const redist::Plan &p;
+    explicit redist_plan_s(std::shared_ptr<const redist::Plan> r) : ref(std::move(r)), p(*ref) {}
 };
 
 namespace redist {
 
 // api.cu: last CUDA error seen by the calling thread inside the library
 extern thread_local int tl_cuda_error;
+
+// api.cu: buffer checks (alignment; destination tiles and the `scratch_range` bytes at `scratch` disjoint
+// from each other and from every source), then the plan's kernel launches on the stream.  Shared by
+// every execute entry point; allocates nothing.
+redist_status run_plan(const Plan &p, const void *const *src_shards, void *const *dst_shards, void *scratch,
+                       size_t scratch_range, void *cuda_stream);
 
 // planner.cpp
 redist_status synthesize(Plan &p);

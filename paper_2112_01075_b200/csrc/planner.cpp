@@ -66,8 +66,12 @@ struct Search {
     std::vector<int> tgt_exps;     // target exponents [r*np]
 
     bool allow_over = false;       // ignore REDIST_NO_OVERPARTITION (fallback when it leaves no path)
+    i64 lat;                       // per-step latency, in elements, added to every edge weight: the cost
+                                   // model of Section 6.2 counts bytes only, while small transfers are bound
+                                   // by the latency of each collective (Section 8, third research question);
+                                   // 0 = the paper's weights
 
-    explicit Search(const Plan &plan) : p(plan), r(plan.rank), np(0), M(0) {}
+    explicit Search(const Plan &plan) : p(plan), r(plan.rank), np(0), M(0), lat(std::max<i64>(0, plan.tuning.step_latency)) {}
 
     i64 pow_of(const std::vector<int> &e) const
     {
@@ -149,7 +153,7 @@ struct Search {
                         }
                     Key nk = key;
                     for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] + e[q]);
-                    relax(nk, 0, WeakStep{REDIST_STEP_DYNSLICE, i, -1, e, m});
+                    relax(nk, lat, WeakStep{REDIST_STEP_DYNSLICE, i, -1, e, m});
                 });
         }
         // alltoall(i -> j, m): m from the primes on dim i, m | c_j, weight localsize (phases 0, 1)
@@ -168,7 +172,7 @@ struct Search {
                             nk[j * np + q] = uint8_t(nk[j * np + q] + e[q]);
                         }
                         nk[r * np] = 1;
-                        relax(nk, L, WeakStep{REDIST_STEP_ALLTOALL, i, j, e, m});
+                        relax(nk, L + lat, WeakStep{REDIST_STEP_ALLTOALL, i, j, e, m});
                     });
                 }
             }
@@ -183,7 +187,7 @@ struct Search {
                 Key nk = key;
                 for (int q = 0; q < np; ++q) nk[i * np + q] = uint8_t(nk[i * np + q] - e[q]);
                 nk[r * np] = 2;
-                relax(nk, L * m, WeakStep{REDIST_STEP_ALLGATHER, i, -1, e, m});
+                relax(nk, L * m + lat, WeakStep{REDIST_STEP_ALLGATHER, i, -1, e, m});
             });
         }
     }
@@ -298,9 +302,9 @@ struct Search {
     }
     // Sequences of weak cost strictly below `bound` and of at most `max_steps` steps, those with the
     // cheapest continuation first, at most `max_paths` of them.  The search of Section 7.3 leaves the
-    // final permutation out of the edge weights ("not a graph edge"), so a sequence that is not a
-    // shortest path can still be the cheaper plan once its permutation -- or the lack of one -- is
-    // counted.  Call after run().
+    // final permutation out of the edge weights, so a sequence that is not a shortest path can still be
+    // the cheaper plan once its permutation -- or the lack of one -- is counted.  Weights and `bound`
+    // include the per-step latency.  Call after run().
     void near(i64 bound, int max_steps, size_t max_paths, std::vector<std::vector<WeakStep>> &paths) const
     {
         using Key = std::vector<uint8_t>;
@@ -833,23 +837,27 @@ redist_status synthesize(Plan &p)
     //    of the plan found so far, and keep the cheapest total (then the fewest steps)
     if (p.flags & REDIST_COST_PERMUTE) {
         std::vector<std::vector<WeakStep>> near;
-        S.near(p.cost, int(steps.size()) + 3, 256, near);
+        const i64 lat = S.lat;
+        i64 best_total = p.cost + lat * i64(steps.size());       // every collective of the plan pays the latency
+        S.near(best_total, int(steps.size()) + 3, 256, near);
         for (const auto &cand : near) {
             i64 weak = 0;
             std::vector<Step> st;
             ConcreteState e;
             if (!L.lower(cand, st, e)) continue;
             for (const Step &s : st)
-                weak += s.kind == REDIST_STEP_DYNSLICE    ? 0
-                        : s.kind == REDIST_STEP_ALLGATHER ? product(s.local_after)
-                                                          : product(s.local_before);
-            if (weak >= p.cost) continue;
+                weak += lat + (s.kind == REDIST_STEP_DYNSLICE    ? 0
+                               : s.kind == REDIST_STEP_ALLGATHER ? product(s.local_after)
+                                                                 : product(s.local_before));
+            if (weak >= best_total) continue;
             i64 cost = 0, height = 0;
             if (finish(st, e, cost, height) != REDIST_OK) continue;
-            if (cost < p.cost || (cost == p.cost && st.size() < steps.size())) {
+            const i64 total = cost + lat * i64(st.size());
+            if (total < best_total || (total == best_total && st.size() < steps.size())) {
                 steps = st;
                 p.cost = cost;
                 p.height = height;
+                best_total = total;
             }
         }
     }

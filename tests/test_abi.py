@@ -66,6 +66,30 @@ def test_execute_rejects_bad_buffers_before_touching_the_gpu():
         assert e.value.status == 5                  # scratch missing
 
 
+def test_every_tensor_entry_point_checks_its_tiles_before_the_foreign_call():
+    """execute, execute_static and execute_host share one check: a wrong number of tiles, a tile of the
+    wrong size, a non-contiguous tile or a tile in the wrong memory is refused with EINVAL before the
+    library sees a pointer (the C entry points cannot know how large the caller's buffers are)."""
+    import pytest
+    torch = pytest.importorskip("torch")
+    p = api.Plan((2,), ((8, 8), ((0,), ())), ((8, 8), ((), (0,))), 4, api.FUSE_NONE)
+    good = [torch.zeros(128, dtype=torch.uint8) for _ in range(2)]
+    short = [torch.zeros(112, dtype=torch.uint8), good[1]]
+    strided = [torch.zeros(256, dtype=torch.uint8)[::2], good[1]]
+    for call in (p.execute, p.execute_static):
+        for s, d in ((good[:1], good), (good, good + good), (short, good), (good, short), (strided, good), (good, good)):
+            with pytest.raises(api.RedistError) as e:
+                call(s, d)                      # the last pair is well-shaped but lives in host memory
+            assert e.value.status == 1
+    for s, d in ((good[:1], good), (short, good), (good, strided)):
+        with pytest.raises(api.RedistError) as e:
+            p.execute_host(s, d, None, None)
+        assert e.value.status == 1
+    with pytest.raises(api.RedistError) as e:
+        p.bind([4096], [8192, 12288])
+    assert e.value.status == 1
+
+
 def test_pretty_prints_the_sequence_in_the_papers_notation():
     p = api.Plan((4, 2), ((8, 2048, 4096), ((0,), (), (1,))), ((8, 2048, 4096), ((), (0, 1), ())), 2)
     text = p.pretty(("x", "y"))

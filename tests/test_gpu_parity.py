@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 from paper_2112_01075_b200 import api, workloads as wl
+from _buffers import Carved
 from _plancheck import types_of
 
 torch = pytest.importorskip("torch")
@@ -17,18 +18,23 @@ MODES = [api.FUSE_ADJACENT, api.FUSE_NONE, api.FUSE_ALL, api.NAIVE]
 MODE_NAMES = {0: "adjacent", 1: "unfused", 2: "all", 3: "naive"}
 
 
-def run_gpu(mesh, src, dst, e, src_tiles, flags=api.FUSE_ADJACENT, stream=None):
+def run_gpu(mesh, src, dst, e, src_tiles, flags=api.FUSE_ADJACENT, stream=None, bound=False):
+    """Plan and execute on tiles carved out of one canary-filled buffer (tiles aligned to 16 bytes and no
+    better, sources packed, guard bands around every destination tile and the scratch); afterwards every
+    guard byte must be intact and the sources unchanged.  `bound`: through redist_bind /
+    redist_bound_execute instead of redist_execute."""
     plan = api.Plan(mesh, src, dst, e, flags)
-    dev_src = [torch.from_numpy(np.ascontiguousarray(t)).cuda() for t in src_tiles]
-    nbytes = plan.local_elems(1) * e
-    dev_dst = [torch.full((nbytes,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
-    scratch = plan.alloc_scratch()
-    if scratch is not None:
-        scratch.fill_(0xDD)
-    plan.execute(dev_src, dev_dst, scratch, stream)
+    mem = Carved(torch, src_tiles, plan.n_devices, plan.local_elems(1) * e, plan.scratch_bytes)
+    if bound:
+        s = stream if stream is not None else torch.cuda.current_stream()
+        call = plan.bind([t.data_ptr() for t in mem.src], [t.data_ptr() for t in mem.dst],
+                         mem.scratch.data_ptr() if mem.scratch is not None else 0, plan.scratch_bytes)
+        call(s.cuda_stream)
+    else:
+        plan.execute(mem.src, mem.dst, mem.scratch, stream)
     torch.cuda.synchronize()
-    out = [t.cpu().numpy() for t in dev_dst]
-    return plan, out
+    mem.check(f"{mesh} {src} -> {dst} e={e} flags={flags}")
+    return plan, mem.results()
 
 
 def assert_same(got, want, what=""):
@@ -118,7 +124,7 @@ def random_problems_small_and_odd(n_problems, extra_flags=0):
         src_tiles = oracle.reslice(mesh, src, G)
         want = oracle.redistribute(mesh, src, dst, src_tiles)
         mode = MODES[t % 4] | extra_flags
-        plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
+        plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode, bound=(t // 4) % 2 == 1)
         n_multi += plan.num_launches >= 3
         variants.update(plan.launch_info(q).variant for q in range(plan.num_launches))
         assert_same(got, want, f"{mesh} {src} -> {dst} e={e} mode={mode}")
@@ -137,42 +143,33 @@ def test_random_problems_with_the_permutation_counted():
     random_problems_small_and_odd(300, api.COST_PERMUTE)
 
 
-def _random_problems_in_a_fresh_process(env, n_problems, expect):
-    import os
-    import subprocess
-    import sys
-    here = os.path.dirname(os.path.abspath(__file__))
-    code = ("import sys; sys.path[:0] = [%r, %r]\n"
-            "from test_gpu_parity import random_problems_small_and_odd\n"
-            "v = random_problems_small_and_odd(%d)\n"
-            "assert %s, v\n" % (here, os.path.dirname(here), n_problems, expect))
-    res = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, **env), capture_output=True,
-                         text=True, timeout=600)
-    assert res.returncode == 0, res.stderr[-2000:]
+def test_register_kernels_behind_the_tuning_values():
+    """With the bulk-copy kernels (zip included) and the gather walk switched off the same problems run
+    on the plain register kernels."""
+    with api.tuning(bulk=0, gather=0):
+        v = random_problems_small_and_odd(300)
+    assert v == {0, 1, 2, 3}, v
 
 
-def test_register_kernels_behind_the_tuning_knobs():
-    """With the bulk-copy kernels (zip included) and the gather walk switched off (environment read when
-    the library first builds a launch, hence a fresh process) the same problems run on the plain
-    register kernels."""
-    _random_problems_in_a_fresh_process({"REDIST_BULK": "0", "REDIST_GATHER": "0"}, 300, "v == {0, 1, 2, 3}")
-
-
-@pytest.mark.parametrize("env", [
-    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_LUT": "0", "REDIST_ZIP_PER_RUN": "0"},     # flat walk only
-    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_LUT": "0", "REDIST_ZIP_BY_RANGE": "1"},    # by-range walk, else flat
-    {"REDIST_ZIP_PERIODIC": "0", "REDIST_ZIP_PER_RUN": "0"},                            # tabulated places, else flat
+@pytest.mark.parametrize("values", [
+    {"zip_walks": 0},                               # flat walk only
+    {"zip_walks": 2, "zip_by_range_slots": 1},      # by-range walk, else flat
+    {"zip_walks": 4},                               # tabulated places, else flat
 ], ids=["flat", "by_range", "tabulated"])
-def test_zip_kernels_with_each_chunk_map(env):
-    """The zip kernels pick one of several ways to map a target chunk to its units; the knobs force the
-    ones that the default choice (periodic walk) seldom leaves work for."""
-    _random_problems_in_a_fresh_process(env, 400, "7 in v")
+def test_zip_kernels_with_each_chunk_map(values):
+    """The zip kernels pick one of several ways to map a target chunk to its units; the tuning values
+    force the ones that the default choice (periodic walk) seldom leaves work for."""
+    with api.tuning(**values):
+        v = random_problems_small_and_odd(400)
+    assert 7 in v, v
 
 
 def test_gather_walk_wherever_it_applies():
-    """REDIST_GATHER=2 sends every eligible launch through the gather walk, including long source rows
-    that are scattered into several target tiles and 16-byte units (not chosen by default)."""
-    _random_problems_in_a_fresh_process({"REDIST_GATHER": "2", "REDIST_ZIP": "0"}, 600, "5 in v and 7 not in v")
+    """gather = 2 sends every eligible launch through the gather walk, including long source rows that
+    are scattered into several target tiles and 16-byte units (not chosen by default)."""
+    with api.tuning(gather=2, zip=0):
+        v = random_problems_small_and_odd(600)
+    assert 5 in v and 7 not in v, v
 
 
 def test_round_trip_on_the_gpu():
@@ -332,11 +329,28 @@ def test_evaluation_like_problems_full_size(name):
     torch.cuda.empty_cache()
 
 
+_C4 = {}
+
+
+def config4_global():
+    """The 4 GiB global array of the random sweep, generated once for the tests that need it."""
+    if "G" not in _C4:
+        _C4["G"] = wl.global_array_bytes(wl.CONFIG4_SHAPE, 4, "random_bits", wl.CONFIG4_FILL_SEED)
+    return _C4["G"]
+
+
+def launch_class(plan):
+    """What decides which kernel code runs on what shape of work: the variant of every launch, the
+    largest fan-out, the number of launches and the shortest contiguous run."""
+    li = [plan.launch_info(q) for q in range(plan.num_launches)]
+    return (tuple(i.variant for i in li), max(i.fanout for i in li), plan.num_launches, min(i.run_bytes for i in li))
+
+
 def test_random_sweep_full_size_samples():
-    """Three pairs of the sweep at the full [64,128,256,512] f32 shape (4 GiB global), chosen by
-    device footprint; all target tiles compared."""
+    """Three multi-step pairs of the sweep at the full [64,128,256,512] f32 shape (4 GiB global), chosen by
+    device footprint; every target tile compared with the oracle's."""
     pairs = wl.config4()
-    G = wl.global_array_bytes(wl.CONFIG4_SHAPE, 4, "random_bits", wl.CONFIG4_FILL_SEED)
+    G = config4_global()
     oracle.set_threads(oracle.max_threads())
     done = 0
     try:
@@ -356,6 +370,62 @@ def test_random_sweep_full_size_samples():
     finally:
         oracle.set_threads(1)
     assert done == 3
+
+
+def test_random_sweep_full_size_every_launch_class():
+    """The sweep at full size in the launch configuration the benchmark times, one pair for every class
+    of launch (kernel variant, fan-out, launches, shortest run) that occurs among the 100 pairs.  The
+    global array goes to the device once; source tiles are cut from it at the oracle's base offsets
+    (replicas share one buffer, as in the benchmark); every target tile is compared on the device with
+    the block of the global array at the oracle's base offset for that device -- the definition of the
+    result -- and the first and last device's tiles also on the host with the oracle's own tile."""
+    pairs = wl.config4()
+    classes = {}
+    for i, w in enumerate(pairs):
+        src, dst = types_of(w)
+        classes.setdefault(launch_class(api.Plan(w.mesh_shape, src, dst, 4)), i)
+    assert len(classes) >= 20
+    G = config4_global()
+    Gd = torch.from_numpy(G).cuda()
+
+    def cut(off, tile):
+        t = Gd
+        for k, (o, c) in enumerate(zip(off, tile)):
+            t = t.narrow(k, int(o), int(c))
+        return t
+
+    ran = set()
+    for key, i in sorted(classes.items()):
+        w = pairs[i]
+        src, dst = types_of(w)
+        plan = api.Plan(w.mesh_shape, src, dst, 4)
+        n = plan.n_devices
+        tile_s, off_s = oracle.base_offsets(w.mesh_shape, src)
+        tile_d, off_d = oracle.base_offsets(w.mesh_shape, dst)
+        owned, dev_src = {}, []
+        for d in range(n):
+            k = tuple(int(o) for o in off_s[d])
+            if k not in owned:
+                owned[k] = cut(k, tile_s).contiguous().reshape(-1)
+            dev_src.append(owned[k])
+        nb = plan.local_elems(1) * 4
+        dev_dst = [torch.full((nb,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(n)]
+        plan.execute(dev_src, dev_dst, plan.alloc_scratch())
+        torch.cuda.synchronize()
+        assert launch_class(plan) == key
+        for d in range(n):
+            want = cut(off_d[d], tile_d)
+            assert torch.equal(dev_dst[d].view(tuple(tile_d) + (4,)), want), f"{w.name}: device {d} differs"
+        for d in (0, n - 1):
+            want = oracle.tile_of(w.mesh_shape, dst, G, d)
+            assert np.array_equal(dev_dst[d].cpu().numpy().reshape(want.shape), want), f"{w.name}: device {d} (host)"
+        ran.add(key)
+        del dev_src, dev_dst, owned
+        torch.cuda.empty_cache()
+    assert ran == set(classes)        # every class present among the 100 pairs ran at full size
+    del Gd
+    _C4.clear()
+    torch.cuda.empty_cache()
 
 
 def test_execute_can_be_captured_in_a_cuda_graph_and_replayed():

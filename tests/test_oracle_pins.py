@@ -142,6 +142,8 @@ def test_brute_force_ownership_and_result(mesh):
         for d in range(len(want)):
             assert got[d].shape == want[d].shape
             assert np.array_equal(got[d], want[d]), (mesh, gshape, a1, a2, d)
+            # the one-tile form (used where all tiles do not fit in host memory at once)
+            assert np.array_equal(oracle.tile_of(mesh, (gshape, a2), G, d), want[d])
         # ownership: every global element lies in the tile of exactly N/#tiles devices
         tile, off = oracle.base_offsets(mesh, (gshape, a1))
         count = np.zeros(gshape, dtype=np.int64)

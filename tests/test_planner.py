@@ -234,7 +234,7 @@ def test_error_statuses():
         api.Plan((2048,), ((4096,), ((0,),)), ((4096,), ((),)), 4)
     assert e.value.status == 10                                 # more virtual devices than supported
     with pytest.raises(api.RedistError) as e:
-        api.Plan((2,), ((4,), ((0,),)), ((4,), ((),)), 4, flags=64)
+        api.Plan((2,), ((4,), ((0,),)), ((4,), ((),)), 4, flags=128)
     assert e.value.status == 1
 
 
@@ -264,9 +264,11 @@ def all_strong_types(mesh, gshape):
     return out
 
 
-def brute_force_optimum(mesh, gshape, a1, a2):
+def brute_force_optimum(mesh, gshape, a1, a2, lat=0, count_permute=True):
     """Dijkstra over strong types with the four typing rules (multi-axes forms included) and
-    localsize <= M; returns the minimal cost of a memory-constrained sequence."""
+    localsize <= M; returns the minimal cost of a memory-constrained sequence.  `lat` is added to every
+    dynslice / alltoall / allgather; with `count_permute` off an allpermute is free (the view of the
+    search of Section 7.3, which leaves the permutation out of the edge weights)."""
     M = max(C.localsize(mesh, gshape, a1), C.localsize(mesh, gshape, a2))
     nodes = [t for t in all_strong_types(mesh, gshape) if C.localsize(mesh, gshape, t) <= M]
     by_local = {}
@@ -286,22 +288,22 @@ def brute_force_optimum(mesh, gshape, a1, a2):
         L = C.localsize(mesh, gshape, t)
         for u in by_local[C.localtype(mesh, gshape, t)]:
             if u != t:
-                nxt.append((u, L))
+                nxt.append((u, L if count_permute else 0))
         unused = [a for a in range(len(mesh)) if a not in C.used_axes(t)]
         for i in range(rank):
             for n_ax in range(1, len(t[i]) + 1):
                 u = C.t_allgather(mesh, gshape, t, i, n_ax)
-                nxt.append((u, C.localsize(mesh, gshape, u)))
+                nxt.append((u, C.localsize(mesh, gshape, u) + lat))
                 for j in range(rank):
                     if j != i:
                         try:
-                            nxt.append((C.t_alltoall(mesh, gshape, t, i, j, n_ax), L))
+                            nxt.append((C.t_alltoall(mesh, gshape, t, i, j, n_ax), L + lat))
                         except C.TypeError_:
                             pass
             for k in range(1, len(unused) + 1):
                 for seq in itertools.permutations(unused, k):
                     try:
-                        nxt.append((C.t_dynslice(mesh, gshape, t, i, seq), 0))
+                        nxt.append((C.t_dynslice(mesh, gshape, t, i, seq), lat))
                     except C.TypeError_:
                         pass
         for u, w in nxt:
@@ -371,19 +373,121 @@ def test_counting_the_permutation_on_evaluation_shaped_problems():
 
 def test_planner_throughput_on_evaluation_shaped_problems():
     """Section 8 reports synthesis in under a second per problem (unoptimised Python); the host planner
-    here must stay far below that on 300 problems of the same shape (3 mesh axes, up to 6-D)."""
+    here must stay far below that on 1000 problems of the same shape (3 mesh axes, up to 6-D), synthesized
+    afresh (REDIST_NO_CACHE); asked for again, every one of them comes out of the plan cache."""
     import time
-    ws = wl.evaluation_like_problems(300)
+    ws = wl.evaluation_like_problems(1000)
     worst, t0 = 0.0, time.perf_counter()
+    costs = []
     for w in ws:
         t1 = time.perf_counter()
-        p = api.Plan(w.mesh_shape, w.src, w.dst, 4)
+        p = api.Plan(w.mesh_shape, w.src, w.dst, 4, api.NO_CACHE)
         worst = max(worst, time.perf_counter() - t1)
         assert p.height <= max(p.local_elems(0), p.local_elems(1))
         assert p.step_kinds().count("allpermute") <= 1
+        costs.append(p.cost)
         p.close()
     total = time.perf_counter() - t0
     assert worst < 0.25 and total / len(ws) < 0.05, (worst, total)
+    # the cache holds the 256 most recent plans: the last 200 problems, planned twice, hit the second time
+    api.plan_cache_clear()
+    recent = ws[-200:]
+    for w in recent:
+        api.Plan(w.mesh_shape, w.src, w.dst, 4).close()
+    t0 = time.perf_counter()
+    for w, c in zip(recent, costs[-200:]):
+        p = api.Plan(w.mesh_shape, w.src, w.dst, 4)
+        assert p.cost == c
+        p.close()
+    again = time.perf_counter() - t0
+    hits, misses, entries = api.plan_cache_stats()
+    assert (hits, misses, entries) == (200, 200, 200)
+    assert again / 200 < total / len(ws)          # a hit costs less than a synthesis
+
+
+def test_plan_cache_returns_the_same_plan_for_the_same_request():
+    api.plan_cache_clear()
+    mesh, src, dst = (4, 2), ((8, 64, 64), ((0,), (), (1,))), ((8, 64, 64), ((), (0, 1), ()))
+    p1 = api.Plan(mesh, src, dst, 2)
+    assert api.plan_cache_stats() == (0, 1, 1)
+    p2 = api.Plan(mesh, src, dst, 2)
+    assert api.plan_cache_stats() == (1, 1, 1)
+    assert p1.describe() == p2.describe()
+    p3 = api.Plan(mesh, src, dst, 2, api.NO_CACHE)                  # synthesized afresh, cache untouched
+    assert api.plan_cache_stats() == (1, 1, 1) and p3.describe() == p1.describe()
+    assert api.Plan(mesh, src, dst, 4).elem_bytes == 4 and api.plan_cache_stats() == (1, 2, 2)   # other element size
+    assert api.Plan(mesh, src, dst, 2, api.FUSE_NONE).num_launches == 2 and api.plan_cache_stats() == (1, 3, 3)
+    with api.tuning(bulk=0):                                         # other tuning values: another plan
+        p4 = api.Plan(mesh, src, dst, 2)
+    assert api.plan_cache_stats() == (1, 4, 4)
+    assert p4.launch_info(0).variant != p1.launch_info(0).variant
+    p1.close()                                                       # a handle is a reference: the others stay valid
+    assert p2.step_kinds() == ["alltoall", "alltoall"] and p2.describe()["cost"] == p3.cost
+    rng = np.random.default_rng(3)
+    for _ in range(300):                                             # more distinct requests than the cache keeps
+        g = tuple(int(v) * 4 for v in rng.integers(1, 50, size=2))
+        api.Plan((2, 2), (g, ((0,), (1,))), (g, ((1,), (0,))), 4).close()
+    assert api.plan_cache_stats()[2] <= 256
+    api.plan_cache_clear()
+    assert api.plan_cache_stats() == (0, 0, 0)
+
+
+def test_tuning_values_are_validated_and_copied_into_new_plans_only():
+    mesh, src, dst = (2,), ((64, 2048), ((0,), ())), ((64, 2048), ((), (0,)))      # aligned 4 KiB runs
+    before = api.Plan(mesh, src, dst, 4, api.NO_CACHE)
+    assert api.tuning_get("bulk") == 1
+    with pytest.raises(api.RedistError):
+        api.tuning_set("no_such_value", 1)
+    with pytest.raises(api.RedistError):
+        api.tuning_set("gather", 3)
+    with api.tuning(bulk=0):
+        assert api.tuning_get("bulk") == 0
+        inside = api.Plan(mesh, src, dst, 4, api.NO_CACHE)
+    assert api.tuning_get("bulk") == 1
+    assert before.launch_info(0).variant == 4 and inside.launch_info(0).variant in (0, 1)
+    assert api.Plan(mesh, src, dst, 4, api.NO_CACHE).launch_info(0).variant == 4
+
+
+@pytest.mark.parametrize("mesh", [(2, 2), (2, 3), (2, 2, 2), (2, 2, 3)])
+def test_step_latency_buys_fewer_collectives(mesh):
+    """Small transfers are bound by the latency of each collective, not by bytes (Section 8, third research
+    question).  With the tuning value step_latency = 0 the plan is the default one; with a latency far
+    above any byte cost the searched part of the plan (everything but the final permutation, which the
+    search of Section 7.3 never weighs) has the fewest collectives any memory-constrained sequence can
+    have, and among those the fewest bytes -- checked against a brute-force search over strong types.
+    Every plan is still replayed step by step against the typing rules and the oracle."""
+    big = 10 ** 9
+    rng = np.random.default_rng(len(mesh) * 11 + mesh[-1])
+    fewer = 0
+    for _ in range(10):
+        src, dst = random_problem(rng, mesh, max_rank=2, mult=2)
+        d0 = check_plan(mesh, src, dst, 4)
+        with api.tuning(step_latency=0):
+            assert check_plan(mesh, src, dst, 4)["steps"] == d0["steps"]
+        with api.tuning(step_latency=big):
+            d1 = check_plan(mesh, src, dst, 4)
+        searched = [s for s in d1["steps"] if s["kind"] != "allpermute"]
+        opt = brute_force_optimum(mesh, src[0], src[1], dst[1], lat=big, count_permute=False)
+        assert len(searched) == opt // big, (mesh, src, dst)
+        assert sum(s["cost"] for s in searched) == opt % big, (mesh, src, dst)
+        n0 = len([s for s in d0["steps"] if s["kind"] != "allpermute"])
+        assert len(searched) <= n0
+        fewer += len(searched) < n0
+    return fewer
+
+
+def test_step_latency_example():
+    """The over-partitioning example of Section 7.2 on the mesh {x:4, y:2, z:4}: by bytes the cheapest
+    sequence slices over the idle axis first, moves a quarter of the data and gathers at the end (cost
+    384, four collectives); when every collective costs a large latency the two plain alltoalls of the
+    figure's left column win (cost 512, two collectives)."""
+    mesh, g = (4, 2, 4), (8, 8, 8, 4)
+    src, dst = (g, ((1, 0), (), (), ())), (g, ((), (1,), (0,), ()))
+    d0 = check_plan(mesh, src, dst, 4)
+    with api.tuning(step_latency=10 ** 12):
+        d1 = check_plan(mesh, src, dst, 4)
+    assert ([s["kind"] for s in d0["steps"]], d0["cost"]) == (["dynslice", "alltoall", "allpermute", "allgather"], 384)
+    assert ([s["kind"] for s in d1["steps"]], d1["cost"]) == (["alltoall", "alltoall"], 512)
 
 
 def test_no_overpartition_flag_only_filters_the_axes_it_slices():
