@@ -313,6 +313,24 @@ size_t redist_plan_describe(const redist_plan_t *plan, char *buf, size_t cap);
 redist_status redist_base_offsets(int32_t n_mesh_axes, const int64_t *mesh_shape, const redist_type *type,
                                   int64_t *out_tile, int64_t *out_offsets);
 
+/*
+ * redist_plan_gpu_split -- byte accounting for running the plan with its virtual devices spread over
+ * several GPUs (host only; nothing in this library moves data between GPUs).  The paper executes its
+ * collectives between real devices (Section 8) and discusses individual device-to-device transfers
+ * derived from the base offset maps as the alternative (Section 9); this is that derivation for one
+ * launch.  Virtual device d is placed on GPU d / (N / n_gpus): the leading mesh coordinates choose the
+ * GPU, so n_gpus must be the product of the leading mesh axis sizes times a divisor of the next one.
+ *
+ *   launch          index of a kernel launch of the plan (redist_plan_num_launches)
+ *   bytes           host; receives n_gpus * n_gpus numbers, row-major: bytes[s * n_gpus + t] = bytes that
+ *                   GPU s reads from tiles it holds and writes into tiles that live on GPU t (a replicated
+ *                   source tile is read on the receiving GPU when that GPU holds a replica, else from the
+ *                   lowest-numbered holder).  The diagonal stays inside a GPU; the sum over the matrix is
+ *                   the launch's bytes_written; with n_gpus = 1 it is that single number.
+ * Errors: EINVAL (also for an n_gpus that is no prefix of the mesh), ENOMEM.
+ */
+redist_status redist_plan_gpu_split(const redist_plan_t *plan, int32_t n_gpus, int32_t launch, int64_t *bytes);
+
 const char *redist_status_string(redist_status status);
 
 /* The last CUDA error code (cudaError_t as int) seen by the calling thread inside this library. */

@@ -34,6 +34,7 @@ EXPORTS = (
     "redist_bind", "redist_bound_execute", "redist_bound_destroy",
     "redist_plan_cache_stats", "redist_plan_cache_clear",
     "redist_tuning_set", "redist_tuning_get", "redist_tuning_reset", "redist_debug_bounds_report",
+    "redist_plan_gpu_split",
     "redist_plan_num_devices", "redist_plan_rank", "redist_plan_local_elems", "redist_plan_scratch_bytes",
     "redist_plan_scratch_bytes_per_device", "redist_plan_staging_bytes", "redist_plan_alignment",
     "redist_plan_height", "redist_plan_cost", "redist_plan_num_steps", "redist_plan_num_launches",
@@ -134,6 +135,8 @@ def load() -> ctypes.CDLL:
     lib.redist_tuning_get.restype = i32
     lib.redist_tuning_reset.argtypes = []
     lib.redist_tuning_reset.restype = None
+    lib.redist_plan_gpu_split.argtypes = [vp, i32, i32, ctypes.POINTER(i64)]
+    lib.redist_plan_gpu_split.restype = i32
     lib.redist_debug_bounds_report.argtypes = [ctypes.POINTER(i64)]
     lib.redist_debug_bounds_report.restype = i32
     _lib = lib
@@ -276,6 +279,15 @@ class Plan:
         """(read, written) HBM bytes summed over the launches."""
         infos = [self.launch_info(q) for q in range(self.num_launches)]
         return sum(i.bytes_read for i in infos), sum(i.bytes_written for i in infos)
+
+    def gpu_split(self, n_gpus: int, launch: int):
+        """``redist_plan_gpu_split``: ``m[s][t]`` = bytes GPU ``s`` would read locally and write to GPU ``t``
+        if the virtual devices were spread over ``n_gpus`` GPUs by a prefix of the mesh axes."""
+        out = (ctypes.c_int64 * (n_gpus * n_gpus))()
+        rc = self._lib.redist_plan_gpu_split(self._h, n_gpus, launch, out)
+        if rc:
+            raise RedistError(rc, "redist_plan_gpu_split")
+        return [[int(out[s * n_gpus + t]) for t in range(n_gpus)] for s in range(n_gpus)]
 
     def describe(self) -> dict:
         n = self._lib.redist_plan_describe(self._h, None, 0)

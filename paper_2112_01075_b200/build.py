@@ -24,7 +24,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_obj")
 LIB = os.path.join(HERE, "libredist_b200.so")
 LIB_BOUNDS = os.path.join(HERE, "libredist_b200_bounds.so")
-SOURCES = ["api.cu", "kernels.cu", "static_scratch.cu", "planner.cpp", "descriptor.cpp", "describe.cpp"]
+SOURCES = ["api.cu", "kernels.cu", "static_scratch.cu", "planner.cpp", "descriptor.cpp", "describe.cpp", "multi_gpu.cpp"]
 HEADERS = ["plan.hpp", "copy_params.h", "kernels.h"]
 CHECKED = ["kernels.cu"]          # sources that differ in the checked build
 

@@ -447,7 +447,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     }
     const int N = p.n_devices;
     out.src_holder.assign(size_t(nt1), -1);
+    out.src_tile_of.assign(size_t(N), -1);
     if (!a.shared_global) {
+        for (int d = 0; d < N; ++d) out.src_tile_of[d] = a.tile_of[d];
         for (int d = N - 1; d >= 0; --d) out.src_holder[a.tile_of[d]] = d;   // lowest id holding the tile
         for (int32_t h : out.src_holder)
             if (h < 0) return REDIST_EINTERNAL;
@@ -482,6 +484,8 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     G.src_tile_bytes = uint64_t(std::max<i64>(0, l1 * e - tune.test_shrink_tiles));
     G.dst_tile_bytes = uint64_t(std::max<i64>(0, l2 * e - tune.test_shrink_tiles));
     out.run_bytes = run_bytes;
+    out.src_tile = a.tile;
+    out.dst_tile = b.tile;
     out.src_tile_bytes = l1 * e;
     out.dst_tile_bytes = l2 * e;
     out.bytes_read = gsize * e;

@@ -80,10 +80,12 @@ struct Launch {
     int first_step = 0, n_steps = 0, kernel = 0;
     BufKind from = BUF_SRC, to = BUF_DST;
     CopyGeometry geo;                    // what the kernel receives (without pointers)
+    std::vector<int32_t> src_tile_of;    // [devices]                source tile each device holds (-1: shared buffer)
     std::vector<int32_t> src_holder;     // [source tiles]           device whose buffer is read
     std::vector<int32_t> dst_devs;       // [target tiles * fanout]  devices that receive the tile
     i64 run_bytes = 0, bytes_read = 0, bytes_written = 0;
     i64 src_tile_bytes = 0, dst_tile_bytes = 0;
+    std::vector<i64> src_tile, dst_tile;     // tile shapes of the two layouts
 };
 
 struct Plan {

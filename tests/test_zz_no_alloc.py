@@ -65,10 +65,14 @@ def test_plans_beyond_the_built_in_array_are_refused():
     w = wl.config2()                                      # unfused: 16 MiB per virtual device
     plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, api.FUSE_NONE)
     assert plan.scratch_bytes > api.STATIC_SCRATCH_BYTES
-    fake = [torch.empty(16, dtype=torch.uint8, device="cuda")] * plan.n_devices
+    nb = plan.local_elems(0) * w.elem_bytes
+    src = [torch.empty(nb, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
+    dst = [torch.full((nb,), 0xEE, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
     with pytest.raises(api.RedistError) as e:
-        plan.execute_static(fake, fake)
-    assert e.value.status == 5                            # refused before anything runs
+        plan.execute_static(src, dst)
+    assert e.value.status == 5                            # refused ...
+    torch.cuda.synchronize()
+    assert all(bool((t == 0xEE).all()) for t in dst)      # ... before anything ran
 
 
 STATIC_CASES = [   # mesh, global shape, source axes, target axes, element bytes: small plans that need scratch when unfused
