@@ -15,7 +15,7 @@
  *     types").  Tile size = global size / product of the listed axis sizes; it must divide
  *     (rule wf-dim).  Axes a type does not list replicate the data.
  *   - Virtual device id = row-major index of the device's mesh coordinates over mesh_shape
- *     (last mesh axis fastest).  The paper leaves this numbering to the runtime (Section 2.2).
+ *     (last mesh axis fastest).  The paper leaves this numbering to the runtime (Section 2.1).
  *   - A tile is dense, row-major, last dimension contiguous, without padding.
  *   - All functions return a redist_status; nothing throws, aborts or prints across this
  *     boundary.  Output arguments are untouched on failure.

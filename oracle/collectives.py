@@ -2,7 +2,7 @@
 
 Used to check a synthesized sequence of collectives step by step; never imported by the product.
 
-A *type* here is a list, per array dimension, of mesh-axis indices (minor-to-major, Section 2.2)
+A *type* here is a list, per array dimension, of mesh-axis indices (minor-to-major, Section 2.1)
 over a mesh given as a tuple of axis sizes; the global shape is carried separately.
 
 Rules follow the figure "Typing collective operations" (T-AllGather, T-DynSlice, T-AllToAll,

@@ -6,7 +6,7 @@
  * What it computes is the *definition* of a redistribution, not the paper's algorithm:
  *   1. every device's base offset under a distributed type  (base offset maps D[[.]] and T[[.]],
  *      the figure "Semantics for distributed dimensions and types", part (a); axis order inside
- *      a dimension is minor-to-major, Section 2.2);
+ *      a dimension is minor-to-major, Section 2.1);
  *   2. the logical global array is assembled from the source tiles, tile of device d placed at
  *      its base offset (Section 4.1, "Semantics for distributed array types");
  *   3. every device's target tile is the slice of that global array at its base offset under the
@@ -14,11 +14,11 @@
  *      (Section 4.2), so exactly one result is correct.
  * There is no plan, no collective, no blocking beyond a row-wise memcpy of the last dimension.
  *
- * Conventions the paper leaves open (chosen once, stated in the design notes): tiles are dense
+ * Conventions the paper leaves open (chosen once, the same on both sides): tiles are dense
  * row-major; a device id is the row-major index of its coordinates over mesh_shape (last mesh
  * axis fastest).
  *
- * Pins (tests, no GPU): the worked example [8{"x","y"}32] of Section 2.2; the lemma that the
+ * Pins (tests, no GPU): the worked example [8{"x","y"}32] of Section 2.1; the lemma that the
  * image of D[[c{xs}n]] is all multiples of c below n; brute-force ownership enumeration written
  * separately in Python; the closed form for a linear-index fill; a numpy stack/transpose
  * formulation for 1-D meshes; A->B->A round trips.

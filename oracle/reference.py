@@ -1,7 +1,7 @@
 """TEST INFRASTRUCTURE -- ctypes front end of the C oracle ``redist_oracle.c``.
 
 A distributed type is passed as ``(global_shape, axes)`` where ``axes[k]`` lists the mesh axes
-(indices into ``mesh_shape``) that partition dimension ``k``, minor-to-major (Section 2.2 of the
+(indices into ``mesh_shape``) that partition dimension ``k``, minor-to-major (Section 2.1 of the
 paper).  Tiles are numpy ``uint8`` arrays of shape ``(*tile_shape, elem_bytes)``; everything is
 compared bytewise because the synthetic bf16/f32 patterns include NaNs.
 """

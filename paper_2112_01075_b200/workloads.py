@@ -5,7 +5,7 @@ offsets, no tiling, no plan): it names meshes and distributed types and fills gl
 It imports nothing else from this package, so test infrastructure can use it without loading
 the CUDA library.
 
-Notation (Section 2.2 of the paper, "Distributed array types"): a distributed type gives, per
+Notation (Section 2.1 of the paper, "Distributed array types"): a distributed type gives, per
 array dimension, the ordered list of mesh axes that partition it, listed minor-to-major (the
 first listed axis varies fastest).  Axes are named here by their index into ``mesh_shape``.
 A virtual device id is the row-major index of its coordinates over ``mesh_shape`` (last mesh

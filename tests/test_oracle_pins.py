@@ -22,7 +22,7 @@ def all_coords(mesh):
 
 
 def split_interval(mesh, n, ax, coord):
-    """Section 2.2 in words: the dimension is split over the last-listed (major) axis first, then
+    """Section 2.1 in words: the dimension is split over the last-listed (major) axis first, then
     every piece is split further along the axis listed before it, and so on."""
     lo, hi = 0, n
     for a in reversed(ax):
@@ -47,7 +47,7 @@ def linear_global(gshape):
 # ------------------------------------------------------------------------------ worked example
 
 def test_golden_axis_order_offsets():
-    names, mesh, (gshape, axes, tiles), rows = load_offset_table("sec2_2_axis_order_offsets.txt")
+    names, mesh, (gshape, axes, tiles), rows = load_offset_table("sec2_1_axis_order_offsets.txt")
     tile, off = oracle.base_offsets(mesh, (gshape, axes))
     assert tile == tiles
     for ix, iy, expect in rows:
