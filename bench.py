@@ -255,7 +255,7 @@ def time_legs(torch, legs, steps, warmup, per_launch=False, graphs=None):
 def kernel_name(api, li) -> str:
     kname = {"naive_gather": "allgather", "naive_slice": "dynslice", "copy": "allpermute"}.get(
         api.KERNELS[li.kernel], api.KERNELS[li.kernel])
-    return f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk', 7: '_zip'}.get(li.variant, '') }_kernel"
+    return f"redist_{kname}{ {4: '_bulk', 5: '_gather', 6: '_ragged_bulk', 7: '_zip', 8: '_box'}.get(li.variant, '') }_kernel"
 
 
 def spawn_ranks(n: int):

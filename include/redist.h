@@ -119,8 +119,9 @@ typedef struct redist_launch_info {
     int32_t fanout;                /* destination replicas stored per element read                     */
     int32_t variant;               /* kernel variant: 0 rows, 1 chunks, 2 ragged chunks, 3 units (register
                                       kernels), 4 TMA bulk copies, 5 gather walk, 6 ragged rows loaded by
-                                      TMA bulk copies, 7 zip through shared memory; the kernel is named
-                                      redist_<collective>[_bulk|_gather|_ragged_bulk|_zip]_kernel      */
+                                      TMA bulk copies, 7 zip through shared memory, 8 super-boxes through
+                                      shared memory; the kernel is named
+                                      redist_<collective>[_bulk|_gather|_ragged_bulk|_zip|_box]_kernel */
 } redist_launch_info;
 
 /*
@@ -161,6 +162,9 @@ void redist_plan_cache_clear(void);
  *   "gather"             0..2   gather walk: never / where measured faster (default 1) / wherever it applies
  *   "zip"                0..2   zip kernels: never / only where the gather walk is not chosen / wherever
  *                               they apply (default 2)
+ *   "box"                0..2   super-box kernels (several interleaving dimensions staged through shared
+ *                               memory at once): never / where the other short-run paths do badly
+ *                               (default 1) / wherever they apply
  *   "zip_walks"          0..7   chunk-to-unit maps the zip kernels may use: 1 periodic + 2 by range +
  *                               4 tabulated (default 7; the flat walk is always available)
  *   "zip_by_range_slots" >= 1   fewest chunk slots of a range for the by-range walk (default 256)

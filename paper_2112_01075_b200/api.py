@@ -334,7 +334,7 @@ class Plan:
             lines.append(f"  --{label}, cost {st['cost']}--> {fmt(st['post_axes'])}")
         for L in d["launches"]:
             g = L["geometry"]
-            how = "ragged rows, TMA bulk loads" if g["bulk"] == 2 else "TMA bulk copies" if g["bulk"] else ("rows", "chunks", "units", "gather walk", "zip through shared memory")[g["mode"]]
+            how = "ragged rows, TMA bulk loads" if g["bulk"] == 2 else "TMA bulk copies" if g["bulk"] else ("rows", "chunks", "units", "gather walk", "zip through shared memory", "super-boxes through shared memory")[g["mode"]]
             lines.append(f"  launch {L['kernel']}: steps {L['first_step']}..{L['first_step'] + L['n_steps'] - 1}, "
                          f"{L['from']} -> {L['to']}, runs of {L['run_bytes']} B, {g['n_items']} items, {how}")
         lines.append(f"  cost {d['cost']}, height {d['height']} <= max(localsize) "

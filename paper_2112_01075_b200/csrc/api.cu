@@ -71,6 +71,7 @@ const TuningName kTuningNames[] = {
     {"bulk", &Tuning::bulk, 0, 1},
     {"gather", &Tuning::gather, 0, 2},
     {"zip", &Tuning::zip, 0, 2},
+    {"box", &Tuning::box, 0, 2},
     {"zip_walks", &Tuning::zip_walks, 0, 7},
     {"zip_by_range_slots", &Tuning::zip_by_range_slots, 1, 1 << 20},
     {"item_kb", &Tuning::item_kb, 0, 1024},
@@ -477,7 +478,7 @@ redist_status redist_plan_launch_info(const redist_plan_t *plan, int32_t launch,
     o.bytes_written = L.bytes_written;
     o.n_items = L.geo.n_items;
     o.fanout = int32_t(L.geo.fanout);
-    o.variant = L.geo.bulk == 2 ? 6 : L.geo.bulk ? 4 : (L.geo.mode == kModeZip ? 7 : L.geo.mode == kModeGather ? 5 : L.geo.mode == kModeRows ? 0 : L.geo.mode == kModeUnits ? 3 : (L.geo.aligned ? 1 : 2));
+    o.variant = L.geo.bulk == 2 ? 6 : L.geo.bulk ? 4 : (L.geo.mode == kModeBox ? 8 : L.geo.mode == kModeZip ? 7 : L.geo.mode == kModeGather ? 5 : L.geo.mode == kModeRows ? 0 : L.geo.mode == kModeUnits ? 3 : (L.geo.aligned ? 1 : 2));
     *out = o;
     return REDIST_OK;
 }

@@ -41,6 +41,16 @@
 //               contiguous segment per stream -- are brought into shared memory by bulk copies, and
 //               the threads assemble target-aligned 16-byte chunks from shared memory, where a
 //               scattered access costs no cache-line lookups.
+//   kModeBox    short runs whose pieces interleave along SEVERAL dimensions, or along one whose neighbouring
+//               row digit is only a few rows long.  The item is widened from a box to a "super-box": in
+//               each of the innermost differing dimensions (the inner dimensions, at most kMaxBoxDims) it
+//               spans lcm(source tile, target tile) indices, so that it covers whole tiles of both sides
+//               there, times per_block rows of the dimension just outside them.  Its source bytes are then
+//               one long contiguous segment per source tile it touches, its target bytes one long contiguous
+//               range per target tile: the segments come into shared memory by bulk copies, and the ranges
+//               are written in target-aligned 16-byte chunks whose units are found through a table of one
+//               row's unit places (the place of a unit is separable: a term that depends on the target tile
+//               plus a term that depends on the position inside the row).
 //   kModeUnits  runs shorter than 256 bytes that are not 16-byte aligned: the same flat walk over
 //               pieces of unit_bytes.  Only the outer row digits go through the shared table; the
 //               innermost row digit is part of the walk (row payload = tab_inner.d runs), so that a
@@ -56,7 +66,9 @@ constexpr int kMaxRowDigits = 8;
 constexpr int kBlockThreads = 256;
 constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: one row segment per thread
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
-constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3, kModeZip = 4;
+constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3, kModeZip = 4, kModeBox = 5;
+constexpr int kMaxBoxDims = 3;         // inner dimensions of a kModeBox item
+constexpr int kBoxSegments = 64;       // source segments, and target ranges, of one kModeBox item at most
 constexpr int kZipSmallTile = 23 * 1024; // kModeZip items with at most this much shared memory run with 128 threads
 constexpr int kZipSegments = 256;      // source segments (table rows times streams) of one kModeZip item
 constexpr int kMaxGatherLevels = 2;    // innermost row digits that can be part of a stretch (kModeGather)
@@ -121,6 +133,21 @@ struct CopyGeometry {
     FastDiv row_n[kMaxRowDigits];
     int64_t row_b1[kMaxRowDigits];       // byte stride of the row digit, source / target
     int64_t row_b2[kMaxRowDigits];
+    uint32_t unit_mul[kMaxUnitDigits];   // kModeBox: boxes per super-box along the digit (the digit counts super-boxes); else 1
+    uint32_t bx_n;                   // kModeBox: inner dimensions, listed outer to inner below
+    FastDiv bx_c2[kMaxBoxDims];      //   target tile extent (a digit of a position inside a target row)
+    FastDiv bx_c1[kMaxBoxDims];      //   source tile extent
+    FastDiv bx_n1[kMaxBoxDims];      //   source tiles per super-box along the dimension
+    FastDiv bx_n2[kMaxBoxDims];      //   target tiles per super-box along the dimension
+    uint32_t bx_ts1[kMaxBoxDims];    //   tile-index strides, source / target
+    uint32_t bx_ts2[kMaxBoxDims];
+    uint32_t bx_st1[kMaxBoxDims];    //   bytes between neighbouring indices of the dimension inside a source segment row
+    uint32_t bx_seg[kMaxBoxDims];    //   segments between neighbouring source tiles of the dimension (mixed radix over bx_n1)
+    FastDiv bx_trail;                // kModeBox: units of a run (innermost digit of a position inside a target row; the last
+                                     //           inner dimension counts runs: its extents below are divided by the gcd)
+    FastDiv bx_s2;                   // kModeBox: bytes of one row (of the dimension outside the inner ones) in a target range
+    uint32_t bx_s1;                  //           ... in a source segment
+    uint32_t bx_nseg, bx_nrng;       // kModeBox: source segments / target ranges of an item
     uint32_t wait_polls;             // bulk-copy kernels: mbarrier polls before a block gives up (bounded wait)
     uint32_t test_extra_tx;          // test only: bytes announced on the mbarrier beyond what the copies deliver, so
                                      // that every copy lands but the phase never completes (0 in every real plan)

@@ -113,6 +113,25 @@ void describe(Plan &p)
         fd(o, G.gl_n, G.gl_levels);
         o << ",\"gl_b1\":";
         raw(o, G.gl_b1, G.gl_levels);
+        o << ",\"bx_n\":" << G.bx_n << ",\"bx_s1\":" << G.bx_s1 << ",\"bx_s2\":" << G.bx_s2.d << ",\"bx_nseg\":" << G.bx_nseg
+          << ",\"bx_nrng\":" << G.bx_nrng << ",\"bx_trail\":" << G.bx_trail.d << ",\"bx_c1\":";
+        fd(o, G.bx_c1, G.bx_n);
+        o << ",\"bx_c2\":";
+        fd(o, G.bx_c2, G.bx_n);
+        o << ",\"bx_n1\":";
+        fd(o, G.bx_n1, G.bx_n);
+        o << ",\"bx_n2\":";
+        fd(o, G.bx_n2, G.bx_n);
+        o << ",\"bx_ts1\":";
+        raw(o, G.bx_ts1, G.bx_n);
+        o << ",\"bx_ts2\":";
+        raw(o, G.bx_ts2, G.bx_n);
+        o << ",\"bx_st1\":";
+        raw(o, G.bx_st1, G.bx_n);
+        o << ",\"bx_seg\":";
+        raw(o, G.bx_seg, G.bx_n);
+        o << ",\"unit_mul\":";
+        raw(o, G.unit_mul, G.n_unit);
         o << ",\"unit_n\":";
         fd(o, G.unit_n, G.n_unit);
         o << ",\"unit_m1\":";

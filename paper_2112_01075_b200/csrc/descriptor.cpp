@@ -73,6 +73,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.unit_ts2[nu] = uint32_t(ts2[k]);
         G.unit_b1[nu] = g[k] * es1[k] * e;
         G.unit_b2[nu] = g[k] * es2[k] * e;
+        G.unit_mul[nu] = 1;
         n_boxes *= nq[k];
         if (n_boxes >= (1ll << 31)) return REDIST_EUNSUPPORTED;
         ++nu;
@@ -122,6 +123,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                 G.unit_ts2[pos] = T.unit_ts2[u];
                 G.unit_b1[pos] = T.unit_b1[u];
                 G.unit_b2[pos] = T.unit_b2[u];
+                G.unit_mul[pos] = T.unit_mul[u];
                 if (u == T.inner_digit) G.inner_digit = pos;
                 ++pos;
             };
@@ -254,7 +256,169 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         // a source segment of a full item should be worth a bulk copy
         if (piece_stride == run_bytes && d.b1 == bs && d.b2 == bd && d.n * bs >= 256 && d.n * bd >= kZipMinRange && m <= 16) zip_n = d.n;
     }
-    if (zip_n > 0) {
+    // box: the item is a super-box -- lcm(source tile, target tile) indices in each of the innermost
+    // differing dimensions ("inner" dimensions, kp and as many before it as it takes to make the
+    // contiguous pieces on both sides long), times a block of rows of the dimension K just outside them.
+    // Source bytes: one contiguous segment per source tile touched; target bytes: one contiguous range
+    // per target tile touched.  Chosen (tuning value "box": 0 never, 2 wherever it applies) for short
+    // runs where the zip kernels do not apply or would zip a digit of only a few rows.
+    struct BoxDim {
+        int k;
+        i64 c1, c2, E;
+    };
+    std::vector<BoxDim> bxd;      // inner dimensions, outer to inner
+    int bxK = -2;                 // the dimension outside them (-1: none)
+    i64 bx_s1 = 0, bx_s2 = 0, bx_cnt = 0, bx_gK = 1;
+    const i64 kBoxTile = 38 * 1024;
+    if (tune.box > 0 && kBulk && vec >= 4 && kp >= 0 && run_bytes < 2048 && nq[kp] > 1) {
+        i64 trail = e;                               // bytes of the identical trailing dimensions
+        for (int k = kp + 1; k < r; ++k) trail *= a.tile[k];
+        i64 s1 = trail, s2 = trail, sup = trail, n1 = 1, n2 = 1;
+        bool ok = true;
+        int k = kp;
+        while (ok) {
+            const i64 c1 = a.tile[k], c2 = b.tile[k];
+            if (c1 % c2 != 0 && c2 % c1 != 0) ok = false;      // neither tile size divides the other: not separable
+            const i64 E = std::max(c1, c2);
+            if (ok && (sup * E > kBoxTile || n1 * (E / c1) > kBoxSegments || n2 * (E / c2) > kBoxSegments ||
+                       s2 * c2 / vec > 4096))
+                ok = false;
+            if (!ok) break;
+            bxd.insert(bxd.begin(), BoxDim{k, c1, c2, E});
+            s1 *= c1;
+            s2 *= c2;
+            sup *= E;
+            n1 *= E / c1;
+            n2 *= E / c2;
+            // long enough with the rows of the next dimension out?  (segments of 512 bytes on both sides)
+            const i64 gk = k > 0 ? g[k - 1] : 1;
+            if (std::min(s1, s2) * std::min<i64>(gk, std::max<i64>(1, kItemBytes / sup)) >= 512 || k == 0 ||
+                int(bxd.size()) == kMaxBoxDims)
+                break;
+            --k;
+        }
+        if (!bxd.empty() && (ok || int(bxd.size()) > 0)) {
+            // (a failed extension keeps what was accepted so far)
+            bxK = bxd.front().k - 1;
+            bx_gK = bxK >= 0 ? g[bxK] : 1;
+            bx_s1 = s1;
+            bx_s2 = s2;
+            i64 cnt = std::max<i64>(1, std::min<i64>(bx_gK, kItemBytes / sup));
+            while (cnt > 1 && n1 * (round_up(cnt * s1, 16) + 32) > kBoxTile) --cnt;
+            bx_cnt = cnt;
+            const bool fits = n1 * (round_up(cnt * s1, 16) + 32) + 2 * (s2 / vec) + 16 * n2 <= 44 * 1024;
+            const bool worth = std::min(s1, s2) * cnt >= 128;
+            // default policy: where the unit walk or the gather walk would run, and where the zip kernels
+            // would zip a digit of fewer than 16 rows
+            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_n < 16 && run_bytes < 512
+                                                            : run_bytes < 256 && (g_levels >= 0 || !G.aligned));
+            if (!fits || !worth || !wanted || sup > (1ll << 30)) bxK = -2;
+        }
+    }
+    if (bxK >= -1) {
+        // unit digits from scratch: boxes of g for the dimensions up to K, super-boxes for the inner ones
+        n_boxes = 1;
+        nu = 0;
+        size_t bi = 0;
+        for (int k = 0; k < r; ++k) {
+            const bool in = k >= bxd.front().k && k <= kp;
+            const i64 mul = in ? bxd[bi].E / g[k] : 1;
+            if (in) ++bi;
+            if (nq[k] == 1) continue;
+            G.unit_n[nu] = make_div(uint32_t(nq[k] / mul));
+            G.unit_mul[nu] = uint32_t(mul);
+            G.unit_m1[nu] = make_div(uint32_t(m1[k]));
+            G.unit_m2[nu] = make_div(uint32_t(m2[k]));
+            G.unit_ts1[nu] = uint32_t(ts1[k]);
+            G.unit_ts2[nu] = uint32_t(ts2[k]);
+            G.unit_b1[nu] = g[k] * es1[k] * e;
+            G.unit_b2[nu] = g[k] * es2[k] * e;
+            n_boxes *= nq[k] / mul;
+            ++nu;
+        }
+        G.n_unit = nu;
+        G.inner_n = make_div(1);
+        G.inner_digit = 0xffffffffu;
+        G.inner_span = 1;
+        G.inner_mul = 1;
+        inner = 1;
+        G.fast_boxes = make_div(1);
+        // row digits: the dimensions before K (merged where both sides stay contiguous), K itself, then the
+        // inner dimensions but the last as plain row digits of a box (the kernel does not use those: it
+        // works on the super-box, whose rows are described by the bx_ fields)
+        rows.clear();
+        for (int k = 0; k < bxK; ++k)
+            if (g[k] > 1) rows.push_back(RowDigit{g[k], es1[k] * e, es2[k] * e});
+        for (size_t q = rows.size(); q-- > 1;) {
+            RowDigit &o = rows[q - 1], &in = rows[q];
+            if (o.b1 == in.n * in.b1 && o.b2 == in.n * in.b2) {
+                in.n *= o.n;
+                rows.erase(rows.begin() + (q - 1));
+            }
+        }
+        const size_t n_outer = rows.size();
+        i64 tab_rows = 1;
+        for (const RowDigit &d : rows) tab_rows *= d.n;
+        rows.push_back(RowDigit{bx_gK, bxK >= 0 ? es1[bxK] * e : 0, bxK >= 0 ? es2[bxK] * e : 0});
+        for (size_t q = 0; q + 1 < bxd.size(); ++q)
+            if (g[bxd[q].k] > 1) rows.push_back(RowDigit{g[bxd[q].k], es1[bxd[q].k] * e, es2[bxd[q].k] * e});
+        if (rows.size() > size_t(kMaxRowDigits)) return REDIST_EUNSUPPORTED;
+        n_rows = 1;
+        for (size_t q = 0; q < rows.size(); ++q) {
+            G.row_n[q] = make_div(uint32_t(rows[q].n));
+            G.row_b1[q] = rows[q].b1;
+            G.row_b2[q] = rows[q].b2;
+            n_rows *= rows[q].n;
+        }
+        G.n_row = uint32_t(rows.size());
+        G.mode = kModeBox;
+        G.rows = uint32_t(tab_rows);
+        G.n_row_tab = uint32_t(n_outer);
+        G.tab_inner = make_div(uint32_t(bx_gK));
+        G.units_per_run = make_div(uint32_t(run_bytes / vec));
+        G.rows_per_item = 1;
+        G.per_block = uint32_t(bx_cnt);
+        const i64 ncb = (bx_gK + bx_cnt - 1) / bx_cnt;
+        G.col_blocks = make_div(uint32_t(ncb));
+        i64 trail = e;
+        for (int k = kp + 1; k < r; ++k) trail *= a.tile[k];
+        i64 n1 = 1, n2 = 1;
+        G.bx_n = uint32_t(bxd.size());
+        // The innermost digit of a position inside a target row is the unit inside a run (the run is
+        // contiguous on both sides, and the unit size divides it but not necessarily the trailing
+        // dimensions); the last inner dimension therefore counts runs: its extents are divided by the gcd.
+        const i64 gl = g[kp];
+        for (size_t q = bxd.size(); q-- > 0;) {
+            // inner to outer: strides inside a source segment row, segment steps
+            i64 st = run_bytes, seg = 1;
+            for (size_t w = q + 1; w < bxd.size(); ++w) {
+                st *= bxd[w].c1 / (w + 1 == bxd.size() ? gl : 1);
+                seg *= bxd[w].E / bxd[w].c1;
+            }
+            const i64 sc = q + 1 == bxd.size() ? gl : 1;
+            G.bx_c1[q] = make_div(uint32_t(bxd[q].c1 / sc));
+            G.bx_c2[q] = make_div(uint32_t(bxd[q].c2 / sc));
+            G.bx_n1[q] = make_div(uint32_t(bxd[q].E / bxd[q].c1));
+            G.bx_n2[q] = make_div(uint32_t(bxd[q].E / bxd[q].c2));
+            G.bx_ts1[q] = uint32_t(ts1[bxd[q].k]);
+            G.bx_ts2[q] = uint32_t(ts2[bxd[q].k]);
+            G.bx_st1[q] = uint32_t(st);
+            G.bx_seg[q] = uint32_t(seg);
+            n1 *= bxd[q].E / bxd[q].c1;
+            n2 *= bxd[q].E / bxd[q].c2;
+        }
+        G.bx_trail = make_div(uint32_t(run_bytes / vec));
+        G.bx_s1 = uint32_t(bx_s1);
+        G.bx_s2 = make_div(uint32_t(bx_s2));
+        G.bx_nseg = uint32_t(n1);
+        G.bx_nrng = uint32_t(n2);
+        G.zip_seg_pitch = uint32_t(round_up(bx_cnt * bx_s1, 16) + 32);
+        G.stage_pitch = uint32_t(G.zip_seg_pitch * n1);
+        G.zip_lut_units = uint32_t(bx_s2 / vec);
+        G.zip_slots = make_div(uint32_t(bx_cnt * bx_s2 / 16 + 1));
+        G.gl_m = make_div(1);
+        ipb = tab_rows * ncb;
+    } else if (zip_n > 0) {
         const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);
         const i64 nseg = long_dst ? m : 1;                 // source segments per table row

@@ -23,10 +23,12 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     run = G["run_bytes"]
     assert run == L["run_bytes"] and run > 0
     unit_n = G["unit_n"]
+    unit_mul = G["unit_mul"]
+    assert all(m >= 1 for m in unit_mul) and (G["mode"] == 5 or all(m == 1 for m in unit_mul))
     n_boxes = _prod(unit_n)
     rows = _prod(G["row_n"])
     tab_rows = G["rows"]
-    assert tab_rows * G["tab_inner"] == rows
+    assert tab_rows * G["tab_inner"] == rows or G["mode"] == 5
     inner, span, mul = G["inner_n"], G["inner_span"], G["inner_mul"]
     assert inner * mul == span
     assert G["n_items"] == n_boxes * G["items_per_box"] * inner
@@ -81,6 +83,31 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             assert not G["zip_period"] and G["zip_lut_units"] == rpb * (m * run if long_dst else run) // unit <= 2048
             assert G["stage_pitch"] * rpi + 4 * G["zip_lut_units"] <= 42 * 1024
         assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
+    elif G["mode"] == 5:    # super-boxes: lcm(source tile, target tile) in the inner dimensions, staged by bulk copies
+        nb = G["bx_n"]
+        assert 1 <= nb <= 3 and unit >= 4 and inner == span == mul == 1 and G["rows_per_item"] == 1
+        c1, c2, n1, n2 = G["bx_c1"], G["bx_c2"], G["bx_n1"], G["bx_n2"]
+        trail = G["bx_trail"] * unit
+        for q in range(nb):
+            assert c1[q] % c2[q] == 0 or c2[q] % c1[q] == 0          # separable places
+            assert c1[q] * n1[q] == c2[q] * n2[q] == max(c1[q], c2[q])
+            assert G["bx_st1"][q] == trail * _prod(c1[q + 1:]) and G["bx_seg"][q] == _prod(n1[q + 1:])
+        assert G["bx_s1"] == trail * _prod(c1) and G["bx_s2"] == trail * _prod(c2)
+        assert G["bx_nseg"] == _prod(n1) <= 64 and G["bx_nrng"] == _prod(n2) <= 64
+        assert run == trail and min(c1[-1], c2[-1]) == 1     # the last inner dimension counts runs
+        nK, cnt = G["tab_inner"], G["per_block"]
+        n_out = G["n_row_tab"]
+        assert G["row_n"][n_out] == nK and 1 <= cnt <= nK and G["col_blocks"] == -(-nK // cnt)
+        assert tab_rows == _prod(G["row_n"][:n_out]) and rows == tab_rows * nK * _prod(G["row_n"][n_out + 1:])
+        if nK > 1:
+            assert G["row_b1"][n_out] == G["bx_s1"] and G["row_b2"][n_out] == G["bx_s2"]   # rows of K are contiguous
+        assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= cnt * G["bx_s1"] + 30
+        assert G["stage_pitch"] == G["zip_seg_pitch"] * G["bx_nseg"] <= 38 * 1024
+        assert G["zip_lut_units"] * unit == G["bx_s2"] and G["zip_lut_units"] <= 4096
+        assert G["zip_slots"] >= cnt * G["bx_s2"] // 16 + 1
+        assert G["items_per_box"] == tab_rows * G["col_blocks"]
+        # the digits of the inner dimensions count super-boxes: unit_mul boxes of the gcd size each
+        assert _prod(unit_mul) >= 1
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
         assert unit == 16 and max_chunks <= 256 and G["lanes"] == max_chunks
         assert G["rows_per_pass"] == 256 // G["lanes"] and G["rows_per_item"] % G["rows_per_pass"] == 0
@@ -104,12 +131,13 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         s2 += dg * G["row_b2"][q]
     col = np.arange(run, dtype=np.int64)
     written = {}
-    for boxp in range(n_boxes * span):
+    for boxp in range(n_boxes * span * _prod(unit_mul)):
         box, piece = divmod(boxp, span)          # a gather item covers `mul` consecutive pieces
         rem, t1, t2, o1, o2 = box, 0, 0, 0, 0
         for u in range(len(unit_n) - 1, -1, -1):
-            q = rem % unit_n[u]
-            rem //= unit_n[u]
+            # (a super-box digit counts unit_mul boxes: enumerate them all)
+            q = rem % (unit_n[u] * unit_mul[u])
+            rem //= unit_n[u] * unit_mul[u]
             if u == G["inner_digit"]:
                 q = q * span + piece
             a1, b1 = divmod(q, G["unit_m1"][u])
@@ -128,7 +156,77 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             dst[idx] = data
             w = written.setdefault(dev, np.zeros(dst.shape[0], dtype=np.int32))
             np.add.at(w, idx.reshape(-1), 1)
+    if G["mode"] == 5:
+        check_box_items(L, src_bufs, dst_bufs)
     return written
+
+
+def check_box_items(L: dict, src_bufs, dst_bufs):
+    """The super-box kernel works from its own description of an item (segments, ranges, the table of unit
+    places and the corners of the target tiles).  Replay that arithmetic item by item, as the kernel does
+    it, and require that it reproduces what the box-by-box interpretation above has just written."""
+    G = L["geometry"]
+    fan, unit = G["fanout"], G["unit_bytes"]
+    nb = G["bx_n"]
+    c1, c2, n1, n2 = G["bx_c1"], G["bx_c2"], G["bx_n1"], G["bx_n2"]
+    s1, s2, pitch = G["bx_s1"], G["bx_s2"], G["zip_seg_pitch"]
+    n_out = G["n_row_tab"]
+    place = np.zeros(G["zip_lut_units"], dtype=np.int64)
+    for p in range(G["zip_lut_units"]):
+        rest, off = divmod(p, G["bx_trail"])
+        off *= unit
+        for q in range(nb - 1, -1, -1):
+            rest, i = divmod(rest, c2[q])
+            hi, lo = divmod(i, c1[q])
+            off += hi * G["bx_seg"][q] * pitch + lo * G["bx_st1"][q]
+        assert off < 65536
+        place[p] = off
+    for item in range(G["n_items"]):
+        rest, part = divmod(item, G["items_per_box"])          # inner_n = fast_boxes = 1 in this mode
+        t1 = t2 = o1 = o2 = 0
+        for u in range(len(G["unit_n"]) - 1, -1, -1):
+            rest, q = divmod(rest, G["unit_n"][u])
+            q *= G["unit_mul"][u]
+            a1, b1 = divmod(q, G["unit_m1"][u])
+            a2, b2 = divmod(q, G["unit_m2"][u])
+            t1 += a1 * G["unit_ts1"][u]
+            t2 += a2 * G["unit_ts2"][u]
+            o1 += b1 * G["unit_b1"][u]
+            o2 += b2 * G["unit_b2"][u]
+        group, cb = divmod(part, G["col_blocks"])
+        r1 = r2 = 0
+        rem = group
+        for q in range(n_out - 1, -1, -1):
+            rem, dg = divmod(rem, G["row_n"][q])
+            r1 += dg * G["row_b1"][q]
+            r2 += dg * G["row_b2"][q]
+        a = cb * G["per_block"]
+        cnt = min(G["per_block"], G["tab_inner"] - a)
+        so, d0 = o1 + r1 + a * s1, o2 + r2 + a * s2
+        mis = so % 16
+        stage = np.zeros(G["stage_pitch"] + 64, dtype=np.uint8)
+        for t in range(G["bx_nseg"]):
+            rem, tile = t, t1
+            for q in range(nb - 1, -1, -1):
+                rem, d = divmod(rem, n1[q])
+                tile += d * G["bx_ts1"][q]
+            src = src_bufs(L["src_holder"][tile])
+            assert so + cnt * s1 <= src.shape[0]
+            stage[t * pitch + mis:t * pitch + mis + cnt * s1] = src[so:so + cnt * s1]
+        for t in range(G["bx_nrng"]):
+            rem, tile, base = t, t2, mis
+            for q in range(nb - 1, -1, -1):
+                rem, d = divmod(rem, n2[q])
+                tile += d * G["bx_ts2"][q]
+                hi, lo = divmod(d * c2[q], c1[q])
+                base += hi * G["bx_seg"][q] * pitch + lo * G["bx_st1"][q]
+            x = np.arange(0, cnt * s2, unit, dtype=np.int64)
+            at = base + (x // s2) * s1 + place[(x % s2) // unit]
+            got = stage[at[:, None] + np.arange(unit)[None, :]].reshape(-1)
+            for f in range(fan):
+                dst = dst_bufs(L["dst_devs"][tile * fan + f])
+                assert d0 + cnt * s2 <= dst.shape[0]
+                assert np.array_equal(dst[d0:d0 + cnt * s2], got), (item, t, f)
 
 
 def run_plan(desc: dict, src_tiles):

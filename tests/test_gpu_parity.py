@@ -164,6 +164,47 @@ def test_zip_kernels_with_each_chunk_map(values):
     assert 7 in v, v
 
 
+def test_super_box_kernels_wherever_they_apply():
+    """box = 2 sends every launch whose inner dimensions allow it through the super-box kernels (by default
+    only where the zip, gather and unit walks do badly)."""
+    with api.tuning(box=2):
+        v = random_problems_small_and_odd(600)
+    assert 8 in v, v
+    with api.tuning(box=0):
+        v = random_problems_small_and_odd(300)
+    assert 8 not in v, v
+
+
+BOXES = [   # mesh, global shape, source axes, target axes, element bytes: several dimensions interleave at run granularity
+    ((4, 4, 4), (8, 12, 2, 28, 20, 12), ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,)), 4),   # 12-byte runs, 3 inner dimensions
+    ((4, 4, 2), (2, 8, 8, 30, 4, 8), ((), (), (), (), (1,), (0,)), ((), (1,), (0,), (2,), (), ()), 4),      # 8-byte runs from 16 tiles
+    ((2, 2, 2), (6, 6, 6, 48, 10, 26), ((), (2,), (), (0,), (), ()), ((), (), (1,), (), (2,), (0,)), 4),   # 52-byte runs, short zipped digit
+    ((2, 3), (6, 9, 10, 6), ((), (1,), (0,), ()), ((), (), (), (1,)), 2),                                  # odd primes, 2-byte elements
+    ((2, 2, 2), (4, 8, 12, 6), ((0,), (1,), (2,), ()), ((), (2,), (0,), (1,)), 8),                          # every dimension changes, fan-out 1
+    ((2, 2, 2), (4, 8, 12, 6), ((0,), (1,), (2,), ()), ((), (), (0,), ()), 4),                              # replicated target: fan-out 4
+]
+
+
+@pytest.mark.parametrize("mesh,gshape,a1,a2,e", BOXES)
+def test_super_box_kernels(mesh, gshape, a1, a2, e):
+    """Short runs that interleave along several dimensions: the item is widened to a super-box, staged in
+    shared memory segment by segment and written out range by range (launch variant 8).  Both directions,
+    fused and collective by collective, with the kernels on by default and forced."""
+    rng = np.random.default_rng(sum(gshape) + e)
+    G = rng.integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+    seen = set()
+    for src, dst in (((gshape, a1), (gshape, a2)), ((gshape, a2), (gshape, a1))):
+        src_tiles = oracle.reslice(mesh, src, G)
+        want = oracle.reslice(mesh, dst, G)
+        for box in (1, 2):
+            with api.tuning(box=box):
+                for mode in (api.FUSE_ADJACENT, api.FUSE_NONE):
+                    plan, got = run_gpu(mesh, src, dst, e, src_tiles, mode)
+                    seen.update(plan.launch_info(q).variant for q in range(plan.num_launches))
+                    assert_same(got, want, f"super-box {mesh} {src} -> {dst} box={box} mode={mode}")
+    assert 8 in seen
+
+
 def test_gather_walk_wherever_it_applies():
     """gather = 2 sends every eligible launch through the gather walk, including long source rows that
     are scattered into several target tiles and 16-byte units (not chosen by default)."""

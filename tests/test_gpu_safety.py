@@ -53,6 +53,12 @@ with api.tuning(bulk=0, gather=0):
     variants |= T.random_problems_small_and_odd(200)
 with api.tuning(gather=2, zip=0):
     variants |= T.random_problems_small_and_odd(200)
+with api.tuning(box=2):
+    variants |= T.random_problems_small_and_odd(400)
+with api.tuning(box=0):
+    variants |= T.random_problems_small_and_odd(200)
+for case in T.BOXES:
+    T.test_super_box_kernels(*case)
 for values in ({"zip_walks": 0}, {"zip_walks": 2, "zip_by_range_slots": 1}, {"zip_walks": 4}):
     with api.tuning(**values):
         variants |= T.random_problems_small_and_odd(200)
@@ -78,7 +84,7 @@ for w in T.MEDIUM:
         _, got = T.run_gpu(w.mesh_shape, src, dst, w.elem_bytes, tiles, mode)
         T.assert_same(got, want, w.name)
 torch.cuda.synchronize()
-assert variants >= {0, 1, 2, 3, 4, 5, 6, 7}, variants
+assert variants >= {0, 1, 2, 3, 4, 5, 6, 7, 8}, variants
 rep = api.debug_bounds_report()
 assert rep[0] == 0, "out-of-range access skipped: count %d, line %d, block %d, side %d, distance %d" % rep
 assert api.redist_bulk_timeouts() == 0
@@ -116,6 +122,7 @@ TIMEOUT_CASES = {
     4: ((2,), (64, 2048), ((0,), ()), ((), (0,)), 2),          # aligned 2 KiB runs: plain bulk copies, 16 blocks
     6: ((2,), (16, 2050), ((), (0,)), ((), ()), 4),            # ragged 4100-byte runs: bulk-loaded chunk walk, 8 blocks
     7: ((2,), (1024, 24), ((), (0,)), ((), ()), 4),            # 48-byte runs zipped through shared memory, 7 blocks
+    8: ((2, 2), (8, 8, 24, 12), ((), (), (0,), (1,)), ((), (0,), (), ()), 4),    # super-boxes, 16 blocks
 }
 
 TIMEOUT_RUN = r"""
@@ -129,7 +136,7 @@ for variant, (mesh, gshape, a1, a2, e) in sorted(TIMEOUT_CASES.items()):
     src, dst = (gshape, a1), (gshape, a2)
     G = np.random.default_rng(variant).integers(0, 256, size=gshape + (e,), dtype=np.uint8)
     tiles, want = oracle.reslice(mesh, src, G), oracle.reslice(mesh, dst, G)
-    with api.tuning(test_extra_tx=16, wait_polls=4096):
+    with api.tuning(test_extra_tx=16, wait_polls=4096, box=2 if variant == 8 else 0):
         broken = api.Plan(mesh, src, dst, e)
     li = broken.launch_info(0)
     assert broken.num_launches == 1 and li.variant == variant and 1 <= li.n_items <= 16, (variant, li.variant, li.n_items)
