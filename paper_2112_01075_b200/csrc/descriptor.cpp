@@ -290,9 +290,12 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             sup *= E;
             n1 *= E / c1;
             n2 *= E / c2;
-            // long enough with the rows of the next dimension out?  (segments of 512 bytes on both sides)
+            // enough with the rows of the next dimension out?  (segments of 512 bytes on both sides, and an
+            // item of at least half the usual size: a block pays for its decode, its barrier and its table
+            // of places whatever it moves)
             const i64 gk = k > 0 ? g[k - 1] : 1;
-            if (std::min(s1, s2) * std::min<i64>(gk, std::max<i64>(1, kItemBytes / sup)) >= 512 || k == 0 ||
+            const i64 cmax = std::min<i64>(gk, std::max<i64>(1, kItemBytes / sup));
+            if ((std::min(s1, s2) * cmax >= 512 && sup * cmax >= kItemBytes / 2) || k == 0 ||
                 int(bxd.size()) == kMaxBoxDims)
                 break;
             --k;
@@ -307,7 +310,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             while (cnt > 1 && n1 * (round_up(cnt * s1, 16) + 32) > kBoxTile) --cnt;
             bx_cnt = cnt;
             const bool fits = n1 * (round_up(cnt * s1, 16) + 32) + 2 * (s2 / vec) + 16 * n2 <= 44 * 1024;
-            const bool worth = std::min(s1, s2) * cnt >= 128;
+            // (forced, any item will do; by default only items worth a block)
+            const bool worth = tune.box >= 2 ? std::min(s1, s2) * cnt >= 128
+                                             : std::min(s1, s2) * cnt >= 256 && sup * cnt >= kItemBytes / 4;
             // default policy: where the unit walk or the gather walk would run, and where the zip kernels
             // would zip a digit of fewer than 16 rows
             const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_n < 16 && run_bytes < 512

@@ -51,7 +51,7 @@ variants = set()
 variants |= T.random_problems_small_and_odd(600)
 with api.tuning(bulk=0, gather=0):
     variants |= T.random_problems_small_and_odd(200)
-with api.tuning(gather=2, zip=0):
+with api.tuning(gather=2, zip=0, box=0):
     variants |= T.random_problems_small_and_odd(200)
 with api.tuning(box=2):
     variants |= T.random_problems_small_and_odd(400)

@@ -520,7 +520,8 @@ KERNEL_CHOICE = [   # mesh, global shape, source axes, target axes, element byte
     ((4, 2), (8, 2048, 4096), ((0,), (), (1,)), ((), (0, 1), ()), 2, [4]),             # 4 KiB aligned runs: bulk copies
     ((2,), (64, 24), ((), ()), ((), (0,)), 4, [7]),                                    # 48-byte runs unzipped into 2 tiles
     ((2,), (64, 24), ((), (0,)), ((), ()), 4, [7]),                                    # and zipped back
-    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4, [5]),                      # interleave without a contiguous row digit
+    ((4, 2), (5, 8, 36), ((), (1,), (0,)), ((), (), ()), 4, [8]),                      # two dimensions interleave: super-boxes
+    ((4, 4, 4), (8, 12, 2, 28, 20, 12), ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,)), 4, [8]),   # three
     ((2, 2), (16, 6, 4), ((), (0,), ()), ((), (), (0, 1)), 8, [3]),                    # 8-byte runs scattered: unit walk
     ((2,), (6, 70), ((0,), ()), ((), ()), 4, [6]),                                     # ragged 840-byte runs: bulk-loaded chunk walk
     ((4,), (16, 16), ((0,), ()), ((), (0,)), 4, [0]),                                  # aligned 16-byte runs, too few rows to zip: rows
