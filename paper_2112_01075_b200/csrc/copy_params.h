@@ -45,7 +45,8 @@
 //               row digit is only a few rows long.  The item is widened from a box to a "super-box": in
 //               each of the innermost differing dimensions (the inner dimensions, at most kMaxBoxDims) it
 //               spans lcm(source tile, target tile) indices, so that it covers whole tiles of both sides
-//               there, times per_block rows of the dimension just outside them.  Its source bytes are then
+//               there, times per_block rows of the dimension just outside them, times rows_per_item rows of
+//               the dimensions further out.  Its source bytes are then
 //               one long contiguous segment per source tile it touches, its target bytes one long contiguous
 //               range per target tile: the segments come into shared memory by bulk copies, and the ranges
 //               are written in target-aligned 16-byte chunks whose units are found through a table of one
@@ -68,7 +69,8 @@ constexpr int kBulkThreads = 64;       // block size of the bulk-copy kernels: o
 constexpr int kMaxRowsFlat = 1024;     // rows of one item in the flat-walk modes (16 bytes of smem each)
 constexpr int kModeRows = 0, kModeChunks = 1, kModeUnits = 2, kModeGather = 3, kModeZip = 4, kModeBox = 5;
 constexpr int kMaxBoxDims = 3;         // inner dimensions of a kModeBox item
-constexpr int kBoxSegments = 64;       // source segments, and target ranges, of one kModeBox item at most
+constexpr int kBoxSegments = 256;      // source segments, and target ranges, of one kModeBox item at most
+constexpr int kBoxRows = 32;           // outer rows of one kModeBox item at most
 constexpr int kZipSmallTile = 23 * 1024; // kModeZip items with at most this much shared memory run with 128 threads
 constexpr int kZipSegments = 256;      // source segments (table rows times streams) of one kModeZip item
 constexpr int kMaxGatherLevels = 2;    // innermost row digits that can be part of a stretch (kModeGather)
@@ -147,7 +149,8 @@ struct CopyGeometry {
                                      //           inner dimension counts runs: its extents below are divided by the gcd)
     FastDiv bx_s2;                   // kModeBox: bytes of one row (of the dimension outside the inner ones) in a target range
     uint32_t bx_s1;                  //           ... in a source segment
-    uint32_t bx_nseg, bx_nrng;       // kModeBox: source segments / target ranges of an item
+    uint32_t bx_nseg, bx_nrng;       // kModeBox: source segments / target ranges of one outer row of an item
+    FastDiv bx_nseg_div, bx_nrng_div;
     uint32_t wait_polls;             // bulk-copy kernels: mbarrier polls before a block gives up (bounded wait)
     uint32_t test_extra_tx;          // test only: bytes announced on the mbarrier beyond what the copies deliver, so
                                      // that every copy lands but the phase never completes (0 in every real plan)

@@ -268,7 +268,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     };
     std::vector<BoxDim> bxd;      // inner dimensions, outer to inner
     int bxK = -2;                 // the dimension outside them (-1: none)
-    i64 bx_s1 = 0, bx_s2 = 0, bx_cnt = 0, bx_gK = 1;
+    i64 bx_s1 = 0, bx_s2 = 0, bx_cnt = 0, bx_gK = 1, bx_rpi = 1;
     const i64 kBoxTile = 38 * 1024;
     if (tune.box > 0 && kBulk && vec >= 4 && kp >= 0 && run_bytes < 2048 && nq[kp] > 1) {
         i64 trail = e;                               // bytes of the identical trailing dimensions
@@ -280,7 +280,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             const i64 c1 = a.tile[k], c2 = b.tile[k];
             if (c1 % c2 != 0 && c2 % c1 != 0) ok = false;      // neither tile size divides the other: not separable
             const i64 E = std::max(c1, c2);
-            if (ok && (sup * E > kBoxTile || n1 * (E / c1) > kBoxSegments || n2 * (E / c2) > kBoxSegments ||
+            if (ok && (sup * E > kBoxTile || n1 * (E / c1) > kBoxSegments / 4 || n2 * (E / c2) > kBoxSegments / 4 ||
                        s2 * c2 / vec > 4096))
                 ok = false;
             if (!ok) break;
@@ -290,14 +290,12 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             sup *= E;
             n1 *= E / c1;
             n2 *= E / c2;
-            // enough with the rows of the next dimension out?  (segments of 512 bytes on both sides, and an
-            // item of at least half the usual size: a block pays for its decode, its barrier and its table
-            // of places whatever it moves)
+            // long enough with the rows of the next dimension out?  (segments of 512 bytes on both sides;
+            // an item is then filled up with further outer rows, so the inner dimensions need not grow for
+            // the sake of its size)
             const i64 gk = k > 0 ? g[k - 1] : 1;
             const i64 cmax = std::min<i64>(gk, std::max<i64>(1, kItemBytes / sup));
-            if ((std::min(s1, s2) * cmax >= 512 && sup * cmax >= kItemBytes / 2) || k == 0 ||
-                int(bxd.size()) == kMaxBoxDims)
-                break;
+            if (std::min(s1, s2) * cmax >= 512 || k == 0 || int(bxd.size()) == kMaxBoxDims) break;
             --k;
         }
         if (!bxd.empty() && (ok || int(bxd.size()) > 0)) {
@@ -309,10 +307,18 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             i64 cnt = std::max<i64>(1, std::min<i64>(bx_gK, kItemBytes / sup));
             while (cnt > 1 && n1 * (round_up(cnt * s1, 16) + 32) > kBoxTile) --cnt;
             bx_cnt = cnt;
-            const bool fits = n1 * (round_up(cnt * s1, 16) + 32) + 2 * (s2 / vec) + 16 * n2 <= 44 * 1024;
+            // outer rows per item: fill the item up, within the segment and range tables and the tile
+            i64 outer_rows = 1;
+            for (int q = 0; q < bxK; ++q) outer_rows *= g[q];
+            const i64 seg_pitch = round_up(cnt * s1, 16) + 32;
+            i64 rpi = std::max<i64>(1, kItemBytes / (cnt * sup));
+            rpi = std::min<i64>(std::min<i64>(rpi, outer_rows), std::min<i64>(kBoxRows, kBoxSegments / std::max(n1, n2)));
+            rpi = std::max<i64>(1, std::min<i64>(rpi, kBoxTile / (seg_pitch * n1)));
+            bx_rpi = rpi;
+            const bool fits = rpi * n1 * seg_pitch + 2 * (s2 / vec) + 16 <= 44 * 1024;
             // (forced, any item will do; by default only items worth a block)
             const bool worth = tune.box >= 2 ? std::min(s1, s2) * cnt >= 128
-                                             : std::min(s1, s2) * cnt >= 256 && sup * cnt >= kItemBytes / 4;
+                                             : std::min(s1, s2) * cnt >= 256 && sup * cnt * rpi >= kItemBytes / 4;
             // default policy: where the unit walk or the gather walk would run, and where the zip kernels
             // would zip a digit of fewer than 16 rows
             const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_n < 16 && run_bytes < 512
@@ -381,7 +387,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.n_row_tab = uint32_t(n_outer);
         G.tab_inner = make_div(uint32_t(bx_gK));
         G.units_per_run = make_div(uint32_t(run_bytes / vec));
-        G.rows_per_item = 1;
+        G.rows_per_item = uint32_t(bx_rpi);
         G.per_block = uint32_t(bx_cnt);
         const i64 ncb = (bx_gK + bx_cnt - 1) / bx_cnt;
         G.col_blocks = make_div(uint32_t(ncb));
@@ -417,12 +423,14 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.bx_s2 = make_div(uint32_t(bx_s2));
         G.bx_nseg = uint32_t(n1);
         G.bx_nrng = uint32_t(n2);
+        G.bx_nseg_div = make_div(uint32_t(n1));
+        G.bx_nrng_div = make_div(uint32_t(n2));
         G.zip_seg_pitch = uint32_t(round_up(bx_cnt * bx_s1, 16) + 32);
-        G.stage_pitch = uint32_t(G.zip_seg_pitch * n1);
+        G.stage_pitch = uint32_t(G.zip_seg_pitch * n1);          // one outer row of the item
         G.zip_lut_units = uint32_t(bx_s2 / vec);
         G.zip_slots = make_div(uint32_t(bx_cnt * bx_s2 / 16 + 1));
         G.gl_m = make_div(1);
-        ipb = tab_rows * ncb;
+        ipb = (tab_rows + bx_rpi - 1) / bx_rpi * ncb;
     } else if (zip_n > 0) {
         const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);

@@ -1311,11 +1311,12 @@ REDIST_DEFINE_ZIP_KERNEL(redist_allpermute_zip_kernel)
 REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
 
 // ---- kModeBox: super-box items, several interleaving dimensions at once -------------------------
-// One item per block: per_block rows (of the dimension K outside the inner ones) of one super-box.
-// Source side: bx_nseg segments, one per source tile the super-box touches, each cnt * bx_s1 contiguous
-// bytes at the same offset inside its tile (so all segments share one misalignment), brought into
-// shared memory at a uniform pitch by one bulk copy each.  Target side: bx_nrng ranges, one per target
-// tile, each cnt * bx_s2 contiguous bytes at the same offset inside its tile.  The place in shared
+// One item per block: rows_per_item outer rows times per_block rows (of the dimension K outside the inner
+// ones) of one super-box.  Source side, per outer row: bx_nseg segments, one per source tile the
+// super-box touches, each cnt * bx_s1 contiguous bytes at the same offset inside its tile (so the segments
+// of a row share one misalignment), brought into shared memory at a uniform pitch by one bulk copy each.
+// Target side, per outer row: bx_nrng ranges, one per target tile, each cnt * bx_s2 contiguous bytes at
+// the same offset inside its tile.  The place in shared
 // memory of the unit at byte x of range t is
 //     base[t] + (x / bx_s2) * bx_s1 + place[(x % bx_s2) / unit]
 // base[t]: where the target tile's corner lies (segment and offset inside the segment's row), place[]:
@@ -1326,7 +1327,7 @@ REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
 // while its copies are in flight; a unit then costs a table read and the read of the unit.
 template <typename T, int NT>
 __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char *tile, uint32_t *base_of,
-                                         uint32_t *tile_of, uint32_t mbar, unsigned int *wait_failed)
+                                         uint32_t *tile_of, int64_t *row_d0, uint32_t mbar, unsigned int *wait_failed)
 {
     constexpr int kPer = 16 / int(sizeof(T));
     const CopyGeometry &g = P.g;
@@ -1336,33 +1337,37 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
     const uint32_t item = blockIdx.x;
     if (item >= g.n_items) return;
     const BoxBase b = decode_box(P, item);
-    const uint32_t group = fdiv(b.part, g.col_blocks);          // outer row
+    const uint32_t group = fdiv(b.part, g.col_blocks);          // group of outer rows
     const uint32_t cb = b.part - group * g.col_blocks.d;
+    const uint32_t row0 = group * g.rows_per_item;
+    const uint32_t nr = min(g.rows_per_item, g.rows - row0);
     const uint32_t a = cb * g.per_block;                       // first row of dimension K
     const uint32_t cnt = min(g.per_block, g.tab_inner.d - a);
     const uint32_t s1 = g.bx_s1, s2 = g.bx_s2.d;
     const uint32_t nseg = g.bx_nseg, nrng = g.bx_nrng;
     const uint32_t pitch = g.zip_seg_pitch;
-    int64_t r1, r2;
-    row_offsets(g, group, r1, r2, int(g.n_row_tab));
-    const int64_t so = b.o1 + r1 + int64_t(a) * s1;              // offset of every segment inside its source tile
-    const int64_t d0 = b.o2 + r2 + int64_t(a) * s2;              // offset of every range inside its target tile
-    const uint32_t mis = uint32_t(so) & 15u;                     // tiles start on 16-byte boundaries
     const uint32_t seg_bytes = cnt * s1, rng_bytes = cnt * s2;
+    const FastDiv nseg_div = g.bx_nseg_div, nrng_div = g.bx_nrng_div;
     if (tid == 0) {
         *wait_failed = 0;
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(nseg) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(nr * nseg) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     wait_for_previous_kernel();
-    for (uint32_t t = tid; t < nseg; t += nthreads) {
-        uint32_t rem = t, t1 = b.t1;
+    // one thread per source segment: (outer row, source tile of the super-box)
+    for (uint32_t t = tid; t < nr * nseg && CHK_IDX(t, uint32_t(kBoxSegments)); t += nthreads) {
+        const uint32_t r = fdiv(t, nseg_div);
+        uint32_t rem = t - r * nseg, t1 = b.t1;
         for (int q = int(g.bx_n) - 1; q >= 0; --q) {
             const uint32_t nx = fdiv(rem, g.bx_n1[q]);
             t1 += (rem - nx * g.bx_n1[q].d) * g.bx_ts1[q];
             rem = nx;
         }
+        int64_t r1, r2;
+        row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
+        const int64_t so = b.o1 + r1 + int64_t(a) * s1;          // offset of the row's segments inside their source tiles
+        const uint32_t mis = uint32_t(so) & 15u;                 // (tiles start on 16-byte boundaries)
         const char *src = P.src[t1] + so;
         const uint32_t bytes = (mis + seg_bytes + 15u) & ~15u;
         const bool safe = CHK_SRC(P, src - mis, bytes) && CHK_SMEM(t * pitch, bytes);
@@ -1373,9 +1378,9 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
                          ::"r"(smem_addr(tile) + t * pitch), "l"(src - mis), "r"(bytes), "r"(mbar)
                          : "memory");
     }
-    // while the copies are in flight: the place of every unit position of one target row, and the corner
-    // of every target tile
-    uint16_t *place = reinterpret_cast<uint16_t *>(tile + size_t(g.stage_pitch));
+    // while the copies are in flight: the place of every unit position of one target row, the corner of
+    // every target tile in every outer row, and where every outer row's ranges start in their tiles
+    uint16_t *place = reinterpret_cast<uint16_t *>(tile + size_t(g.stage_pitch) * g.rows_per_item);
     const uint32_t row_units = g.zip_lut_units;
     for (uint32_t p = tid; p < row_units; p += nthreads) {
         uint32_t rest = fdiv(p, g.bx_trail);
@@ -1387,10 +1392,15 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
             const uint32_t hi = fdiv(i, g.bx_c1[q]);
             off += hi * g.bx_seg[q] * pitch + (i - hi * g.bx_c1[q].d) * g.bx_st1[q];
         }
-        if (CHK_SMEM(g.stage_pitch + p * 2u, 2u)) place[p] = uint16_t(off);
+        if (CHK_SMEM(g.stage_pitch * g.rows_per_item + p * 2u, 2u)) place[p] = uint16_t(off);
     }
-    for (uint32_t t = tid; t < nrng && CHK_IDX(t, uint32_t(kBoxSegments)); t += nthreads) {
-        uint32_t rem = t, t2 = b.t2, off = mis;
+    for (uint32_t t = tid; t < nr * nrng && CHK_IDX(t, uint32_t(kBoxSegments)); t += nthreads) {
+        const uint32_t r = fdiv(t, nrng_div);
+        const uint32_t tt = t - r * nrng;
+        int64_t r1, r2;
+        row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
+        const uint32_t mis = uint32_t(b.o1 + r1 + int64_t(a) * s1) & 15u;
+        uint32_t rem = tt, t2 = b.t2, off = r * g.stage_pitch + mis;
         for (int q = int(g.bx_n) - 1; q >= 0; --q) {
             const uint32_t nx = fdiv(rem, g.bx_n2[q]);
             const uint32_t d = rem - nx * g.bx_n2[q].d;
@@ -1401,33 +1411,35 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
             off += hi * g.bx_seg[q] * pitch + (x - hi * g.bx_c1[q].d) * g.bx_st1[q];
         }
         base_of[t] = off;
-        tile_of[t] = t2 * fanout;
+        if (r == 0) tile_of[tt] = t2 * fanout;
+        if (tt == 0 && CHK_IDX(r, uint32_t(kBoxRows))) row_d0[r] = b.o2 + r2 + int64_t(a) * s2;
     }
     __syncthreads();
     if (!mbar_wait_bounded(mbar, 0, g.wait_polls)) {
         bulk_wait_ran_out(mbar, wait_failed, g.wait_polls);
         return;
     }
-    uint32_t head, chunks;
-    split_run(rng_bytes, d0, head, chunks);
-    // whole chunks: flat walk over (range, chunk), neighbouring lanes on neighbouring chunks
+    // whole chunks: flat walk over (outer row, range, chunk), neighbouring lanes on neighbouring chunks
     const uint32_t slots = g.zip_slots.d;
-    const uint32_t row_u = row_units;
-    for (uint32_t idx = tid; idx < nrng * slots; idx += nthreads) {
-        const uint32_t t = fdiv(idx, g.zip_slots);
-        const uint32_t c = idx - t * slots;
+    for (uint32_t idx = tid; idx < nr * nrng * slots; idx += nthreads) {
+        const uint32_t q = fdiv(idx, g.zip_slots);                // (outer row, range)
+        const uint32_t c = idx - q * slots;
+        const uint32_t r = fdiv(q, nrng_div);
+        const int64_t d0 = row_d0[r];
+        uint32_t head, chunks;
+        split_run(rng_bytes, d0, head, chunks);
         if (c >= chunks) continue;
         const uint32_t x = head + (c << 4);
-        uint32_t j = fdiv(x, g.bx_s2);
+        const uint32_t j = fdiv(x, g.bx_s2);
         uint32_t p = (x - j * s2) / uint32_t(sizeof(T));
-        uint32_t at = base_of[t] + j * s1;
+        uint32_t at = base_of[q] + j * s1;
         union {
             uint4 v;
             T t[kPer];
         } u;
 #pragma unroll
         for (int i = 0; i < kPer; ++i) {
-            if (p == row_u) {
+            if (p == row_units) {
                 p = 0;
                 at += s1;
             }
@@ -1435,27 +1447,31 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
             u.t[i] = CHK_SMEM(w, uint32_t(sizeof(T))) ? *reinterpret_cast<const T *>(tile + w) : T();
             ++p;
         }
-        char *const *dt = &P.dst[tile_of[t]];
+        char *const *dt = &P.dst[tile_of[q - r * nrng]];
         for (uint32_t f = 0; f < fanout; ++f)
             if (CHK_DST(P, dt[f] + d0 + x, 16)) st_stream(reinterpret_cast<uint4 *>(dt[f] + d0 + x), u.v);
     }
     // ragged ends of the ranges, unit by unit
     constexpr uint32_t kSlots = 16u / uint32_t(sizeof(T)) - 1u;
     if constexpr (kSlots > 0) {
-        const uint32_t toff = head + (chunks << 4);
-        for (uint32_t idx = tid; idx < nrng * kSlots * 2u; idx += nthreads) {
-            const uint32_t t = idx / (kSlots * 2u);
-            const uint32_t w = idx - t * (kSlots * 2u);
+        for (uint32_t idx = tid; idx < nr * nrng * kSlots * 2u; idx += nthreads) {
+            const uint32_t q = idx / (kSlots * 2u);
+            const uint32_t w = idx - q * (kSlots * 2u);
             const bool is_head = w < kSlots;
             const uint32_t slot = is_head ? w : w - kSlots;
+            const uint32_t r = fdiv(q, nrng_div);
+            const int64_t d0 = row_d0[r];
+            uint32_t head, chunks;
+            split_run(rng_bytes, d0, head, chunks);
+            const uint32_t toff = head + (chunks << 4);
             const uint32_t count = (is_head ? head : rng_bytes - toff) / uint32_t(sizeof(T));
             if (slot >= count) continue;
             const uint32_t x = (is_head ? 0u : toff) + slot * uint32_t(sizeof(T));
             const uint32_t j = fdiv(x, g.bx_s2);
-            const uint32_t at = base_of[t] + j * s1 + place[(x - j * s2) / uint32_t(sizeof(T))];
+            const uint32_t at = base_of[q] + j * s1 + place[(x - j * s2) / uint32_t(sizeof(T))];
             if (!CHK_SMEM(at, uint32_t(sizeof(T)))) continue;
             const T val = *reinterpret_cast<const T *>(tile + at);
-            char *const *dt = &P.dst[tile_of[t]];
+            char *const *dt = &P.dst[tile_of[q - r * nrng]];
             for (uint32_t f = 0; f < fanout; ++f)
                 if (CHK_DST(P, dt[f] + d0 + x, uint32_t(sizeof(T)))) *reinterpret_cast<T *>(dt[f] + d0 + x) = val;
         }
@@ -1469,14 +1485,15 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
         extern __shared__ __align__(128) unsigned char tile[];                                       \
         __shared__ uint32_t base_of[kBoxSegments];                                                   \
         __shared__ uint32_t tile_of[kBoxSegments];                                                   \
+        __shared__ int64_t row_d0[kBoxRows];                                                         \
         __shared__ __align__(8) unsigned long long mbar_storage;                                     \
         __shared__ unsigned int wait_failed;                                                         \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         const uint32_t mbar = smem_addr(&mbar_storage);                                              \
         switch (P.g.unit_bytes) {                                                                    \
-        case 16: box_body<uint4, NT>(P, tile, base_of, tile_of, mbar, &wait_failed); break;          \
-        case 8: box_body<uint2, NT>(P, tile, base_of, tile_of, mbar, &wait_failed); break;           \
-        default: box_body<uint32_t, NT>(P, tile, base_of, tile_of, mbar, &wait_failed); break;       \
+        case 16: box_body<uint4, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break;  \
+        case 8: box_body<uint2, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break;   \
+        default: box_body<uint32_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
         }                                                                                            \
     }
 
@@ -1612,7 +1629,7 @@ cudaError_t prepare_copy(int kernel, const CopyGeometry &geo, const char *const 
         pl.block = kBulkThreads;
         pl.smem = size_t(seg * geo.rows_per_item);
     } else if (geo.mode == kModeBox) {
-        pl.smem = size_t(geo.stage_pitch) + size_t(geo.zip_lut_units) * 2 + 16;
+        pl.smem = size_t(geo.stage_pitch) * geo.rows_per_item + size_t(geo.zip_lut_units) * 2 + 16;
     } else if (geo.mode == kModeZip) {
         // small items stored to one or two replicas: eight and more blocks fit an SM, and half as many threads
         // per block means half as many threads that decode the item and wait for its copies (measured

@@ -85,7 +85,8 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
     elif G["mode"] == 5:    # super-boxes: lcm(source tile, target tile) in the inner dimensions, staged by bulk copies
         nb = G["bx_n"]
-        assert 1 <= nb <= 3 and unit >= 4 and inner == span == mul == 1 and G["rows_per_item"] == 1
+        rpi = G["rows_per_item"]
+        assert 1 <= nb <= 3 and unit >= 4 and inner == span == mul == 1 and 1 <= rpi <= 32
         c1, c2, n1, n2 = G["bx_c1"], G["bx_c2"], G["bx_n1"], G["bx_n2"]
         trail = G["bx_trail"] * unit
         for q in range(nb):
@@ -93,7 +94,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
             assert c1[q] * n1[q] == c2[q] * n2[q] == max(c1[q], c2[q])
             assert G["bx_st1"][q] == trail * _prod(c1[q + 1:]) and G["bx_seg"][q] == _prod(n1[q + 1:])
         assert G["bx_s1"] == trail * _prod(c1) and G["bx_s2"] == trail * _prod(c2)
-        assert G["bx_nseg"] == _prod(n1) <= 64 and G["bx_nrng"] == _prod(n2) <= 64
+        assert G["bx_nseg"] == _prod(n1) and G["bx_nrng"] == _prod(n2) and rpi * max(G["bx_nseg"], G["bx_nrng"]) <= 256
         assert run == trail and min(c1[-1], c2[-1]) == 1     # the last inner dimension counts runs
         nK, cnt = G["tab_inner"], G["per_block"]
         n_out = G["n_row_tab"]
@@ -102,10 +103,10 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         if nK > 1:
             assert G["row_b1"][n_out] == G["bx_s1"] and G["row_b2"][n_out] == G["bx_s2"]   # rows of K are contiguous
         assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= cnt * G["bx_s1"] + 30
-        assert G["stage_pitch"] == G["zip_seg_pitch"] * G["bx_nseg"] <= 38 * 1024
+        assert G["stage_pitch"] == G["zip_seg_pitch"] * G["bx_nseg"] and G["stage_pitch"] * rpi <= 38 * 1024
         assert G["zip_lut_units"] * unit == G["bx_s2"] and G["zip_lut_units"] <= 4096
         assert G["zip_slots"] >= cnt * G["bx_s2"] // 16 + 1
-        assert G["items_per_box"] == tab_rows * G["col_blocks"]
+        assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
         # the digits of the inner dimensions count super-boxes: unit_mul boxes of the gcd size each
         assert _prod(unit_mul) >= 1
     elif G["mode"] == 0:    # rows: aligned runs of at most 256 chunks
@@ -194,39 +195,46 @@ def check_box_items(L: dict, src_bufs, dst_bufs):
             o1 += b1 * G["unit_b1"][u]
             o2 += b2 * G["unit_b2"][u]
         group, cb = divmod(part, G["col_blocks"])
-        r1 = r2 = 0
-        rem = group
-        for q in range(n_out - 1, -1, -1):
-            rem, dg = divmod(rem, G["row_n"][q])
-            r1 += dg * G["row_b1"][q]
-            r2 += dg * G["row_b2"][q]
         a = cb * G["per_block"]
         cnt = min(G["per_block"], G["tab_inner"] - a)
-        so, d0 = o1 + r1 + a * s1, o2 + r2 + a * s2
-        mis = so % 16
-        stage = np.zeros(G["stage_pitch"] + 64, dtype=np.uint8)
-        for t in range(G["bx_nseg"]):
-            rem, tile = t, t1
-            for q in range(nb - 1, -1, -1):
-                rem, d = divmod(rem, n1[q])
-                tile += d * G["bx_ts1"][q]
-            src = src_bufs(L["src_holder"][tile])
-            assert so + cnt * s1 <= src.shape[0]
-            stage[t * pitch + mis:t * pitch + mis + cnt * s1] = src[so:so + cnt * s1]
-        for t in range(G["bx_nrng"]):
-            rem, tile, base = t, t2, mis
-            for q in range(nb - 1, -1, -1):
-                rem, d = divmod(rem, n2[q])
-                tile += d * G["bx_ts2"][q]
-                hi, lo = divmod(d * c2[q], c1[q])
-                base += hi * G["bx_seg"][q] * pitch + lo * G["bx_st1"][q]
-            x = np.arange(0, cnt * s2, unit, dtype=np.int64)
-            at = base + (x // s2) * s1 + place[(x % s2) // unit]
-            got = stage[at[:, None] + np.arange(unit)[None, :]].reshape(-1)
-            for f in range(fan):
-                dst = dst_bufs(L["dst_devs"][tile * fan + f])
-                assert d0 + cnt * s2 <= dst.shape[0]
-                assert np.array_equal(dst[d0:d0 + cnt * s2], got), (item, t, f)
+        row0 = group * G["rows_per_item"]
+        nr = min(G["rows_per_item"], G["rows"] - row0)
+        stage = np.zeros(G["stage_pitch"] * G["rows_per_item"] + 64, dtype=np.uint8)
+        offs = []
+        for r in range(nr):
+            r1 = r2 = 0
+            rem = row0 + r
+            for q in range(n_out - 1, -1, -1):
+                rem, dg = divmod(rem, G["row_n"][q])
+                r1 += dg * G["row_b1"][q]
+                r2 += dg * G["row_b2"][q]
+            so, d0 = o1 + r1 + a * s1, o2 + r2 + a * s2
+            offs.append((so % 16, d0))
+            for t in range(G["bx_nseg"]):
+                rem, tile = t, t1
+                for q in range(nb - 1, -1, -1):
+                    rem, d = divmod(rem, n1[q])
+                    tile += d * G["bx_ts1"][q]
+                src = src_bufs(L["src_holder"][tile])
+                assert so + cnt * s1 <= src.shape[0]
+                at = (r * G["bx_nseg"] + t) * pitch + so % 16
+                stage[at:at + cnt * s1] = src[so:so + cnt * s1]
+        for r in range(nr):
+            mis, d0 = offs[r]
+            for t in range(G["bx_nrng"]):
+                rem, tile, base = t, t2, r * G["stage_pitch"] + mis
+                for q in range(nb - 1, -1, -1):
+                    rem, d = divmod(rem, n2[q])
+                    tile += d * G["bx_ts2"][q]
+                    hi, lo = divmod(d * c2[q], c1[q])
+                    base += hi * G["bx_seg"][q] * pitch + lo * G["bx_st1"][q]
+                x = np.arange(0, cnt * s2, unit, dtype=np.int64)
+                at = base + (x // s2) * s1 + place[(x % s2) // unit]
+                got = stage[at[:, None] + np.arange(unit)[None, :]].reshape(-1)
+                for f in range(fan):
+                    dst = dst_bufs(L["dst_devs"][tile * fan + f])
+                    assert d0 + cnt * s2 <= dst.shape[0]
+                    assert np.array_equal(dst[d0:d0 + cnt * s2], got), (item, r, t, f)
 
 
 def run_plan(desc: dict, src_tiles):
