@@ -116,7 +116,8 @@ struct CopyGeometry {
     FastDiv zip_cpr;                 // kModeZip: chunk slots per run in the by-range walk; d = 0: walk not used
     FastDiv zip_period;              // kModeZip: chunks after which the chunk -> units map repeats (d = 0: path not used)
     uint32_t zip_period_rows;        // kModeZip: rows of the zipped digit that one period spans
-    uint32_t zip_width;              // kModeZip: lanes that walk one table row together (a multiple of zip_period)
+    uint32_t zip_width;              // kModeZip: lanes that walk one table row together (a multiple of zip_period);
+                                     // kModeBox: lanes that walk one target range together (a power of two, at least a warp)
     uint32_t zip_lut_units;          // kModeZip: units of the longest range when their places are tabulated in shared memory (0: not)
     uint32_t zip_tile_fastest;       // kModeZip, long source rows: 1 = neighbouring lanes write to neighbouring target tiles
     FastDiv gl_n[kMaxGatherLevels];  // kModeGather: extents of those row digits, innermost first
@@ -151,6 +152,7 @@ struct CopyGeometry {
     uint32_t bx_s1;                  //           ... in a source segment
     uint32_t bx_nseg, bx_nrng;       // kModeBox: source segments / target ranges of one outer row of an item
     FastDiv bx_nseg_div, bx_nrng_div;
+    FastDiv bx_row_units_div;        // kModeBox: division by the units of one target row (zip_lut_units)
     uint32_t wait_polls;             // bulk-copy kernels: mbarrier polls before a block gives up (bounded wait)
     uint32_t test_extra_tx;          // test only: bytes announced on the mbarrier beyond what the copies deliver, so
                                      // that every copy lands but the phase never completes (0 in every real plan)

@@ -428,7 +428,15 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.zip_seg_pitch = uint32_t(round_up(bx_cnt * bx_s1, 16) + 32);
         G.stage_pitch = uint32_t(G.zip_seg_pitch * n1);          // one outer row of the item
         G.zip_lut_units = uint32_t(bx_s2 / vec);
+        G.bx_row_units_div = make_div(uint32_t(bx_s2 / vec));
         G.zip_slots = make_div(uint32_t(bx_cnt * bx_s2 / 16 + 1));
+        {
+            // lanes per range: about four chunks each, a whole number of warps, no more groups than ranges
+            const i64 chunks = bx_cnt * bx_s2 / 16, ranges = bx_rpi * n2;
+            i64 w = 32;
+            while (w < kBlockThreads && (w * 4 < chunks || kBlockThreads / w > ranges)) w *= 2;
+            G.zip_width = uint32_t(w);
+        }
         G.gl_m = make_div(1);
         ipb = (tab_rows + bx_rpi - 1) / bx_rpi * ncb;
     } else if (zip_n > 0) {

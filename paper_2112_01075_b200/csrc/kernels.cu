@@ -1325,6 +1325,12 @@ REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
 // byte stride, which is additive in "corner index + index inside the tile" because in every inner
 // dimension one tile extent divides the other.  The block tabulates place[] (one target row) and base[]
 // while its copies are in flight; a unit then costs a table read and the read of the unit.
+// The kernel is bound by instruction issue, not by memory, so work that every thread would repeat is
+// given to one warp: warp 0 alone decodes the item (unit digits -> tiles and offsets), issues the bulk
+// copies and tabulates base[] and the range offsets, while the other warps tabulate place[]; the walk
+// over the ranges then reads everything item-specific from those tables.  Lanes work in groups of
+// zip_width (a power of two) that share out the ranges; a lane strides through its range's chunks and
+// keeps (row, position in row) by adding a constant per step instead of dividing.
 template <typename T, int NT>
 __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char *tile, uint32_t *base_of,
                                          uint32_t *tile_of, int64_t *row_d0, uint32_t mbar, unsigned int *wait_failed)
@@ -1336,9 +1342,11 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
     const uint32_t fanout = g.fanout;
     const uint32_t item = blockIdx.x;
     if (item >= g.n_items) return;
-    const BoxBase b = decode_box(P, item);
-    const uint32_t group = fdiv(b.part, g.col_blocks);          // group of outer rows
-    const uint32_t cb = b.part - group * g.col_blocks.d;
+    // which part of its box the item is (cheap, every thread): group of outer rows, block of rows of K
+    const uint32_t slow = fdiv(item, g.items_per_box);           // inner_n = fast_boxes = 1 in this mode
+    const uint32_t part = item - slow * g.items_per_box.d;
+    const uint32_t group = fdiv(part, g.col_blocks);
+    const uint32_t cb = part - group * g.col_blocks.d;
     const uint32_t row0 = group * g.rows_per_item;
     const uint32_t nr = min(g.rows_per_item, g.rows - row0);
     const uint32_t a = cb * g.per_block;                       // first row of dimension K
@@ -1347,109 +1355,140 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
     const uint32_t nseg = g.bx_nseg, nrng = g.bx_nrng;
     const uint32_t pitch = g.zip_seg_pitch;
     const uint32_t seg_bytes = cnt * s1, rng_bytes = cnt * s2;
-    const FastDiv nseg_div = g.bx_nseg_div, nrng_div = g.bx_nrng_div;
+    const uint32_t row_units = g.zip_lut_units;
+    uint16_t *place = reinterpret_cast<uint16_t *>(tile + size_t(g.stage_pitch) * g.rows_per_item);
     if (tid == 0) {
         *wait_failed = 0;
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(nr * nseg) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    wait_for_previous_kernel();
-    // one thread per source segment: (outer row, source tile of the super-box)
-    for (uint32_t t = tid; t < nr * nseg && CHK_IDX(t, uint32_t(kBoxSegments)); t += nthreads) {
-        const uint32_t r = fdiv(t, nseg_div);
-        uint32_t rem = t - r * nseg, t1 = b.t1;
-        for (int q = int(g.bx_n) - 1; q >= 0; --q) {
-            const uint32_t nx = fdiv(rem, g.bx_n1[q]);
-            t1 += (rem - nx * g.bx_n1[q].d) * g.bx_ts1[q];
-            rem = nx;
+    if (tid < 32u) {
+        const BoxBase b = decode_box(P, item);
+        wait_for_previous_kernel();
+        // one lane per source segment: (outer row, source tile of the super-box)
+        for (uint32_t t = tid; t < nr * nseg && CHK_IDX(t, uint32_t(kBoxSegments)); t += 32u) {
+            const uint32_t r = fdiv(t, g.bx_nseg_div);
+            uint32_t rem = t - r * nseg, t1 = b.t1;
+            for (int q = int(g.bx_n) - 1; q >= 0; --q) {
+                const uint32_t nx = fdiv(rem, g.bx_n1[q]);
+                t1 += (rem - nx * g.bx_n1[q].d) * g.bx_ts1[q];
+                rem = nx;
+            }
+            int64_t r1, r2;
+            row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
+            const int64_t so = b.o1 + r1 + int64_t(a) * s1;      // offset of the row's segments inside their source tiles
+            const uint32_t mis = uint32_t(so) & 15u;             // (tiles start on 16-byte boundaries)
+            const char *src = P.src[t1] + so;
+            const uint32_t bytes = (mis + seg_bytes + 15u) & ~15u;
+            const bool safe = CHK_SRC(P, src - mis, bytes) && CHK_SMEM(t * pitch, bytes);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                         ::"r"(mbar), "r"((safe ? bytes : 0u) + (t == 0 ? g.test_extra_tx : 0u)) : "memory");
+            if (safe)
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_addr(tile) + t * pitch), "l"(src - mis), "r"(bytes), "r"(mbar)
+                             : "memory");
         }
-        int64_t r1, r2;
-        row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
-        const int64_t so = b.o1 + r1 + int64_t(a) * s1;          // offset of the row's segments inside their source tiles
-        const uint32_t mis = uint32_t(so) & 15u;                 // (tiles start on 16-byte boundaries)
-        const char *src = P.src[t1] + so;
-        const uint32_t bytes = (mis + seg_bytes + 15u) & ~15u;
-        const bool safe = CHK_SRC(P, src - mis, bytes) && CHK_SMEM(t * pitch, bytes);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                     ::"r"(mbar), "r"((safe ? bytes : 0u) + (t == 0 ? g.test_extra_tx : 0u)) : "memory");
-        if (safe)
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_addr(tile) + t * pitch), "l"(src - mis), "r"(bytes), "r"(mbar)
-                         : "memory");
-    }
-    // while the copies are in flight: the place of every unit position of one target row, the corner of
-    // every target tile in every outer row, and where every outer row's ranges start in their tiles
-    uint16_t *place = reinterpret_cast<uint16_t *>(tile + size_t(g.stage_pitch) * g.rows_per_item);
-    const uint32_t row_units = g.zip_lut_units;
-    for (uint32_t p = tid; p < row_units; p += nthreads) {
-        uint32_t rest = fdiv(p, g.bx_trail);
-        uint32_t off = (p - rest * g.bx_trail.d) * uint32_t(sizeof(T));
-        for (int q = int(g.bx_n) - 1; q >= 0; --q) {
-            const uint32_t nx = fdiv(rest, g.bx_c2[q]);
-            const uint32_t i = rest - nx * g.bx_c2[q].d;
-            rest = nx;
-            const uint32_t hi = fdiv(i, g.bx_c1[q]);
-            off += hi * g.bx_seg[q] * pitch + (i - hi * g.bx_c1[q].d) * g.bx_st1[q];
+        // the corner of every target tile in every outer row, and where every outer row's ranges start
+        for (uint32_t t = tid; t < nr * nrng && CHK_IDX(t, uint32_t(kBoxSegments)); t += 32u) {
+            const uint32_t r = fdiv(t, g.bx_nrng_div);
+            const uint32_t tt = t - r * nrng;
+            int64_t r1, r2;
+            row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
+            const uint32_t mis = uint32_t(b.o1 + r1 + int64_t(a) * s1) & 15u;
+            uint32_t rem = tt, t2 = b.t2, off = r * g.stage_pitch + mis;
+            for (int q = int(g.bx_n) - 1; q >= 0; --q) {
+                const uint32_t nx = fdiv(rem, g.bx_n2[q]);
+                const uint32_t d = rem - nx * g.bx_n2[q].d;
+                rem = nx;
+                t2 += d * g.bx_ts2[q];
+                const uint32_t x = d * g.bx_c2[q].d;             // index of the tile's corner inside the super-box
+                const uint32_t hi = fdiv(x, g.bx_c1[q]);
+                off += hi * g.bx_seg[q] * pitch + (x - hi * g.bx_c1[q].d) * g.bx_st1[q];
+            }
+            base_of[t] = off;
+            if (r == 0) tile_of[tt] = t2 * fanout;
+            if (tt == 0 && CHK_IDX(r, uint32_t(kBoxRows))) row_d0[r] = b.o2 + r2 + int64_t(a) * s2;
         }
-        if (CHK_SMEM(g.stage_pitch * g.rows_per_item + p * 2u, 2u)) place[p] = uint16_t(off);
-    }
-    for (uint32_t t = tid; t < nr * nrng && CHK_IDX(t, uint32_t(kBoxSegments)); t += nthreads) {
-        const uint32_t r = fdiv(t, nrng_div);
-        const uint32_t tt = t - r * nrng;
-        int64_t r1, r2;
-        row_offsets(g, row0 + r, r1, r2, int(g.n_row_tab));
-        const uint32_t mis = uint32_t(b.o1 + r1 + int64_t(a) * s1) & 15u;
-        uint32_t rem = tt, t2 = b.t2, off = r * g.stage_pitch + mis;
-        for (int q = int(g.bx_n) - 1; q >= 0; --q) {
-            const uint32_t nx = fdiv(rem, g.bx_n2[q]);
-            const uint32_t d = rem - nx * g.bx_n2[q].d;
-            rem = nx;
-            t2 += d * g.bx_ts2[q];
-            const uint32_t x = d * g.bx_c2[q].d;                 // index of the tile's corner inside the super-box
-            const uint32_t hi = fdiv(x, g.bx_c1[q]);
-            off += hi * g.bx_seg[q] * pitch + (x - hi * g.bx_c1[q].d) * g.bx_st1[q];
+    } else {
+        // the place of every unit position of one target row (depends on the launch only)
+        for (uint32_t p = tid - 32u; p < row_units; p += nthreads - 32u) {
+            uint32_t rest = fdiv(p, g.bx_trail);
+            uint32_t off = (p - rest * g.bx_trail.d) * uint32_t(sizeof(T));
+            for (int q = int(g.bx_n) - 1; q >= 0; --q) {
+                const uint32_t nx = fdiv(rest, g.bx_c2[q]);
+                const uint32_t i = rest - nx * g.bx_c2[q].d;
+                rest = nx;
+                const uint32_t hi = fdiv(i, g.bx_c1[q]);
+                off += hi * g.bx_seg[q] * pitch + (i - hi * g.bx_c1[q].d) * g.bx_st1[q];
+            }
+            if (CHK_SMEM(g.stage_pitch * g.rows_per_item + p * 2u, 2u)) place[p] = uint16_t(off);
         }
-        base_of[t] = off;
-        if (r == 0) tile_of[tt] = t2 * fanout;
-        if (tt == 0 && CHK_IDX(r, uint32_t(kBoxRows))) row_d0[r] = b.o2 + r2 + int64_t(a) * s2;
+        wait_for_previous_kernel();
     }
     __syncthreads();
     if (!mbar_wait_bounded(mbar, 0, g.wait_polls)) {
         bulk_wait_ran_out(mbar, wait_failed, g.wait_polls);
         return;
     }
-    // whole chunks: flat walk over (outer row, range, chunk), neighbouring lanes on neighbouring chunks
-    const uint32_t slots = g.zip_slots.d;
-    for (uint32_t idx = tid; idx < nr * nrng * slots; idx += nthreads) {
-        const uint32_t q = fdiv(idx, g.zip_slots);                // (outer row, range)
-        const uint32_t c = idx - q * slots;
-        const uint32_t r = fdiv(q, nrng_div);
+    // whole chunks: groups of W lanes share out the ranges (outer row, target tile)
+    const uint32_t W = g.zip_width;                              // power of two, 32 .. block size
+    const uint32_t n_groups = nthreads / W;
+    const uint32_t lane = tid & (W - 1u);
+    const uint32_t step_units = W * uint32_t(kPer);              // units between a lane's consecutive chunks
+    const uint32_t dj = fdiv(step_units, g.bx_row_units_div);
+    const uint32_t dp = step_units - dj * row_units;
+    for (uint32_t q = tid / W; q < nr * nrng; q += n_groups) {
+        const uint32_t r = fdiv(q, g.bx_nrng_div);
         const int64_t d0 = row_d0[r];
         uint32_t head, chunks;
         split_run(rng_bytes, d0, head, chunks);
-        if (c >= chunks) continue;
-        const uint32_t x = head + (c << 4);
-        const uint32_t j = fdiv(x, g.bx_s2);
-        uint32_t p = (x - j * s2) / uint32_t(sizeof(T));
-        uint32_t at = base_of[q] + j * s1;
-        union {
-            uint4 v;
-            T t[kPer];
-        } u;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            if (p == row_units) {
-                p = 0;
-                at += s1;
-            }
-            const uint32_t w = at + place[p];
-            u.t[i] = CHK_SMEM(w, uint32_t(sizeof(T))) ? *reinterpret_cast<const T *>(tile + w) : T();
-            ++p;
-        }
+        if (lane >= chunks) continue;
         char *const *dt = &P.dst[tile_of[q - r * nrng]];
-        for (uint32_t f = 0; f < fanout; ++f)
-            if (CHK_DST(P, dt[f] + d0 + x, 16)) st_stream(reinterpret_cast<uint4 *>(dt[f] + d0 + x), u.v);
+        char *d_first = dt[0] + d0 + head;
+        const uint32_t base = base_of[q];
+        const uint32_t x0 = head + (lane << 4);
+        uint32_t j = fdiv(x0, g.bx_s2);
+        uint32_t p = (x0 - j * s2) / uint32_t(sizeof(T));
+        for (uint32_t c = lane; c < chunks; c += W) {
+            const uint32_t at = base + j * s1;
+            union {
+                uint4 v;
+                T t[kPer];
+            } u;
+            if (p + uint32_t(kPer) <= row_units) {
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    const uint32_t w = at + place[p + uint32_t(i)];
+                    u.t[i] = CHK_SMEM(w, uint32_t(sizeof(T))) ? *reinterpret_cast<const T *>(tile + w) : T();
+                }
+            } else {
+                uint32_t pp = p, aa = at;                        // the chunk runs over the end of a row of K
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    if (pp == row_units) {
+                        pp = 0;
+                        aa += s1;
+                    }
+                    const uint32_t w = aa + place[pp];
+                    u.t[i] = CHK_SMEM(w, uint32_t(sizeof(T))) ? *reinterpret_cast<const T *>(tile + w) : T();
+                    ++pp;
+                }
+            }
+            if (fanout == 1) {
+                if (CHK_DST(P, d_first + (c << 4), 16)) st_stream(reinterpret_cast<uint4 *>(d_first + (c << 4)), u.v);
+            } else {
+                for (uint32_t f = 0; f < fanout; ++f)
+                    if (CHK_DST(P, dt[f] + d0 + head + (c << 4), 16))
+                        st_stream(reinterpret_cast<uint4 *>(dt[f] + d0 + head + (c << 4)), u.v);
+            }
+            p += dp;
+            j += dj;
+            if (p >= row_units) {
+                p -= row_units;
+                ++j;
+            }
+        }
     }
     // ragged ends of the ranges, unit by unit
     constexpr uint32_t kSlots = 16u / uint32_t(sizeof(T)) - 1u;
@@ -1459,7 +1498,7 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
             const uint32_t w = idx - q * (kSlots * 2u);
             const bool is_head = w < kSlots;
             const uint32_t slot = is_head ? w : w - kSlots;
-            const uint32_t r = fdiv(q, nrng_div);
+            const uint32_t r = fdiv(q, g.bx_nrng_div);
             const int64_t d0 = row_d0[r];
             uint32_t head, chunks;
             split_run(rng_bytes, d0, head, chunks);
