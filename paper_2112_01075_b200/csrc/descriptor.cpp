@@ -261,7 +261,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // contiguous pieces on both sides long), times a block of rows of the dimension K just outside them.
     // Source bytes: one contiguous segment per source tile touched; target bytes: one contiguous range
     // per target tile touched.  Chosen (tuning value "box": 0 never, 2 wherever it applies) for short
-    // runs where the zip kernels do not apply or would zip a digit of only a few rows.
+    // runs where the zip kernels do not apply or would produce target ranges of a few hundred bytes.
     struct BoxDim {
         int k;
         i64 c1, c2, E;
@@ -321,7 +321,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                                              : std::min(s1, s2) * cnt >= 256 && sup * cnt * rpi >= kItemBytes / 4;
             // default policy: where the unit walk or the gather walk would run, and where the zip kernels
             // would zip a digit of fewer than 16 rows
-            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_n < 16 && run_bytes < 512
+            // (measured on the odd-shape sweep: against the unit walk and the gather walk 1.5-1.7x; against the
+            // zip kernels 1.2-1.26x where their target ranges are short -- each range pays for its own ragged
+            // head and tail --, 0.8-0.9x where they are long)
+            const i64 zip_range = zip_n * (m2[kp] > 1 ? std::max(m1[kp], m2[kp]) * run_bytes : run_bytes);
+            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_range < 768
                                                             : run_bytes < 256 && (g_levels >= 0 || !G.aligned));
             if (!fits || !worth || !wanted || sup > (1ll << 30)) bxK = -2;
         }
