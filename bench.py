@@ -637,6 +637,10 @@ def sweep_rows(torch, api, pairs, flags, fill_seed):
                      "variants": [i.variant for i in li],
                      "fanout": max(i.fanout for i in li), "eff_bytes": eff, "us": round(ms * 1e3, 1),
                      "gbs": round(eff / (ms * 1e-3) / 1e9, 1),
+                     # what the launches actually move (every intermediate is written and read again when the
+                     # sequence runs collective by collective), per second: the efficiency of the kernels
+                     "traffic_gbs": round(sum(i.bytes_read + i.bytes_written for i in li) / (ms * 1e-3) / 1e9, 1),
+                     "launch_runs": [i.run_bytes for i in li], "kernels": plan.launch_kernels(),
                      "scratch_per_device": plan.scratch_bytes_per_device, "plan_cost_elems": plan.cost})
         del src, dst, owned, scratch, call, plan
         torch.cuda.empty_cache()
@@ -670,6 +674,8 @@ def run_sweep(args):
             "plan_cost_elems_total": sum(r["plan_cost_elems"] for r in rows), "geomean_gbs": round(geomean(g), 1),
             "min_gbs": min(g), "max_gbs": max(g), "median_gbs": statistics.median(g),
             "total_gbs": round(sum(r["eff_bytes"] for r in rows) / sum(r["us"] * 1e-6 for r in rows) / 1e9, 1),
+            "traffic_geomean_gbs": round(geomean([r["traffic_gbs"] for r in rows]), 1),
+            "traffic_min_gbs": min(r["traffic_gbs"] for r in rows),
             "peak": peak, "peak_source": how, "pairs_below_70pct_of_peak": sum(x < 0.7 * peak for x in g)}
     if args.dump:
         with open(args.dump, "w") as f:

@@ -151,7 +151,7 @@ def test_factor_decomposition_example():
 
 def test_oversharding_example_cost_bounds():
     """Mesh {x:4, y:2, z:4}: the printed sequences cost 512 and 384; the search may not do worse than
-    the better one on the weak graph (the final permutation is not a graph edge, Section 7.3)."""
+    the better one on the weak graph (the search of Section 7.3 gives the final permutation no edge weight)."""
     mesh, gshape = (4, 2, 4), (8, 8, 8, 4)
     src, dst = (gshape, ((1, 0), (), (), ())), (gshape, ((), (1,), (0,), ()))
     d = check_plan(mesh, src, dst, 4)
