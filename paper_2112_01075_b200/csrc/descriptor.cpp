@@ -192,7 +192,11 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         for (int k = 0; k < r; ++k) nt *= b.ntiles[k];
         fan = p.n_devices / nt;
     }
-    const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 4 ? 8 : fan >= 2 ? 16 : 32) * 1024;
+    // (the 256-thread kernels: 32 KiB up to fan-out 3, 16 KiB up to 7, 8 KiB from 8.  Every thread of a block
+    // decodes the item, so small items pay for it dearly: measured on eleven fan-out problems of the odd-shape
+    // sweep, 16 -> 32 KiB at fan-out 2: 4.34-5.07 -> 5.12-6.51 TB/s; 8 -> 16 KiB at fan-out 4: 4.69-5.57 ->
+    // 6.07-6.28; at fan-out 8, 8 KiB stays best: 5.74 against 5.17)
+    const i64 kItemBytes = kItemKb > 0 ? kItemKb * 1024 : (fan >= 8 ? 8 : fan >= 4 ? 16 : 32) * 1024;
     // Items of the plain bulk-copy kernels: measured best at 20 KiB (12 / 6 KiB for fan-out >= 2 / >= 4) once
     // the kernels wait for their predecessor only after decoding the item -- finer tail, more blocks ready
     // behind the wait.
