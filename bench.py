@@ -433,6 +433,8 @@ def run_ours(args):
             torch.cuda.empty_cache()
     if rank == 0 and world == 1 and args.fuse == "adjacent" and not args.lean and not args.no_configs:
         line["configs"] = run_configs(torch, api, gen)
+    if rank == 0 and world == 1 and args.others:
+        line["others"] = run_others(torch, api, gen, args)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:

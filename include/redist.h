@@ -171,6 +171,8 @@ void redist_plan_cache_clear(void);
  *   "item_kb"            0..1024 KiB read per work item; 0 (default) = 32 / 16 / 8 by fan-out, and 20 / 12 / 6
  *                               in the bulk-copy kernels
  *   "pdl"                0/1    1: kernels use programmatic dependent launch (default); 0: plain stream order
+ *   "nvtx"               0/1    1: redist_execute and redist_execute_static wrap every kernel launch in an NVTX
+ *                               range named after the collective, for timeline profilers (default 0)
  *   "step_latency"       >= 0   elements added to the cost of every collective while searching: small
  *                               transfers are bound by per-step latency, not by bytes (Section 8, the
  *                               third research question); 0 (default) is the paper's cost model

@@ -1,5 +1,6 @@
 // The C boundary: plan creation (with the plan cache and the tuning values), execution and queries.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cstring>
@@ -76,6 +77,7 @@ const TuningName kTuningNames[] = {
     {"zip_by_range_slots", &Tuning::zip_by_range_slots, 1, 1 << 20},
     {"item_kb", &Tuning::item_kb, 0, 1024},
     {"pdl", &Tuning::pdl, 0, 1},
+    {"nvtx", &Tuning::nvtx, 0, 1},
     {"step_latency", &Tuning::step_latency, 0, int64_t(1) << 50},
     {"wait_polls", &Tuning::wait_polls, 1, int64_t(1) << 30},
     {"test_extra_tx", &Tuning::test_extra_tx, 0, 1 << 20},
@@ -173,11 +175,17 @@ redist_status run_plan(const Plan &p, const void *const *src_shards, void *const
     if (rc != REDIST_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     PreparedLaunch pl;
+    static const char *const kNames[] = {"redist dynslice", "redist alltoall", "redist allgather", "redist allpermute",
+                                         "redist copy", "redist fused", "redist naive gather", "redist naive slice"};
     for (const Launch &L : p.launches) {
         if (L.geo.n_items == 0) continue;
         rc = prepare_launch(p, L, src_shards, dst_shards, static_cast<char *>(scratch), pl);
         if (rc != REDIST_OK) return rc;
+        // an NVTX range around every launch names the step for a timeline profiler (tuning value "nvtx")
+        const bool mark = p.tuning.nvtx != 0;
+        if (mark) nvtxRangePushA(kNames[L.kernel >= 0 && L.kernel < 8 ? L.kernel : 5]);
         cudaError_t ce = launch_prepared(pl, stream);
+        if (mark) nvtxRangePop();
         if (ce != cudaSuccess) {
             tl_cuda_error = int(ce);
             return REDIST_ECUDA;
