@@ -485,8 +485,13 @@ def test_execute_can_be_captured_in_a_cuda_graph_and_replayed():
             plan.execute(d_src, d_dst, scratch, side)          # warm-up outside the capture
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
+        bound = plan.bind([t.data_ptr() for t in d_src], [t.data_ptr() for t in d_dst],
+                          scratch.data_ptr() if scratch is not None else 0, plan.scratch_bytes)
         with torch.cuda.graph(g, stream=side):
-            plan.execute(d_src, d_dst, scratch, torch.cuda.current_stream())
+            if flags == api.FUSE_NONE:      # the bound form is launches only: it captures the same way
+                bound(torch.cuda.current_stream().cuda_stream)
+            else:
+                plan.execute(d_src, d_dst, scratch, torch.cuda.current_stream())
         for seed in (11, 12):
             _, _, tiles, expect = make_case(w, seed=seed)
             for t, h in zip(d_src, tiles):
