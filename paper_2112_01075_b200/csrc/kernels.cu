@@ -33,6 +33,9 @@
 //                target in whole 16-byte chunks and fetches every unit from its computed source.
 //   kModeZip     the same interleaving (either direction) when the row digit next to it is contiguous
 //                on both sides: source segments staged in shared memory by bulk copies (zip_body).
+//   kModeBox     short runs that interleave along several dimensions at once: the item is widened to a
+//                super-box that covers whole tiles of both sides in those dimensions, staged in shared
+//                memory segment by segment and written out range by range (box_body).
 // Index decoding uses multiply-shift division by host-computed constants; the per-item decode (box ->
 // tiles and base offsets) is amortised over ~32 KiB of data.  Every kernel starts with
 // griddepcontrol.launch_dependents and places griddepcontrol.wait after the decode of its first work
