@@ -206,8 +206,8 @@ void redist_tuning_reset(void);
  *                   that is 0.  Contents are undefined afterwards.
  *   cuda_stream     a cudaStream_t (NULL = default stream) on the current device
  * Ownership: all buffers and the stream belong to the caller.  The call allocates nothing, on the
- * host or on the device (pointer tables and the kernel parameter block live on the call's stack,
- * about 100 KiB), copies no table to the device (tables travel as kernel parameters) and does not
+ * host or on the device (pointer tables and the kernel parameter block live on the call's stack:
+ * about 8 KiB for plans of up to 64 virtual devices, about 100 KiB beyond), copies no table to the device (tables travel as kernel parameters) and does not
  * synchronize.  A plan may be executed from several host threads at once on different streams and
  * buffers.
  * Errors: EINVAL, ESCRATCH, EALIGN (pointers must be multiples of redist_plan_alignment),

@@ -25,6 +25,7 @@ thread_local int tl_cuda_error = 0;
 struct redist_bound_s {
     std::shared_ptr<const redist::Plan> ref;
     std::vector<redist::PreparedLaunch> launches;
+    std::vector<std::vector<max_align_t>> params;     // one parameter block per launch
 };
 
 namespace {
@@ -111,14 +112,17 @@ std::string cache_key(int32_t n_mesh_axes, const int64_t *mesh_shape, const redi
 }
 
 // Buffer checks shared by every execute entry point: pointers present and aligned, destination and
-// scratch ranges disjoint from each other and from every source.  Allocates nothing.
+// scratch ranges disjoint from each other and from every source.  Allocates nothing; CAP bounds the
+// number of virtual devices (the range table lives on the stack).
+template <int CAP>
 redist_status check_buffers(const Plan &p, const void *const *src_shards, void *const *dst_shards, const void *scratch,
                             size_t scratch_range)
 {
     const int N = p.n_devices;
+    if (N > CAP) return REDIST_EINTERNAL;
     const uintptr_t amask = uintptr_t(p.alignment) - 1;
     const i64 sb = p.local_src * p.elem_bytes, db = p.local_dst * p.elem_bytes;
-    Range ranges[2 * REDIST_MAX_DEVICES + 1];
+    Range ranges[2 * CAP + 1];
     int n = 0;
     for (int d = 0; d < N; ++d) {
         if (!src_shards[d] || !dst_shards[d]) return REDIST_EINVAL;
@@ -134,9 +138,11 @@ redist_status check_buffers(const Plan &p, const void *const *src_shards, void *
     return overlaps(ranges, n) ? REDIST_EOVERLAP : REDIST_OK;
 }
 
-// Pointer tables of one launch from the caller's buffers, then the prepared launch.
+// Pointer tables of one launch from the caller's buffers (on the stack, CAP entries), then the prepared
+// launch with its parameter block written to `storage`.
+template <int CAP>
 redist_status prepare_launch(const Plan &p, const Launch &L, const void *const *src_shards, void *const *dst_shards,
-                             char *scratch, PreparedLaunch &pl)
+                             char *scratch, void *storage, size_t storage_bytes, PreparedLaunch &pl)
 {
     const int N = p.n_devices;
     auto buffer = [&](BufKind kind, int32_t dev) -> char * {
@@ -149,12 +155,12 @@ redist_status prepare_launch(const Plan &p, const Launch &L, const void *const *
         }
     };
     const int ns = int(L.src_holder.size()), nd = int(L.dst_devs.size());
-    if (ns > REDIST_MAX_DEVICES || nd > REDIST_MAX_DEVICES) return REDIST_EUNSUPPORTED;
-    const char *stab[REDIST_MAX_DEVICES];
-    char *dtab[REDIST_MAX_DEVICES];
+    if (ns > CAP || nd > CAP) return REDIST_EUNSUPPORTED;
+    const char *stab[CAP];
+    char *dtab[CAP];
     for (int t = 0; t < ns; ++t) stab[t] = buffer(L.from, L.src_holder[t] < 0 ? 0 : L.src_holder[t]);
     for (int t = 0; t < nd; ++t) dtab[t] = buffer(L.to, L.dst_devs[t] < 0 ? 0 : L.dst_devs[t]);
-    cudaError_t ce = prepare_copy(L.kernel, L.geo, stab, ns, dtab, nd, int(p.tuning.pdl), pl);
+    cudaError_t ce = prepare_copy(L.kernel, L.geo, stab, ns, dtab, nd, int(p.tuning.pdl), storage, storage_bytes, pl);
     if (ce != cudaSuccess) {
         tl_cuda_error = int(ce);
         return REDIST_ECUDA;
@@ -162,24 +168,22 @@ redist_status prepare_launch(const Plan &p, const Launch &L, const void *const *
     return REDIST_OK;
 }
 
-}  // namespace
-
-namespace redist {
-
-// Checks, then one kernel launch per entry of the plan's launch list.  Tables and the parameter block
-// live on this call's stack (about 100 KiB); nothing is allocated on the host or on the device.
-redist_status run_plan(const Plan &p, const void *const *src_shards, void *const *dst_shards, void *scratch,
-                       size_t scratch_range, void *cuda_stream)
+// Checks, then one kernel launch per entry of the plan's launch list; tables and parameter block on
+// this frame.
+template <int CAP>
+redist_status run_plan_with(const Plan &p, const void *const *src_shards, void *const *dst_shards, void *scratch,
+                            size_t scratch_range, void *cuda_stream)
 {
-    redist_status rc = check_buffers(p, src_shards, dst_shards, scratch, scratch_range);
+    redist_status rc = check_buffers<CAP>(p, src_shards, dst_shards, scratch, scratch_range);
     if (rc != REDIST_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    alignas(16) unsigned char storage[param_bytes(CAP)];
     PreparedLaunch pl;
     static const char *const kNames[] = {"redist dynslice", "redist alltoall", "redist allgather", "redist allpermute",
                                          "redist copy", "redist fused", "redist naive gather", "redist naive slice"};
     for (const Launch &L : p.launches) {
         if (L.geo.n_items == 0) continue;
-        rc = prepare_launch(p, L, src_shards, dst_shards, static_cast<char *>(scratch), pl);
+        rc = prepare_launch<CAP>(p, L, src_shards, dst_shards, static_cast<char *>(scratch), storage, sizeof storage, pl);
         if (rc != REDIST_OK) return rc;
         // an NVTX range around every launch names the step for a timeline profiler (tuning value "nvtx")
         const bool mark = p.tuning.nvtx != 0;
@@ -192,6 +196,20 @@ redist_status run_plan(const Plan &p, const void *const *src_shards, void *const
         }
     }
     return REDIST_OK;
+}
+
+}  // namespace
+
+namespace redist {
+
+// Checks, then the plan's kernel launches.  Everything lives on this call's stack -- about 8 KiB for
+// plans of up to 64 virtual devices, about 100 KiB beyond; nothing is allocated on the host or the device.
+redist_status run_plan(const Plan &p, const void *const *src_shards, void *const *dst_shards, void *scratch,
+                       size_t scratch_range, void *cuda_stream)
+{
+    return p.n_devices <= kSmallTable
+               ? run_plan_with<kSmallTable>(p, src_shards, dst_shards, scratch, scratch_range, cuda_stream)
+               : run_plan_with<kLargeTable>(p, src_shards, dst_shards, scratch, scratch_range, cuda_stream);
 }
 
 }  // namespace redist
@@ -522,7 +540,9 @@ redist_status redist_bind(const redist_plan_t *plan, const void *const *src_shar
     if (!plan || !src_shards || !dst_shards || !out) return REDIST_EINVAL;
     const Plan &p = plan->p;
     if (p.scratch_bytes > 0 && (!scratch || scratch_bytes < size_t(p.scratch_bytes))) return REDIST_ESCRATCH;
-    redist_status rc = check_buffers(p, src_shards, dst_shards, scratch, size_t(p.scratch_bytes));
+    const bool small = p.n_devices <= kSmallTable;
+    redist_status rc = small ? check_buffers<kSmallTable>(p, src_shards, dst_shards, scratch, size_t(p.scratch_bytes))
+                             : check_buffers<kLargeTable>(p, src_shards, dst_shards, scratch, size_t(p.scratch_bytes));
     if (rc != REDIST_OK) return rc;
     try {
         std::unique_ptr<redist_bound_s> b(new redist_bound_s());
@@ -530,11 +550,17 @@ redist_status redist_bind(const redist_plan_t *plan, const void *const *src_shar
         size_t n = 0;
         for (const Launch &L : p.launches) n += L.geo.n_items != 0;
         b->launches.resize(n);
+        b->params.resize(n);
+        const size_t bytes = param_bytes(small ? kSmallTable : kLargeTable);
         size_t q = 0;
         for (const Launch &L : p.launches) {
             if (L.geo.n_items == 0) continue;
-            rc = prepare_launch(p, L, src_shards, dst_shards, static_cast<char *>(scratch), b->launches[q++]);
+            b->params[q].resize((bytes + sizeof(max_align_t) - 1) / sizeof(max_align_t));
+            char *sc = static_cast<char *>(scratch);
+            rc = small ? prepare_launch<kSmallTable>(p, L, src_shards, dst_shards, sc, b->params[q].data(), bytes, b->launches[q])
+                       : prepare_launch<kLargeTable>(p, L, src_shards, dst_shards, sc, b->params[q].data(), bytes, b->launches[q]);
             if (rc != REDIST_OK) return rc;
+            ++q;
         }
         *out = b.release();
         return REDIST_OK;

@@ -1616,8 +1616,7 @@ template <int NT>
 void fill_params(PreparedLaunch &pl, const CopyGeometry &geo, const char *const *src_tab, int n_src, char *const *dst_tab,
                  int n_dst)
 {
-    static_assert(sizeof(CopyParams<NT>) <= sizeof(pl.params), "parameter block too small");
-    CopyParams<NT> *P = reinterpret_cast<CopyParams<NT> *>(pl.params);
+    CopyParams<NT> *P = static_cast<CopyParams<NT> *>(pl.params);
     P->g = geo;
     for (int i = 0; i < n_src; ++i) P->src[i] = src_tab[i];
     for (int i = 0; i < n_dst; ++i) P->dst[i] = dst_tab[i];
@@ -1649,10 +1648,14 @@ cudaError_t read_bounds_report(long long out[5])
 }
 
 cudaError_t prepare_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
-                         char *const *dst_tab, int n_dst, int pdl, PreparedLaunch &pl)
+                         char *const *dst_tab, int n_dst, int pdl, void *storage, size_t storage_bytes,
+                         PreparedLaunch &pl)
 {
     if (n_src > kLargeTable || n_dst > kLargeTable || n_src < 0 || n_dst < 0) return cudaErrorInvalidValue;
     const bool small = n_src <= kSmallTable && n_dst <= kSmallTable;
+    if (!storage || (reinterpret_cast<uintptr_t>(storage) & 15u) || storage_bytes < param_bytes(small ? kSmallTable : kLargeTable))
+        return cudaErrorInvalidValue;
+    pl.params = storage;
     pl.fn = small ? entry_for<kSmallTable>(kernel, geo) : entry_for<kLargeTable>(kernel, geo);
     if (small)
         fill_params<kSmallTable>(pl, geo, src_tab, n_src, dst_tab, n_dst);
@@ -1699,7 +1702,7 @@ cudaError_t launch_prepared(const PreparedLaunch &pl, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = pl.pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    void *args[1] = {const_cast<unsigned char *>(pl.params)};
+    void *args[1] = {pl.params};
     return cudaLaunchKernelExC(&cfg, pl.fn, args);
 }
 
