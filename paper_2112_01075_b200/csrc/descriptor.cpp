@@ -323,7 +323,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             rpi = std::min<i64>(std::min<i64>(rpi, outer_rows), std::min<i64>(kBoxRows, kBoxSegments / std::max(n1, n2)));
             rpi = std::max<i64>(1, std::min<i64>(rpi, kBoxTile / (seg_pitch * n1)));
             bx_rpi = rpi;
-            const bool fits = rpi * n1 * seg_pitch + 2 * (s2 / vec) + 16 <= 44 * 1024;
+            // (staged segments within the tile; with the table of places and the static tables of the kernel
+            // the block stays below the 48 KiB a launch gets without opting in to more)
+            const bool fits = rpi * n1 * seg_pitch <= kBoxTile && rpi * n1 * seg_pitch + 2 * (s2 / vec) + 16 <= 44 * 1024;
             // (forced, any item will do; by default only items worth a block)
             const bool worth = tune.box >= 2 ? std::min(s1, s2) * cnt >= 128
                                              : std::min(s1, s2) * cnt >= 256 && sup * cnt * rpi >= kItemBytes / 4;
