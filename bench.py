@@ -435,6 +435,8 @@ def run_ours(args):
         line["configs"] = run_configs(torch, api, gen)
     if rank == 0 and world == 1 and args.others:
         line["others"] = run_others(torch, api, gen, args)
+    if rank == 0 and world == 1 and not args.lean:
+        line["spread_model"] = spread_model(api, ws, flags, peak)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -497,6 +499,39 @@ def run_configs(torch, api, gen, reps: int = 30):
                  "scratch_bytes_per_virtual_device_max": max(r["scratch_per_device"] for r in rows),
                  "note": "every eighth of the 100 seeded pairs, each planned, executed and timed on its own "
                          "(global array 4 GiB; 5 timed repetitions per pair after 2 warm-up launches)"}
+    return out
+
+
+def spread_model(api, ws, flags, hbm_gbs, link_gbs=770.0):
+    """NOT a measurement: what redist_plan_gpu_split says would stay inside a GPU and what would cross to
+    a peer if the virtual devices of this workload sat on 2, 4 or 8 GPUs (leading mesh axes choose the
+    GPU), and the time that bounds a step from below -- the slower of local bytes at the measured HBM
+    rate and, for the busiest GPU, bytes out or in at 770 GB/s (measured peer copy per direction)."""
+    out = {}
+    for g in (2, 4, 8):
+        local = cross = 0
+        t_us = 0.0
+        ok = True
+        for w in ws:
+            plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, flags)
+            for q in range(plan.num_launches):
+                try:
+                    m = plan.gpu_split(g, q)
+                except api.RedistError:
+                    ok = False
+                    break
+                li = plan.launch_info(q)
+                loc = sum(m[i][i] for i in range(g))
+                out_b = max(sum(m[i][j] for j in range(g) if j != i) for i in range(g))
+                in_b = max(sum(m[i][j] for i in range(g) if i != j) for j in range(g))
+                local += loc
+                cross += sum(map(sum, m)) - loc
+                # per GPU: its share of the reads and local writes at HBM speed, its link traffic at link speed
+                t_us += max((li.bytes_read + loc) / g / (hbm_gbs * 1e3), max(out_b, in_b) / (link_gbs * 1e3))
+        if ok:
+            out[f"{g}_gpus"] = {"local_bytes_written": local, "cross_bytes_written": cross,
+                                "lower_bound_us_per_step": round(t_us, 1)}
+    out["note"] = "model from redist_plan_gpu_split, not run on several GPUs"
     return out
 
 
