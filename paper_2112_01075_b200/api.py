@@ -441,7 +441,7 @@ class _Bound:
         self._fn, self._destroy = plan._lib.redist_bound_execute, plan._lib.redist_bound_destroy
 
     def __call__(self, stream_ptr: int = 0) -> None:
-        rc = self._fn(self._h, ctypes.c_void_p(stream_ptr or None))
+        rc = self._fn(self._h, stream_ptr or None)      # argtypes convert the integer; nothing is built per call
         if rc:
             raise RedistError(rc, "redist_bound_execute")
 
