@@ -165,6 +165,9 @@ void redist_plan_cache_clear(void);
  *   "box"                0..2   super-box kernels (several interleaving dimensions staged through shared
  *                               memory at once): never / where the other short-run paths do badly
  *                               (default 1) / wherever they apply
+ *   "box_width"          0..256 lanes that share one target range in the super-box kernels (a power of two; other
+ *                               values are ignored); 0 (default): a warp or more as a rule, fewer where the units of
+ *                               one range would fall into a few shared-memory banks
  *   "zip_walks"          0..7   chunk-to-unit maps the zip kernels may use: 1 periodic + 2 by range +
  *                               4 tabulated (default 7; the flat walk is always available)
  *   "zip_by_range_slots" >= 1   fewest chunk slots of a range for the by-range walk (default 256)

@@ -74,6 +74,7 @@ const TuningName kTuningNames[] = {
     {"gather", &Tuning::gather, 0, 2},
     {"zip", &Tuning::zip, 0, 2},
     {"box", &Tuning::box, 0, 2},
+    {"box_width", &Tuning::box_width, 0, 256},
     {"zip_walks", &Tuning::zip_walks, 0, 7},
     {"zip_by_range_slots", &Tuning::zip_by_range_slots, 1, 1 << 20},
     {"item_kb", &Tuning::item_kb, 0, 1024},

@@ -329,14 +329,13 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             // (forced, any item will do; by default only items worth a block)
             const bool worth = tune.box >= 2 ? std::min(s1, s2) * cnt >= 128
                                              : std::min(s1, s2) * cnt >= 256 && sup * cnt * rpi >= kItemBytes / 4;
-            // default policy: where the unit walk or the gather walk would run, and where the zip kernels
-            // would zip a digit of fewer than 16 rows
+            // default policy: where the row, unit or gather walk would run on runs below 256 bytes, and where
+            // the zip kernels would zip a digit of fewer than 16 rows
             // (measured on the odd-shape sweep: against the unit walk and the gather walk 1.5-1.7x; against the
             // zip kernels 1.2-1.26x where their target ranges are short -- each range pays for its own ragged
             // head and tail --, 0.8-0.9x where they are long)
             const i64 zip_range = zip_n * (m2[kp] > 1 ? std::max(m1[kp], m2[kp]) * run_bytes : run_bytes);
-            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_range < 768
-                                                            : run_bytes < 256 && (g_levels >= 0 || !G.aligned));
+            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_range < 768 : run_bytes < 256);
             if (!fits || !worth || !wanted || sup > (1ll << 30)) bxK = -2;
         }
     }
@@ -445,11 +444,89 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         G.bx_row_units_div = make_div(uint32_t(bx_s2 / vec));
         G.zip_slots = make_div(uint32_t(bx_cnt * bx_s2 / 16 + 1));
         {
-            // lanes per range: about four chunks each, a whole number of warps, no more groups than ranges
+            // Lanes per range (a power of two; groups of that many lanes share out the ranges of the item).
+            // Two things decide: how evenly ranges and chunks divide among the groups, and the shared-memory
+            // banks.  Where the units of one target tile sit a power-of-two stride apart in the staged
+            // segments (a tile that takes one element in 4 or 8 of the last dimension), the lanes of a warp
+            // that all work on one range read from 1-4 of the 32 banks; neighbouring ranges start a few
+            // bytes apart, so narrower groups -- several ranges per warp -- spread the reads.  For every
+            // width the banks of the first warp's reads are counted and the time of the item estimated as
+            //     (warp, step) pairs with a lane at work  x  (52 issue slots + wavefronts of the reads)
+            //                                             x  (1 + 4 / warps that have work)
+            // (constants fitted to the measured times of 119 launches at seven widths each; choosing by the
+            // estimate is within 0.3 % of choosing by the measurement, geometric mean, 3.6 % at worst).
             const i64 chunks = bx_cnt * bx_s2 / 16, ranges = bx_rpi * n2;
-            i64 w = 32;
-            while (w < kBlockThreads && (w * 4 < chunks || kBlockThreads / w > ranges)) w *= 2;
-            G.zip_width = uint32_t(w);
+            const uint32_t unit = uint32_t(vec), per = 16u / unit;
+            auto place = [&](uint32_t p) {
+                uint32_t rest = p / G.bx_trail.d, off = (p % G.bx_trail.d) * unit;
+                for (int q = int(G.bx_n) - 1; q >= 0; --q) {
+                    const uint32_t i = rest % G.bx_c2[q].d;
+                    rest /= G.bx_c2[q].d;
+                    off += i / G.bx_c1[q].d * G.bx_seg[q] * G.zip_seg_pitch + i % G.bx_c1[q].d * G.bx_st1[q];
+                }
+                return off;
+            };
+            auto base = [&](uint32_t range) {
+                uint32_t rem = range % uint32_t(n2), off = range / uint32_t(n2) * G.stage_pitch;
+                for (int q = int(G.bx_n) - 1; q >= 0; --q) {
+                    const uint32_t x = rem % G.bx_n2[q].d * G.bx_c2[q].d;
+                    rem /= G.bx_n2[q].d;
+                    off += x / G.bx_c1[q].d * G.bx_seg[q] * G.zip_seg_pitch + x % G.bx_c1[q].d * G.bx_st1[q];
+                }
+                return off;
+            };
+            const uint32_t row_units = G.zip_lut_units;
+            auto wavefronts = [&](i64 width) {                 // of the first warp's reads of one chunk each
+                const uint32_t phase_lanes = 32u * 4u / unit;  // 8- and 16-byte reads go in half and quarter warps
+                uint32_t total = 0;
+                for (uint32_t i = 0; i < per; ++i)
+                    for (uint32_t l0 = 0; l0 < 32u; l0 += phase_lanes) {
+                        uint32_t words[32][32], n_words[32] = {0}, worst = 0;
+                        for (uint32_t l = l0; l < l0 + phase_lanes; ++l) {
+                            const uint32_t range = l / uint32_t(width), c = l % uint32_t(width);
+                            if (i64(range) >= ranges || i64(c) >= chunks) continue;
+                            const uint32_t x = c * per + i;
+                            const uint32_t at = base(range) + x / row_units * G.bx_s1 + place(x % row_units);
+                            for (uint32_t b = 0; b < unit / 4u; ++b) {
+                                const uint32_t word = at / 4u + b, bank = word & 31u;
+                                bool seen = false;
+                                for (uint32_t k = 0; k < n_words[bank]; ++k) seen |= words[bank][k] == word;
+                                if (!seen) words[bank][n_words[bank]++] = word;
+                                worst = std::max(worst, n_words[bank]);
+                            }
+                        }
+                        total += worst;
+                    }
+                return total;
+            };
+            auto estimate = [&](i64 width) {
+                const i64 groups = kBlockThreads / width, steps = (chunks + width - 1) / width;
+                auto ranges_of = [&](i64 group) { return group < ranges ? (ranges - group + groups - 1) / groups : 0; };
+                i64 pairs = 0, busy = 0;
+                if (width >= 32) {
+                    for (i64 gi = 0; gi < groups; ++gi) pairs += ranges_of(gi) * steps * (width / 32);
+                    busy = std::min<i64>(kBlockThreads / 32, std::min(groups, ranges) * (width / 32));
+                } else {
+                    const i64 per_warp = 32 / width;
+                    for (i64 v = 0; v < kBlockThreads / 32; ++v) {
+                        const i64 most = ranges_of(v * per_warp);   // the first group of a warp has the most ranges
+                        pairs += most * steps;
+                        busy += most > 0;
+                    }
+                }
+                return double(pairs) * double(52 + wavefronts(width)) * (1.0 + 4.0 / double(std::max<i64>(1, busy)));
+            };
+            i64 best = 2;
+            double best_cost = estimate(2);
+            for (i64 cand = 4; cand <= 128; cand *= 2) {
+                const double cost = estimate(cand);
+                if (cost < best_cost * 0.999) {
+                    best = cand;
+                    best_cost = cost;
+                }
+            }
+            if (tune.box_width > 0 && (tune.box_width & (tune.box_width - 1)) == 0) best = tune.box_width;
+            G.zip_width = uint32_t(best);
         }
         G.gl_m = make_div(1);
         ipb = (tab_rows + bx_rpi - 1) / bx_rpi * ncb;

@@ -1333,7 +1333,9 @@ REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
 // copies and tabulates base[] and the range offsets, while the other warps tabulate place[]; the walk
 // over the ranges then reads everything item-specific from those tables.  Lanes work in groups of
 // zip_width (a power of two) that share out the ranges; a lane strides through its range's chunks and
-// keeps (row, position in row) by adding a constant per step instead of dividing.
+// keeps (row, position in row) by adding a constant per step instead of dividing.  The host picks the
+// width: a warp or more per range as a rule, fewer lanes -- several ranges per warp -- where the units of
+// one range would all fall into a few shared-memory banks.
 template <typename T, int NT>
 __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char *tile, uint32_t *base_of,
                                          uint32_t *tile_of, int64_t *row_d0, uint32_t mbar, unsigned int *wait_failed)
@@ -1435,7 +1437,7 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
         return;
     }
     // whole chunks: groups of W lanes share out the ranges (outer row, target tile)
-    const uint32_t W = g.zip_width;                              // power of two, 32 .. block size
+    const uint32_t W = g.zip_width;                              // power of two, 1 .. block size
     const uint32_t n_groups = nthreads / W;
     const uint32_t lane = tid & (W - 1u);
     const uint32_t step_units = W * uint32_t(kPer);              // units between a lane's consecutive chunks

@@ -58,6 +58,7 @@ struct Tuning {
     int64_t gather = 1;               // gather walk: 0 never, 1 where measured faster, 2 wherever it applies
     int64_t zip = 2;                  // zip kernels: 0 never, 1 only where the gather walk is not chosen, 2 wherever they apply
     int64_t box = 1;                  // super-box kernels: 0 never, 1 where zip / gather / unit walks do badly, 2 wherever they apply
+    int64_t box_width = 0;            // super-box kernels: lanes per target range (a power of two), 0: chosen per launch
     int64_t zip_walks = 7;            // chunk -> units maps the zip kernels may use: 1 periodic, 2 by range, 4 tabulated
     int64_t zip_by_range_slots = 256; // fewest chunk slots of a range for the by-range walk
     int64_t item_kb = 0;              // KiB read per work item (0: 32 / 16 / 8 by fan-out, bulk copies 20 / 12 / 6)
@@ -69,7 +70,7 @@ struct Tuning {
     int64_t test_shrink_tiles = 0;    // test only: bytes by which the checked build believes every tile to be shorter
     bool operator==(const Tuning &o) const
     {
-        return bulk == o.bulk && gather == o.gather && zip == o.zip && box == o.box && zip_walks == o.zip_walks &&
+        return bulk == o.bulk && gather == o.gather && zip == o.zip && box == o.box && box_width == o.box_width && zip_walks == o.zip_walks &&
                zip_by_range_slots == o.zip_by_range_slots && item_kb == o.item_kb && pdl == o.pdl && nvtx == o.nvtx &&
                step_latency == o.step_latency && wait_polls == o.wait_polls && test_extra_tx == o.test_extra_tx &&
                test_shrink_tiles == o.test_shrink_tiles;

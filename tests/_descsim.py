@@ -105,7 +105,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         assert G["zip_seg_pitch"] % 16 == 0 and G["zip_seg_pitch"] >= cnt * G["bx_s1"] + 30
         assert G["stage_pitch"] == G["zip_seg_pitch"] * G["bx_nseg"] and G["stage_pitch"] * rpi <= 38 * 1024
         assert G["zip_lut_units"] * unit == G["bx_s2"] and G["zip_lut_units"] <= 4096
-        assert G["zip_slots"] >= cnt * G["bx_s2"] // 16 + 1 and G["zip_width"] in (32, 64, 128, 256)
+        assert G["zip_slots"] >= cnt * G["bx_s2"] // 16 + 1 and G["zip_width"] in (1, 2, 4, 8, 16, 32, 64, 128, 256)
         assert G["items_per_box"] == -(-tab_rows // rpi) * G["col_blocks"]
         # the digits of the inner dimensions count super-boxes: unit_mul boxes of the gcd size each
         assert _prod(unit_mul) >= 1

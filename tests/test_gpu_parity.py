@@ -205,6 +205,33 @@ def test_super_box_kernels(mesh, gshape, a1, a2, e):
     assert 8 in seen
 
 
+BANKED = [  # a target tile takes one element in 4 or 8 of the last dimension: its units sit 32 bytes apart
+    ((4, 2, 2), (2, 17, 16, 28, 9, 8), ((1,), (), (2, 0), (), (), ()), ((), (), (), (1,), (), (0, 2)), 4),
+    ((2, 2, 2), (4, 6, 16, 12, 5, 4), ((0,), (), (1, 2), (), (), ()), ((), (), (), (0,), (), (1, 2)), 8),
+]
+
+
+@pytest.mark.parametrize("width", [0, 1, 2, 4, 8, 16, 64])
+def test_super_box_kernels_at_every_lane_group_width(width):
+    """The lanes that share one target range in the super-box kernels: chosen per launch by default (narrower than
+    a warp where one range's units would fall into a few shared-memory banks -- the two BANKED shapes), and every
+    width forced over all the super-box shapes."""
+    seen, widths = set(), set()
+    for mesh, gshape, a1, a2, e in BOXES + BANKED:
+        G = np.random.default_rng(sum(gshape) + e + width).integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+        for src, dst in (((gshape, a1), (gshape, a2)), ((gshape, a2), (gshape, a1))):
+            src_tiles, want = oracle.reslice(mesh, src, G), oracle.reslice(mesh, dst, G)
+            with api.tuning(box=2, box_width=width):
+                plan, got = run_gpu(mesh, src, dst, e, src_tiles)
+            for L in plan.describe()["launches"]:
+                if L["geometry"]["mode"] == 5:
+                    widths.add(L["geometry"]["zip_width"])
+            seen.update(plan.launch_info(q).variant for q in range(plan.num_launches))
+            assert_same(got, want, f"super-box {mesh} {src} -> {dst} width={width}")
+    assert 8 in seen
+    assert widths == {width} if width else min(widths) < 32 <= max(widths), widths
+
+
 def test_gather_walk_wherever_it_applies():
     """gather = 2 sends every eligible launch through the gather walk, including long source rows that
     are scattered into several target tiles and 16-byte units (not chosen by default)."""

@@ -59,6 +59,8 @@ with api.tuning(box=0):
     variants |= T.random_problems_small_and_odd(200)
 for case in T.BOXES:
     T.test_super_box_kernels(*case)
+for width in (0, 1, 4, 16):
+    T.test_super_box_kernels_at_every_lane_group_width(width)
 for values in ({"zip_walks": 0}, {"zip_walks": 2, "zip_by_range_slots": 1}, {"zip_walks": 4}):
     with api.tuning(**values):
         variants |= T.random_problems_small_and_odd(200)
