@@ -330,12 +330,14 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             const bool worth = tune.box >= 2 ? std::min(s1, s2) * cnt >= 128
                                              : std::min(s1, s2) * cnt >= 256 && sup * cnt * rpi >= kItemBytes / 4;
             // default policy: where the row, unit or gather walk would run on runs below 256 bytes, and where
-            // the zip kernels would zip a digit of fewer than 16 rows
+            // the zip kernels would zip a digit of fewer than 8 rows or work on short target ranges
             // (measured on the odd-shape sweep: against the unit walk and the gather walk 1.5-1.7x; against the
-            // zip kernels 1.2-1.26x where their target ranges are short -- each range pays for its own ragged
-            // head and tail --, 0.8-0.9x where they are long)
+            // zip kernels 1.1-1.5x where their target ranges are below 768 bytes -- each range pays for its own
+            // ragged head and tail --, 1.03-1.06x up to 1536 bytes unless the fan-out is 8 or more, 1.04-1.15x
+            // where the zipped digit has fewer than 8 rows, 0.97x elsewhere)
             const i64 zip_range = zip_n * (m2[kp] > 1 ? std::max(m1[kp], m2[kp]) * run_bytes : run_bytes);
-            const bool wanted = tune.box >= 2 || (zip_n > 0 ? zip_range < 768 : run_bytes < 256);
+            const bool wanted = tune.box >= 2 ||
+                                (zip_n > 0 ? (zip_range < 1536 && (zip_range < 768 || fan < 8)) || zip_n < 8 : run_bytes < 256);
             if (!fits || !worth || !wanted || sup > (1ll << 30)) bxK = -2;
         }
     }
