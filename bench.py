@@ -641,9 +641,9 @@ def sweep_rows(torch, api, pairs, flags, fill_seed):
     for w in pairs:
         if G is None or tuple(G.shape[:-1]) != tuple(w.src.global_shape):
             G = None
-            G = torch.randint(0, 256, tuple(w.src.global_shape) + (4,), dtype=torch.uint8, device="cuda",
+            G = torch.randint(0, 256, tuple(w.src.global_shape) + (w.elem_bytes,), dtype=torch.uint8, device="cuda",
                               generator=gen)
-        plan = api.Plan(w.mesh_shape, w.src, w.dst, 4, flags)
+        plan = api.Plan(w.mesh_shape, w.src, w.dst, w.elem_bytes, flags)
         _, offs = api.redist_base_offsets(w.mesh_shape, w.src)
         tiles = api.shard_global(G, w.mesh_shape, w.src)
         owned = {}
@@ -652,7 +652,7 @@ def sweep_rows(torch, api, pairs, flags, fill_seed):
                 owned[o] = tiles[d].clone()
         src = [owned[o] for o in offs]
         del tiles
-        db = plan.local_elems(1) * 4
+        db = plan.local_elems(1) * w.elem_bytes
         dst = [torch.empty(db, dtype=torch.uint8, device="cuda") for _ in range(plan.n_devices)]
         scratch = plan.alloc_scratch()
         call = plan.bind([t.data_ptr() for t in src], [t.data_ptr() for t in dst],
@@ -705,6 +705,10 @@ def run_sweep(args):
         flags |= api.COST_PERMUTE
     if args.only:
         pairs = [w for w in pairs if w.name in args.only.split(",")]
+    if args.elem_bytes:
+        import dataclasses
+        pairs = [dataclasses.replace(w, elem_bytes=args.elem_bytes) for w in pairs]
+        label += ", elements of %d bytes instead of 4" % args.elem_bytes
     rows = sweep_rows(torch, api, pairs[: args.pairs], flags, wl.CONFIG4_FILL_SEED)
     g = [r["gbs"] for r in rows]
     peak, how = measured_peak()
@@ -821,6 +825,8 @@ def main():
                     choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval"])
     ap.add_argument("--pairs", type=int, default=100, help="sweeps: how many problems to run")
     ap.add_argument("--only", default="", help="sweeps: comma-separated problem names to run")
+    ap.add_argument("--elem-bytes", type=int, default=0, choices=[0, 1, 2, 4, 8, 16],
+                    help="sweeps: run the same shapes with elements of this many bytes (0: the workload's own, 4)")
     ap.add_argument("--dump", default="", help="sweeps: write the per-problem table to this JSON file")
     ap.add_argument("--fuse", default="adjacent", choices=["adjacent", "none", "all", "naive"])
     ap.add_argument("--cost-permute", action="store_true",

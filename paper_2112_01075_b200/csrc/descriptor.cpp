@@ -221,7 +221,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     const int kGather = int(tune.gather);
     int g_levels = -1;
     i64 g_stretch = 0;
-    if (kGather > 0 && vec >= 4 && run_bytes < 256 && G.inner_digit != 0xffffffffu && (m1[kp] == 1 || m2[kp] == 1)) {
+    if (kGather > 0 && run_bytes < 256 && G.inner_digit != 0xffffffffu && (m1[kp] == 1 || m2[kp] == 1)) {
         const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);
         const i64 piece_stride = long_dst ? G.unit_b2[G.inner_digit] : G.unit_b1[G.inner_digit];
@@ -246,11 +246,14 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // wherever they apply (measured: within 0.3 % of the best choice per problem on the odd-shape sweep)
     const int kZip = int(tune.zip);
     const i64 kZipMinRange = 128;         // shortest target range of a table row
-    const i64 kZipRun = 2048;             // runs below this many bytes may take the zip kernels
-    // measured: from 2 KiB the plain bulk copy (aligned runs) and the ragged chunk walk are faster
+    // runs below this many bytes may take the zip and super-box kernels: measured, from 2 KiB the plain bulk
+    // copy (aligned runs) and the ragged chunk walk are faster; with units of 1 or 2 bytes (8 or 16 of them to a
+    // chunk) the ragged chunk walk, which shifts whole chunks whatever the unit, wins from 512 bytes unless
+    // every chunk is stored to four or more replicas
+    const i64 kZipRun = vec >= 4 || fan >= 4 ? 2048 : 512;
     const bool zip_run_ok = run_bytes < kZipRun;
     i64 zip_n = 0;
-    if (kZip > 0 && kBulk && (kZip >= 2 || g_levels < 0) && vec >= 4 && zip_run_ok && G.inner_digit != 0xffffffffu &&
+    if (kZip > 0 && kBulk && (kZip >= 2 || g_levels < 0) && zip_run_ok && G.inner_digit != 0xffffffffu &&
         (m1[kp] == 1 || m2[kp] == 1) && !rows.empty()) {
         const bool long_dst = m2[kp] > 1;
         const i64 m = std::max(m1[kp], m2[kp]);
@@ -274,7 +277,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     int bxK = -2;                 // the dimension outside them (-1: none)
     i64 bx_s1 = 0, bx_s2 = 0, bx_cnt = 0, bx_gK = 1, bx_rpi = 1;
     const i64 kBoxTile = 38 * 1024;
-    if (tune.box > 0 && kBulk && vec >= 4 && kp >= 0 && run_bytes < 2048 && nq[kp] > 1) {
+    if (tune.box > 0 && kBulk && kp >= 0 && zip_run_ok && nq[kp] > 1) {
         i64 trail = e;                               // bytes of the identical trailing dimensions
         for (int k = kp + 1; k < r; ++k) trail *= a.tile[k];
         i64 s1 = trail, s2 = trail, sup = trail, n1 = 1, n2 = 1;
@@ -479,7 +482,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             };
             const uint32_t row_units = G.zip_lut_units;
             auto wavefronts = [&](i64 width) {                 // of the first warp's reads of one chunk each
-                const uint32_t phase_lanes = 32u * 4u / unit;  // 8- and 16-byte reads go in half and quarter warps
+                const uint32_t phase_lanes = std::min(32u, 32u * 4u / unit);   // 8- and 16-byte reads go in half and quarter warps
                 uint32_t total = 0;
                 for (uint32_t i = 0; i < per; ++i)
                     for (uint32_t l0 = 0; l0 < 32u; l0 += phase_lanes) {
@@ -489,7 +492,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                             if (i64(range) >= ranges || i64(c) >= chunks) continue;
                             const uint32_t x = c * per + i;
                             const uint32_t at = base(range) + x / row_units * G.bx_s1 + place(x % row_units);
-                            for (uint32_t b = 0; b < unit / 4u; ++b) {
+                            for (uint32_t b = 0; b < std::max(1u, unit / 4u); ++b) {
                                 const uint32_t word = at / 4u + b, bank = word & 31u;
                                 bool seen = false;
                                 for (uint32_t k = 0; k < n_words[bank]; ++k) seen |= words[bank][k] == word;
@@ -593,14 +596,14 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                 G.zip_width = uint32_t(std::min<i64>(want * pc, kBlockThreads / pc * pc));
             }
         }
-        // By-range walk: for runs of 32 bytes and more of 4-byte units (64 and more of 8-byte units; nothing
+        // By-range walk: for runs of eight units and more (32 bytes of 4-byte units, 64 of 8-byte units; nothing
         // to gain with 16-byte units) the chunk slots of a range are numbered (run, i-th target-aligned chunk
         // that starts in the run) -- such a chunk takes its units from that run and, past its end, from the
         // next one, no division per unit -- and a range with 256 slots or more is walked by the whole block.
         const i64 kZipPerRun = (tune.zip_walks & 2) ? 32 : 0;   // shortest run (of 4-byte units) for the by-range walk
         const i64 kZipByRange = std::max<i64>(1, tune.zip_by_range_slots);
         const i64 cpr = (run_bytes + 15) / 16;
-        if (G.zip_period.d == 0 && kZipPerRun > 0 && run_bytes >= kZipPerRun * (vec / 4) && vec < 16 &&
+        if (G.zip_period.d == 0 && kZipPerRun > 0 && run_bytes * 4 >= kZipPerRun * vec && vec < 16 &&
             rpb * (long_dst ? m : 1) * cpr >= kZipByRange) {
             G.zip_cpr = make_div(uint32_t(cpr));
             G.zip_slots = make_div(uint32_t(rpb * (long_dst ? m : 1) * cpr));

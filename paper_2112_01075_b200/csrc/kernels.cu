@@ -648,23 +648,34 @@ __device__ __forceinline__ void gather_body(const CopyParams<NT> &P, RowEntry *r
     }
 }
 
-template <bool LONG_DST, int NT>
+// The gather, zip and super-box kernels come in two builds each: SMALL = false for units of 4, 8 and 16
+// bytes, SMALL = true for units of 1 and 2 bytes (odd run lengths of 8- and 16-bit elements), where a
+// 16-byte chunk is assembled from 8 or 16 units.  They are separate kernels so that the registers the
+// small-unit walks need do not lower the occupancy of the others.
+template <bool LONG_DST, int NT, bool SMALL>
 __device__ __forceinline__ void gather_dispatch(const CopyParams<NT> &P)
 {
     __shared__ RowEntry rowtab[kMaxRowsFlat];
-    switch (P.g.unit_bytes) {
-    case 16: gather_body<LONG_DST, uint4, NT>(P, rowtab); break;
-    case 8: gather_body<LONG_DST, uint2, NT>(P, rowtab); break;
-    default: gather_body<LONG_DST, uint32_t, NT>(P, rowtab); break;
+    if constexpr (SMALL) {
+        if (P.g.unit_bytes == 2)
+            gather_body<LONG_DST, uint16_t, NT>(P, rowtab);
+        else
+            gather_body<LONG_DST, uint8_t, NT>(P, rowtab);
+    } else {
+        switch (P.g.unit_bytes) {
+        case 16: gather_body<LONG_DST, uint4, NT>(P, rowtab); break;
+        case 8: gather_body<LONG_DST, uint2, NT>(P, rowtab); break;
+        default: gather_body<LONG_DST, uint32_t, NT>(P, rowtab); break;
+        }
     }
 }
 
 #define REDIST_DEFINE_GATHER_KERNEL(NAME)                                                            \
-    template <bool LONG_DST, int NT>                                                                 \
+    template <bool LONG_DST, int NT, bool SMALL>                                                     \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
-        gather_dispatch<LONG_DST, NT>(P);                                                            \
+        gather_dispatch<LONG_DST, NT, SMALL>(P);                                                     \
     }
 
 REDIST_DEFINE_GATHER_KERNEL(redist_dynslice_gather_kernel)
@@ -1290,7 +1301,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
 }
 
 #define REDIST_DEFINE_ZIP_KERNEL(NAME)                                                               \
-    template <bool LONG_DST, int NT>                                                                 \
+    template <bool LONG_DST, int NT, bool SMALL>                                                     \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
         extern __shared__ __align__(128) unsigned char tile[];                                       \
@@ -1300,10 +1311,17 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
         __shared__ unsigned int wait_failed;                                                         \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         const uint32_t mbar = smem_addr(&mbar_storage);                                              \
-        switch (P.g.unit_bytes) {                                                                    \
-        case 16: zip_body<LONG_DST, uint4, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break; \
-        case 8: zip_body<LONG_DST, uint2, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break;  \
-        default: zip_body<LONG_DST, uint32_t, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break; \
+        if constexpr (SMALL) {                                                                       \
+            if (P.g.unit_bytes == 2)                                                                 \
+                zip_body<LONG_DST, uint16_t, NT>(P, tile, rowtab, segbase, mbar, &wait_failed);      \
+            else                                                                                     \
+                zip_body<LONG_DST, uint8_t, NT>(P, tile, rowtab, segbase, mbar, &wait_failed);       \
+        } else {                                                                                     \
+            switch (P.g.unit_bytes) {                                                                \
+            case 16: zip_body<LONG_DST, uint4, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break; \
+            case 8: zip_body<LONG_DST, uint2, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break; \
+            default: zip_body<LONG_DST, uint32_t, NT>(P, tile, rowtab, segbase, mbar, &wait_failed); break; \
+            }                                                                                        \
         }                                                                                            \
     }
 
@@ -1523,7 +1541,7 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
 }
 
 #define REDIST_DEFINE_BOX_KERNEL(NAME)                                                               \
-    template <int NT>                                                                                \
+    template <int NT, bool SMALL>                                                                    \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
         extern __shared__ __align__(128) unsigned char tile[];                                       \
@@ -1534,10 +1552,17 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
         __shared__ unsigned int wait_failed;                                                         \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         const uint32_t mbar = smem_addr(&mbar_storage);                                              \
-        switch (P.g.unit_bytes) {                                                                    \
-        case 16: box_body<uint4, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break;  \
-        case 8: box_body<uint2, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break;   \
-        default: box_body<uint32_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+        if constexpr (SMALL) {                                                                       \
+            if (P.g.unit_bytes == 2)                                                                 \
+                box_body<uint16_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed);       \
+            else                                                                                     \
+                box_body<uint8_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed);        \
+        } else {                                                                                     \
+            switch (P.g.unit_bytes) {                                                                \
+            case 16: box_body<uint4, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            case 8: box_body<uint2, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            default: box_body<uint32_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            }                                                                                        \
         }                                                                                            \
     }
 
@@ -1591,16 +1616,25 @@ const void *entry_for(int kernel, const CopyGeometry &geo)
     default: fn = redist_fused##SUFFIX<__VA_ARGS__>; break;                               \
     }
     const bool ld = geo.gl_long_dst != 0;
+    const bool small = geo.unit_bytes < 4;
     if (geo.bulk == 2) {
         REDIST_PICK(_ragged_bulk_kernel, NT)
     } else if (geo.bulk) {
         REDIST_PICK(_bulk_kernel, NT)
     } else if (geo.mode == kModeBox) {
-        REDIST_PICK(_box_kernel, NT)
+        if (small) { REDIST_PICK(_box_kernel, NT, true) } else { REDIST_PICK(_box_kernel, NT, false) }
     } else if (geo.mode == kModeZip) {
-        if (ld) { REDIST_PICK(_zip_kernel, true, NT) } else { REDIST_PICK(_zip_kernel, false, NT) }
+        if (small) {
+            if (ld) { REDIST_PICK(_zip_kernel, true, NT, true) } else { REDIST_PICK(_zip_kernel, false, NT, true) }
+        } else {
+            if (ld) { REDIST_PICK(_zip_kernel, true, NT, false) } else { REDIST_PICK(_zip_kernel, false, NT, false) }
+        }
     } else if (geo.mode == kModeGather) {
-        if (ld) { REDIST_PICK(_gather_kernel, true, NT) } else { REDIST_PICK(_gather_kernel, false, NT) }
+        if (small) {
+            if (ld) { REDIST_PICK(_gather_kernel, true, NT, true) } else { REDIST_PICK(_gather_kernel, false, NT, true) }
+        } else {
+            if (ld) { REDIST_PICK(_gather_kernel, true, NT, false) } else { REDIST_PICK(_gather_kernel, false, NT, false) }
+        }
     } else if (geo.mode == kModeRows) {
         REDIST_PICK(_kernel, 0, NT)
     } else if (geo.mode == kModeUnits) {

@@ -39,7 +39,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         u = G["inner_digit"]
         m1, m2 = G["unit_m1"][u], G["unit_m2"][u]
         long_dst = G["gl_long_dst"] == 1
-        assert unit >= 4 and run < 256 and inner == 1 and mul == span == max(m1, m2) == G["gl_m"] and min(m1, m2) == 1
+        assert run < 256 and inner == 1 and mul == span == max(m1, m2) == G["gl_m"] and min(m1, m2) == 1
         assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
         assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
         lv = G["gl_levels"]
@@ -57,7 +57,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         m1, m2 = G["unit_m1"][u], G["unit_m2"][u]
         long_dst = G["gl_long_dst"] == 1
         m = max(m1, m2)
-        assert unit >= 4 and run < 2048 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 16
+        assert run < 2048 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 16
         assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
         assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
         n = G["row_n"][-1]
@@ -86,7 +86,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
     elif G["mode"] == 5:    # super-boxes: lcm(source tile, target tile) in the inner dimensions, staged by bulk copies
         nb = G["bx_n"]
         rpi = G["rows_per_item"]
-        assert 1 <= nb <= 3 and unit >= 4 and inner == span == mul == 1 and 1 <= rpi <= 32
+        assert 1 <= nb <= 3 and inner == span == mul == 1 and 1 <= rpi <= 32
         c1, c2, n1, n2 = G["bx_c1"], G["bx_c2"], G["bx_n1"], G["bx_n2"]
         trail = G["bx_trail"] * unit
         for q in range(nb):

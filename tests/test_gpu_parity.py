@@ -673,6 +673,36 @@ def test_gather_walk_and_zip_kernels(mesh, gshape, sharded, gathered, e, v_there
             assert_same(got, want, f"interleaved, unfused {mesh} {src} -> {dst}")
 
 
+SMALL_UNITS = [   # mesh, global shape, source axes, target axes, element bytes, unit bytes: odd runs of 8- and 16-bit elements
+    ((2, 4), (6, 10, 28), ((), (), (1,)), ((), (), ()), 2, 2),                                              # 14-byte runs
+    ((2, 2, 2), (8, 6, 60), ((0,), (), (1, 2)), ((0,), (), (1,)), 1, 1),                                   # 15- and 30-byte runs
+    ((8,), (33, 88), ((), (0,)), ((), ()), 2, 2),                                                          # 22-byte runs
+    ((4, 4, 4), (8, 12, 2, 28, 20, 12), ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,)), 2, 2),  # 6-byte runs, 3 inner dimensions
+    ((4, 4, 4), (8, 12, 2, 28, 20, 12), ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,)), 1, 1),  # 3-byte runs
+    ((4, 2, 2), (2, 17, 16, 28, 9, 8), ((1,), (), (2, 0), (), (), ()), ((), (), (), (1,), (), (0, 2)), 2, 2),  # single elements 16 bytes apart
+    ((2, 2, 2), (6, 6, 6, 48, 10, 26), ((), (2,), (), (0,), (), ()), ((), (), (1,), (), (2,), (0,)), 1, 1),  # 13-byte runs
+]
+
+
+@pytest.mark.parametrize("mesh,gshape,a1,a2,e,unit", SMALL_UNITS)
+def test_short_run_kernels_on_one_and_two_byte_units(mesh, gshape, a1, a2, e, unit):
+    """Odd run lengths of 8- and 16-bit elements leave units of 1 or 2 bytes: the zip, super-box and gather kernels
+    assemble a 16-byte chunk from 16 or 8 of them (kernels of their own, so that their registers do not weigh on
+    the others).  Both directions; the default choice and each family forced."""
+    G = np.random.default_rng(sum(gshape) + e).integers(0, 256, size=gshape + (e,), dtype=np.uint8)
+    seen = set()
+    for src, dst in (((gshape, a1), (gshape, a2)), ((gshape, a2), (gshape, a1))):
+        src_tiles, want = oracle.reslice(mesh, src, G), oracle.reslice(mesh, dst, G)
+        for values in ({}, {"box": 2}, {"box": 0}, {"gather": 2, "zip": 0, "box": 0}):
+            with api.tuning(**values):
+                plan, got = run_gpu(mesh, src, dst, e, src_tiles)
+            assert_same(got, want, f"small units {mesh} {src} -> {dst} {values}")
+            for q, L in enumerate(plan.describe()["launches"]):
+                assert L["geometry"]["unit_bytes"] == unit
+                seen.add(plan.launch_info(q).variant)
+    assert seen & {7, 8}, seen
+
+
 @pytest.mark.parametrize("g,variant", [((32768, 32768), 4), ((44739243, 24), 7)])
 def test_four_gib_tiles_need_64_bit_offsets(g, variant):
     """u32 arrays of 4 GiB and a little more (value = global linear index) on two devices: replicated

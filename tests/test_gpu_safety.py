@@ -66,6 +66,8 @@ for values in ({"zip_walks": 0}, {"zip_walks": 2, "zip_by_range_slots": 1}, {"zi
         variants |= T.random_problems_small_and_odd(200)
 for case in T.INTERLEAVED:
     T.test_gather_walk_and_zip_kernels(*case)
+for case in T.SMALL_UNITS:
+    T.test_short_run_kernels_on_one_and_two_byte_units(*case)
 for mesh, gshape, a1, a2, e, v in TP.KERNEL_CHOICE:
     if int(np.prod(gshape)) * e > (8 << 20):
         gshape = tuple(max(8, s // 8) if k else s for k, s in enumerate(gshape))
