@@ -694,7 +694,7 @@ def run_sweep(args):
 
     torch.cuda.set_device(0)
     if args.workload == "c4":
-        pairs, label = wl.config4(), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
+        pairs, label = wl.config4(max(100, args.pairs)), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
     elif args.workload == "adv":
         pairs, label = wl.adversarial_problems(), "adv: the %d problems of the paper's table of largest slow-downs"
     else:
