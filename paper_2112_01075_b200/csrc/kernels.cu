@@ -1150,7 +1150,17 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
         const uint32_t n_groups = width / S;
         const uint32_t grp = tl / S;
         tl -= grp * S;
-        for (uint32_t r = grp; r < nr && grp < n_groups; r += n_groups) {
+        // An item with fewer table rows than groups (one row of 46 runs for 16 target tiles, say) would leave
+        // most groups without work: the groups then share out (table row, target tile) pairs instead.
+        const bool by_pair = nr < n_groups && jn > 1;               // (jn > 1 means jn == m)
+        const uint32_t n_work = by_pair ? nr * jn : nr;
+        for (uint32_t q = grp; q < n_work && grp < n_groups; q += n_groups) {
+            uint32_t r = q, j0 = jb, j1 = jb + jn;
+            if (by_pair) {
+                r = fdiv(q, g.gl_m);
+                j0 = jb + (q - r * m);
+                j1 = j0 + 1u;
+            }
             const int64_t d0 = b.o2 + rowtab[r].s2 + int64_t(a) * (LONG_DST ? run * m : run);
             uint32_t head, chunks;
             split_run(rng_bytes, d0, head, chunks);
@@ -1159,7 +1169,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
             for (int i = 0; i < kPer; ++i)
                 at[i] = uint32_t(reinterpret_cast<const unsigned char *>(zip_src<LONG_DST, T, NT>(
                                      g, tile, segbase, r, jb, head + (tl << 4) + uint32_t(i * sizeof(T)))) - tile);
-            for (uint32_t j = jb; j < jb + jn; ++j) {
+            for (uint32_t j = j0; j < j1; ++j) {
                 uint32_t o = (j - jb) * run;
                 // fan-out 1: the target address is kept in a register (the pointer tables are read through
                 // generic loads, which the stores of the loop would otherwise order behind them)
