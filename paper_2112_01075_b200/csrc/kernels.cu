@@ -1314,7 +1314,7 @@ __device__ __forceinline__ void zip_body(const CopyParams<NT> &P, unsigned char 
 
 #define REDIST_DEFINE_ZIP_KERNEL(NAME)                                                               \
     template <bool LONG_DST, int NT, bool SMALL>                                                     \
-    __global__ void __launch_bounds__(kBlockThreads, SMALL ? 6 : 1) NAME(const __grid_constant__ CopyParams<NT> P) \
+    __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
         extern __shared__ __align__(128) unsigned char tile[];                                       \
         __shared__ RowEntry rowtab[kZipSegments];                                                    \
