@@ -121,7 +121,9 @@ typedef struct redist_launch_info {
                                       kernels), 4 TMA bulk copies, 5 gather walk, 6 ragged rows loaded by
                                       TMA bulk copies, 7 zip through shared memory, 8 super-boxes through
                                       shared memory; the kernel is named
-                                      redist_<collective>[_bulk|_gather|_ragged_bulk|_zip|_box]_kernel */
+                                      redist_<collective>[_bulk|_gather|_ragged_bulk|_zip|_box]_kernel
+                                      (variants 5, 7 and 8 on units of 1 or 2 bytes: redist_fused_..._kernel
+                                      whatever the collective)                                        */
 } redist_launch_info;
 
 /*
