@@ -175,6 +175,9 @@ void redist_plan_cache_clear(void);
  *   "zip_by_range_slots" >= 1   fewest chunk slots of a range for the by-range walk (default 256)
  *   "item_kb"            0..1024 KiB read per work item; 0 (default) = 32 / 16 / 8 by fan-out, and 20 / 12 / 6
  *                               in the bulk-copy kernels
+ *   "l2_hint"            0..4   bulk copies of the plain bulk-copy kernels that carry an L2 evict-first policy: none /
+ *                               loads / stores / both / stores where every segment goes to four or more replicas
+ *                               (default 4)
  *   "pdl"                0/1    1: kernels use programmatic dependent launch (default); 0: plain stream order
  *   "nvtx"               0/1    1: redist_execute and redist_execute_static wrap every kernel launch in an NVTX
  *                               range named after the collective, for timeline profilers (default 0)

@@ -786,10 +786,17 @@ __device__ __forceinline__ void bulk_body(const CopyParams<NT> &P)
     wait_for_previous_kernel();
     if (!mine) return;                   // the other threads have nothing to move and nothing to wait for
     const char *src = b.sbase + s1 + int64_t(seg_off);
+    uint64_t policy = 0;
+    if (g.l2_hint) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
     if (CHK_SRC(P, src, bytes) && CHK_SMEM(tid * bytes, bytes)) {
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(slot), "l"(src), "r"(bytes), "r"(mbar)
-                     : "memory");
+        if (g.l2_hint & 1u)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                         ::"r"(slot), "l"(src), "r"(bytes), "r"(mbar), "l"(policy)
+                         : "memory");
+        else
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(slot), "l"(src), "r"(bytes), "r"(mbar)
+                         : "memory");
     } else {
         // checked build only: the skipped copy's bytes are taken off the count the barrier waits for
         asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
@@ -801,9 +808,14 @@ __device__ __forceinline__ void bulk_body(const CopyParams<NT> &P)
     for (uint32_t f = 0; f < g.fanout; ++f) {
         char *dst = b.dtab[f] + b.o2 + s2 + int64_t(seg_off);
         if (!CHK_DST(P, dst, bytes)) continue;
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     ::"l"(dst), "r"(slot), "r"(bytes)
-                     : "memory");
+        if (g.l2_hint & 2u)
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                         ::"l"(dst), "r"(slot), "r"(bytes), "l"(policy)
+                         : "memory");
+        else
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(dst), "r"(slot), "r"(bytes)
+                         : "memory");
     }
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

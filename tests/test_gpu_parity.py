@@ -143,6 +143,16 @@ def test_random_problems_with_the_permutation_counted():
     random_problems_small_and_odd(300, api.COST_PERMUTE)
 
 
+@pytest.mark.parametrize("hint", [0, 1, 2, 3])
+def test_bulk_copies_with_l2_policies(hint):
+    """The plain bulk-copy kernels with an L2 evict-first policy on their loads, their stores, both or neither."""
+    with api.tuning(l2_hint=hint):
+        for w in MEDIUM[:9]:
+            src, dst, src_tiles, want = make_case(w)
+            plan, got = run_gpu(w.mesh_shape, src, dst, w.elem_bytes, src_tiles)
+            assert_same(got, want, f"{w.name} l2_hint={hint}")
+
+
 def test_register_kernels_behind_the_tuning_values():
     """With the bulk-copy kernels (zip included) and the gather walk switched off the same problems run
     on the plain register kernels."""
