@@ -4,6 +4,8 @@ numpy; costs are compared with the paper's examples and with a brute-force optim
 import heapq
 import itertools
 
+import os
+
 import numpy as np
 import pytest
 
@@ -446,6 +448,47 @@ def test_tuning_values_are_validated_and_copied_into_new_plans_only():
     assert api.tuning_get("bulk") == 1
     assert before.launch_info(0).variant == 4 and inside.launch_info(0).variant in (0, 1)
     assert api.Plan(mesh, src, dst, 4, api.NO_CACHE).launch_info(0).variant == 4
+
+
+TUNING_VALUES = {   # name: (default, lowest, highest) as the header states them
+    "bulk": (1, 0, 1), "gather": (1, 0, 2), "zip": (2, 0, 2), "box": (1, 0, 2), "box_width": (0, 0, 256),
+    "zip_walks": (7, 0, 7), "zip_by_range_slots": (256, 1, 1 << 20), "item_kb": (0, 0, 1024), "l2_hint": (4, 0, 4),
+    "pdl": (1, 0, 1), "nvtx": (0, 0, 1), "step_latency": (0, 0, 1 << 50), "wait_polls": (1 << 18, 1, 1 << 30),
+    "test_extra_tx": (0, 0, 1 << 20), "test_shrink_tiles": (0, 0, 1 << 20),
+}
+
+
+def test_every_tuning_value_has_its_documented_default_and_range():
+    api.tuning_reset()
+    header = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "redist.h")).read()
+    for name, (default, lo, hi) in TUNING_VALUES.items():
+        assert '"%s"' % name in header, name
+        assert api.tuning_get(name) == default, name
+        for bad in (lo - 1, hi + 1):
+            with pytest.raises(api.RedistError):
+                api.tuning_set(name, bad)
+        for good in (lo, hi):
+            api.tuning_set(name, good)
+            assert api.tuning_get(name) == good
+        api.tuning_reset()
+        assert api.tuning_get(name) == default
+    # the lanes per range of the super-box kernels: powers of two are taken, anything else leaves the choice to the library
+    mesh, g = (4, 4, 4), (8, 12, 2, 28, 20, 12)
+    a1, a2 = ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,))
+    def width(**values):
+        with api.tuning(box=2, **values):
+            geo = api.Plan(mesh, (g, a1), (g, a2), 4, api.NO_CACHE).describe()["launches"][0]["geometry"]
+        assert geo["mode"] == 5
+        return geo["zip_width"]
+    chosen = width()
+    assert width(box_width=8) == 8 and width(box_width=64) == 64 and width(box_width=24) == chosen
+    # the evict-first policy of the plain bulk-copy kernels: stores only, and only from fan-out 4, unless told otherwise
+    def hint(mesh, src, dst, **values):
+        with api.tuning(**values):
+            return api.Plan(mesh, src, dst, 2, api.NO_CACHE).describe()["launches"][0]["geometry"]["l2_hint"]
+    rows, cols, repl = ((4096, 4096), ((0,), ())), ((4096, 4096), ((), (0,))), ((4096, 4096), ((), ()))
+    assert hint((8,), rows, cols) == 0 and hint((8,), cols, repl) == 2 and hint((2,), cols, repl) == 0
+    assert hint((8,), rows, cols, l2_hint=3) == 3 and hint((8,), cols, repl, l2_hint=0) == 0
 
 
 @pytest.mark.parametrize("mesh", [(2, 2), (2, 3), (2, 2, 2), (2, 2, 3)])
