@@ -9,7 +9,8 @@
 
 nvcc cross-compiles without a GPU.  The CUDA runtime is linked statically, so the libraries load (and
 their host-only entry points work) on a machine without a driver.  Sources compile in parallel into
-``_obj/``; only what changed is recompiled.
+``_obj/`` -- the kernels as three parts (``-DREDIST_PART=1|2|3``), which brings a full build from over three
+minutes to under two on eight cores; only what changed is recompiled.
 """
 from __future__ import annotations
 
@@ -27,6 +28,9 @@ LIB_BOUNDS = os.path.join(HERE, "libredist_b200_bounds.so")
 SOURCES = ["api.cu", "kernels.cu", "static_scratch.cu", "planner.cpp", "descriptor.cpp", "describe.cpp", "multi_gpu.cpp"]
 HEADERS = ["plan.hpp", "copy_params.h", "kernels.h"]
 CHECKED = ["kernels.cu"]          # sources that differ in the checked build
+# (source, object name, defines): the kernels compile as three parts side by side (see REDIST_PART in kernels.cu)
+UNITS = [(s, os.path.splitext(s)[0], []) for s in SOURCES if s != "kernels.cu"] + \
+        [("kernels.cu", f"kernels_p{k}", [f"REDIST_PART={k}"]) for k in (1, 2, 3)]
 
 
 def _nvcc() -> str:
@@ -75,19 +79,20 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     newest_header = max(os.path.getmtime(d) for d in _deps() if not d.endswith((".cu", ".cpp")))
     jobs = []
-    for src in SOURCES:
+    for src, name, unit_defines in UNITS:
         variants = [("", [])] + ([("_bounds", ["REDIST_BOUNDS"])] if src in CHECKED else [])
         for suffix, defines in variants:
-            obj = os.path.join(OBJ, os.path.splitext(src)[0] + suffix + ".o")
+            obj = os.path.join(OBJ, name + suffix + ".o")
             stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(
                 newest_header, os.path.getmtime(os.path.join(CSRC, src)))
-            jobs.append((src, obj, defines, stale))
+            jobs.append((src, obj, unit_defines + defines, stale))
+    jobs.sort(key=lambda j: not j[0].startswith("kernels"))      # the long compiles first
     with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
         logs = list(pool.map(lambda j: _compile(j[0], j[1], j[2], verbose) if j[3] else "", jobs))
     if verbose:
         sys.stderr.write("".join(logs))
-    plain = [os.path.join(OBJ, os.path.splitext(s)[0] + ".o") for s in SOURCES]
-    checked = [os.path.join(OBJ, os.path.splitext(s)[0] + ("_bounds" if s in CHECKED else "") + ".o") for s in SOURCES]
+    plain = [os.path.join(OBJ, name + ".o") for _, name, _ in UNITS]
+    checked = [os.path.join(OBJ, name + ("_bounds" if src in CHECKED else "") + ".o") for src, name, _ in UNITS]
     _link(plain, LIB)
     _link(checked, LIB_BOUNDS)
     return LIB

@@ -53,6 +53,16 @@
 #include "copy_params.h"
 #include "kernels.h"
 
+// The file compiles as one translation unit (REDIST_PART undefined or 0) or as three that build in parallel
+// (-DREDIST_PART=1: register, bulk-copy and gather kernels plus the host side; 2: zip kernels; 3: super-box
+// kernels).  Kernel templates are instantiated only where entry_for names them, so each part carries its own
+// kernels and nothing else; each part also has its own copy of the device-side counters, which the readers
+// in part 1 add up.
+#ifndef REDIST_PART
+#define REDIST_PART 0
+#endif
+#define REDIST_IN(part) (REDIST_PART == 0 || REDIST_PART == (part))
+
 namespace redist {
 
 namespace {
@@ -1624,6 +1634,13 @@ REDIST_DEFINE_KERNEL(redist_allgather_kernel)
 REDIST_DEFINE_KERNEL(redist_allpermute_kernel)
 REDIST_DEFINE_KERNEL(redist_fused_kernel)
 
+// The part of this file that holds the kernels of a launch (see REDIST_PART at the top).
+inline int part_of(const CopyGeometry &geo)
+{
+    if (geo.bulk) return 1;
+    return geo.mode == kModeBox ? 3 : geo.mode == kModeZip ? 2 : 1;
+}
+
 // Which kernel entry serves a launch: by collective (so that profiles name the step that ran), by item
 // shape and by pointer-table size.
 template <int NT>
@@ -1641,34 +1658,44 @@ const void *entry_for(int kernel, const CopyGeometry &geo)
     }
     const bool ld = geo.gl_long_dst != 0;
     const bool small = geo.unit_bytes < 4;
-    if (geo.bulk == 2) {
-        REDIST_PICK(_ragged_bulk_kernel, NT)
-    } else if (geo.bulk) {
-        REDIST_PICK(_bulk_kernel, NT)
+    (void)ld;
+    (void)small;
     // (launches on units of 1 and 2 bytes all run under the fused-sequence name: a fifth of the
     // instantiations, and of the time to compile them, for a rare case)
-    } else if (geo.mode == kModeBox) {
+    if (part_of(geo) == 3) {
+#if REDIST_IN(3)
         if (small) { fn = redist_fused_box_kernel<NT, true>; } else { REDIST_PICK(_box_kernel, NT, false) }
-    } else if (geo.mode == kModeZip) {
+#endif
+    } else if (part_of(geo) == 2) {
+#if REDIST_IN(2)
         if (small) {
             fn = ld ? redist_fused_zip_kernel<true, NT, true> : redist_fused_zip_kernel<false, NT, true>;
         } else {
             if (ld) { REDIST_PICK(_zip_kernel, true, NT, false) } else { REDIST_PICK(_zip_kernel, false, NT, false) }
         }
-    } else if (geo.mode == kModeGather) {
-        if (small) {
-            fn = ld ? redist_fused_gather_kernel<true, NT, true> : redist_fused_gather_kernel<false, NT, true>;
-        } else {
-            if (ld) { REDIST_PICK(_gather_kernel, true, NT, false) } else { REDIST_PICK(_gather_kernel, false, NT, false) }
-        }
-    } else if (geo.mode == kModeRows) {
-        REDIST_PICK(_kernel, 0, NT)
-    } else if (geo.mode == kModeUnits) {
-        REDIST_PICK(_kernel, 3, NT)
-    } else if (geo.aligned) {
-        REDIST_PICK(_kernel, 1, NT)
+#endif
     } else {
-        REDIST_PICK(_kernel, 2, NT)
+#if REDIST_IN(1)
+        if (geo.bulk == 2) {
+            REDIST_PICK(_ragged_bulk_kernel, NT)
+        } else if (geo.bulk) {
+            REDIST_PICK(_bulk_kernel, NT)
+        } else if (geo.mode == kModeGather) {
+            if (small) {
+                fn = ld ? redist_fused_gather_kernel<true, NT, true> : redist_fused_gather_kernel<false, NT, true>;
+            } else {
+                if (ld) { REDIST_PICK(_gather_kernel, true, NT, false) } else { REDIST_PICK(_gather_kernel, false, NT, false) }
+            }
+        } else if (geo.mode == kModeRows) {
+            REDIST_PICK(_kernel, 0, NT)
+        } else if (geo.mode == kModeUnits) {
+            REDIST_PICK(_kernel, 3, NT)
+        } else if (geo.aligned) {
+            REDIST_PICK(_kernel, 1, NT)
+        } else {
+            REDIST_PICK(_kernel, 2, NT)
+        }
+#endif
     }
 #undef REDIST_PICK
     return reinterpret_cast<const void *>(fn);
@@ -1684,14 +1711,13 @@ void fill_params(PreparedLaunch &pl, const CopyGeometry &geo, const char *const 
     for (int i = 0; i < n_dst; ++i) P->dst[i] = dst_tab[i];
 }
 
-}  // namespace
-
-cudaError_t read_bulk_timeouts(unsigned int *out)
+// this part's counters
+cudaError_t own_bulk_timeouts(unsigned int *out)
 {
     return cudaMemcpyFromSymbol(out, g_bulk_timeouts, sizeof(unsigned int));
 }
 
-cudaError_t read_bounds_report(long long out[5])
+cudaError_t own_bounds_report(long long out[5])
 {
 #ifdef REDIST_BOUNDS
     unsigned long long n = 0;
@@ -1709,6 +1735,71 @@ cudaError_t read_bounds_report(long long out[5])
 #endif
 }
 
+}  // namespace
+
+// What the parts offer each other: the entry point of a launch whose kernels live there, and their counters.
+#define REDIST_DECLARE_PART(N)                                                               \
+    const void *entry_in_part##N(int kernel, const CopyGeometry &geo, bool small_table);     \
+    cudaError_t bulk_timeouts_in_part##N(unsigned int *out);                                  \
+    cudaError_t bounds_report_in_part##N(long long out[5]);
+#define REDIST_DEFINE_PART(N)                                                                \
+    const void *entry_in_part##N(int kernel, const CopyGeometry &geo, bool small_table)      \
+    {                                                                                        \
+        return small_table ? entry_for<kSmallTable>(kernel, geo) : entry_for<kLargeTable>(kernel, geo); \
+    }                                                                                        \
+    cudaError_t bulk_timeouts_in_part##N(unsigned int *out) { return own_bulk_timeouts(out); } \
+    cudaError_t bounds_report_in_part##N(long long out[5]) { return own_bounds_report(out); }
+REDIST_DECLARE_PART(1)
+REDIST_DECLARE_PART(2)
+REDIST_DECLARE_PART(3)
+#if REDIST_PART == 1
+REDIST_DEFINE_PART(1)
+#elif REDIST_PART == 2
+REDIST_DEFINE_PART(2)
+#elif REDIST_PART == 3
+REDIST_DEFINE_PART(3)
+#endif
+
+#if REDIST_PART <= 1      // the host side lives in the single translation unit, or in part 1
+
+cudaError_t read_bulk_timeouts(unsigned int *out)
+{
+#if REDIST_PART == 0
+    return own_bulk_timeouts(out);
+#else
+    unsigned int a = 0, b = 0, c = 0;
+    cudaError_t ce = bulk_timeouts_in_part1(&a);
+    if (ce == cudaSuccess) ce = bulk_timeouts_in_part2(&b);
+    if (ce == cudaSuccess) ce = bulk_timeouts_in_part3(&c);
+    *out = a + b + c;
+    return ce;
+#endif
+}
+
+cudaError_t read_bounds_report(long long out[5])
+{
+#if REDIST_PART == 0
+    return own_bounds_report(out);
+#else
+    // violations added up; the record of the first part that has one
+    long long part[3][5];
+    cudaError_t ce = bounds_report_in_part1(part[0]);
+    if (ce == cudaSuccess) ce = bounds_report_in_part2(part[1]);
+    if (ce == cudaSuccess) ce = bounds_report_in_part3(part[2]);
+    if (ce != cudaSuccess) {
+        for (int i = 0; i < 5; ++i) out[i] = -1;
+        return ce;
+    }
+    for (int i = 0; i < 5; ++i) out[i] = 0;
+    for (int k = 2; k >= 0; --k) {
+        out[0] += part[k][0];
+        if (part[k][0] > 0)
+            for (int i = 1; i < 5; ++i) out[i] = part[k][i];
+    }
+    return cudaSuccess;
+#endif
+}
+
 cudaError_t prepare_copy(int kernel, const CopyGeometry &geo, const char *const *src_tab, int n_src,
                          char *const *dst_tab, int n_dst, int pdl, void *storage, size_t storage_bytes,
                          PreparedLaunch &pl)
@@ -1718,7 +1809,13 @@ cudaError_t prepare_copy(int kernel, const CopyGeometry &geo, const char *const 
     if (!storage || (reinterpret_cast<uintptr_t>(storage) & 15u) || storage_bytes < param_bytes(small ? kSmallTable : kLargeTable))
         return cudaErrorInvalidValue;
     pl.params = storage;
+#if REDIST_PART == 0
     pl.fn = small ? entry_for<kSmallTable>(kernel, geo) : entry_for<kLargeTable>(kernel, geo);
+#else
+    pl.fn = part_of(geo) == 3   ? entry_in_part3(kernel, geo, small)
+            : part_of(geo) == 2 ? entry_in_part2(kernel, geo, small)
+                                : entry_in_part1(kernel, geo, small);
+#endif
     if (small)
         fill_params<kSmallTable>(pl, geo, src_tab, n_src, dst_tab, n_dst);
     else
@@ -1767,5 +1864,7 @@ cudaError_t launch_prepared(const PreparedLaunch &pl, cudaStream_t stream)
     void *args[1] = {pl.params};
     return cudaLaunchKernelExC(&cfg, pl.fn, args);
 }
+
+#endif   // REDIST_PART <= 1
 
 }  // namespace redist
