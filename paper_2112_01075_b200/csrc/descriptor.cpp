@@ -261,7 +261,15 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
         const RowDigit &d = rows.back();
         const i64 bs = long_dst ? run_bytes : m * run_bytes, bd = long_dst ? m * run_bytes : run_bytes;
         // a source segment of a full item should be worth a bulk copy
-        if (piece_stride == run_bytes && d.b1 == bs && d.b2 == bd && d.n * bs >= 256 && d.n * bd >= kZipMinRange && m <= 16) zip_n = d.n;
+        // (one row of the zipped digit must fit the item's shared-memory tile: m segments of a run each, or one
+        // segment of a long row; with up to 16 tiles and runs below 2 KiB it always does.  17 to 64 tiles, measured
+        // on 32: target rows zipped from 32 tiles and stored to 32 replicas 2.2-3.7 -> 5.3-5.5 TB/s against the
+        // ragged chunk walk; long source rows unzipped into 32 tiles 3.8-4.5 -> 5.6-5.7 on runs of 260-372 bytes,
+        // but 0.94x from 512 bytes, where the ragged chunk walk stays)
+        const i64 one_row = (long_dst ? m : 1) * ((long_dst ? run_bytes : m * run_bytes) + 48);
+        if (piece_stride == run_bytes && d.b1 == bs && d.b2 == bd && d.n * bs >= 256 && d.n * bd >= kZipMinRange && m <= 64 &&
+            one_row <= 38 * 1024 && (m <= 16 || long_dst || run_bytes < 512))
+            zip_n = d.n;
     }
     // box: the item is a super-box -- lcm(source tile, target tile) indices in each of the innermost
     // differing dimensions ("inner" dimensions, kp and as many before it as it takes to make the

@@ -57,7 +57,7 @@ def run_launch(L: dict, src_bufs, dst_bufs):
         m1, m2 = G["unit_m1"][u], G["unit_m2"][u]
         long_dst = G["gl_long_dst"] == 1
         m = max(m1, m2)
-        assert run < 2048 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 16
+        assert run < 2048 and inner == 1 and mul == span == m == G["gl_m"] and min(m1, m2) == 1 and m <= 64
         assert (m2 > 1) == long_dst and G["units_per_run"] * unit == run
         assert (G["unit_b2"][u] if long_dst else G["unit_b1"][u]) == run
         n = G["row_n"][-1]

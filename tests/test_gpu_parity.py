@@ -661,6 +661,9 @@ INTERLEAVED = [   # mesh, global shape, sharded type, gathered type, element byt
     ((2, 2), (16, 6, 4), ((), (), (0, 1)), ((), (0,), ()), 8, 5, 3),
     ((2, 2, 2), (6, 5, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4, 7, 7),
     ((2, 2, 2), (700, 3, 56), ((), (), (0, 1, 2)), ((), (), (0,)), 4, 7, 7),      # many row groups, ragged last one
+    ((2, 4, 4), (6, 416), ((), (0, 1, 2)), ((), ()), 4, 7, 7),                      # 32 tiles zipped into one row, 52-byte runs
+    ((4, 4, 4), (8, 320), ((), (2, 1, 0)), ((), ()), 4, 5, 7),                      # 64 tiles, 20-byte runs
+    ((2, 4, 4), (5, 4, 864), ((), (), (0, 1, 2)), ((), (), ()), 2, 7, 7),           # 32 tiles, 54-byte runs of 2-byte units
 ]
 
 
