@@ -347,8 +347,28 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             // ragged head and tail --, 1.03-1.06x up to 1536 bytes unless the fan-out is 8 or more, 1.04-1.15x
             // where the zipped digit has fewer than 8 rows, 0.97x elsewhere)
             const i64 zip_range = zip_n * (m2[kp] > 1 ? std::max(m1[kp], m2[kp]) * run_bytes : run_bytes);
+            // Two more cases go to the super-boxes, found by probing row-to-column transposes over 8-64 tiles:
+            // zip launches that could use neither the periodic nor the by-range walk (tabulated or flat walk:
+            // 0.88x of the super-boxes on 33 problems of the sweep, 2.8-3.0 against 4.1-5.2 TB/s on 2-byte units),
+            // and long source rows of runs up to 16 bytes unzipped into 32 or more tiles, where every store
+            // instruction of the zip walk scatters 16-byte pieces over as many tiles (2.3-2.8 against 4.5-5.8 TB/s).
+            bool zip_slow = false;
+            if (zip_n > 0) {
+                const bool ld = m2[kp] > 1;
+                const i64 zm = std::max(m1[kp], m2[kp]), row_bytes = zm * run_bytes;
+                const i64 zseg = ld ? zm : 1, seg_row = ld ? run_bytes : row_bytes;
+                i64 rpb = std::max<i64>(1, std::min<i64>(zip_n, kItemBytes / row_bytes));
+                rpb = std::max<i64>(1, std::min<i64>(rpb, (38 * 1024 / zseg - 48) / seg_row));
+                const i64 L = ld ? row_bytes : run_bytes, pc = L / std::gcd<i64>(16, L);
+                const i64 lanes_needed = !ld && run_bytes <= 16 ? pc * zm : pc;
+                const bool periodic = (tune.zip_walks & 1) && lanes_needed <= kBlockThreads - 1 && rpb * L / 16 >= 2 * pc;
+                const bool by_range = (tune.zip_walks & 2) && run_bytes * 4 >= 32 * vec && vec < 16 &&
+                                      rpb * (ld ? zm : 1) * ((run_bytes + 15) / 16) >= std::max<i64>(1, tune.zip_by_range_slots);
+                zip_slow = (!periodic && !by_range) || (!ld && run_bytes <= 16 && zm >= 32);
+            }
             const bool wanted = tune.box >= 2 ||
-                                (zip_n > 0 ? (zip_range < 1536 && (zip_range < 768 || fan < 8)) || zip_n < 8 : run_bytes < 256);
+                                (zip_n > 0 ? (zip_range < 1536 && (zip_range < 768 || fan < 8)) || zip_n < 8 || zip_slow
+                                           : run_bytes < 256);
             if (!fits || !worth || !wanted || sup > (1ll << 30)) bxK = -2;
         }
     }
