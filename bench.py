@@ -697,6 +697,10 @@ def run_sweep(args):
         pairs, label = wl.config4(max(100, args.pairs)), "c4: f32 [64,128,256,512], mesh {x:2,y:4,z:2}, %d seeded random pairs"
     elif args.workload == "adv":
         pairs, label = wl.adversarial_problems(), "adv: the %d problems of the paper's table of largest slow-downs"
+    elif args.workload == "probes":
+        pairs, label = wl.structured_probes(), \
+            "probes: %d transposes, slices and allgathers with every mesh axis on one dimension, 8-64 devices, odd widths"
+        args.pairs = max(args.pairs, len(pairs))
     else:
         pairs, label = wl.evaluation_like_problems(args.pairs), \
             "eval: %d random problems shaped like the paper's evaluation sample (3 mesh axes, <= 6-D, 64-800 MB)"
@@ -822,7 +826,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5",
-                    choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval"])
+                    choices=["c1", "c2", "c3", "c3a", "c3b", "c3c", "c4", "c5", "c5a", "c5b", "adv", "eval", "probes"])
     ap.add_argument("--pairs", type=int, default=100, help="sweeps: how many problems to run")
     ap.add_argument("--only", default="", help="sweeps: comma-separated problem names to run")
     ap.add_argument("--elem-bytes", type=int, default=0, choices=[0, 1, 2, 4, 8, 16],
@@ -855,7 +859,7 @@ def main():
             api.tuning_set(k.strip(), int(v))
     if args.standin:
         run_standin(args)
-    elif args.workload in ("c4", "adv", "eval"):
+    elif args.workload in ("c4", "adv", "eval", "probes"):
         if args.impl == "reference":
             raise SystemExit("the sweeps (c4, adv, eval) are GPU-side measurements; use another workload for --impl reference")
         run_sweep(args)

@@ -229,6 +229,37 @@ def adversarial_problems() -> List[Workload]:
                      "adversarial table") for i, (n, g, s, d) in enumerate(spec)]
 
 
+def structured_probes() -> List[Workload]:
+    """Shapes a random sample seldom draws: every mesh axis on ONE dimension, over 8, 16, 32 and 64 devices, with
+    odd widths per device.  Row-to-column transposes (2- and 4-byte elements, widths of 3 to 257 elements),
+    and slices / allgathers of the last dimension of a replicated array (4-byte elements, widths of 33 to 401).
+    About 256 MB (transposes) and 200 MB (slices) of global data each."""
+    meshes = {8: (2, 2, 2), 16: (2, 2, 4), 32: (2, 4, 4), 64: (4, 4, 4)}
+    names = ("a", "b", "c")
+    out: List[Workload] = []
+    for n, mesh in meshes.items():
+        axes = [0, 1, 2]
+        for e in (4, 2):
+            for w in (3, 7, 13, 33, 65, 129, 257):
+                cols = n * w
+                rows = max(n, ((256 << 20) // (cols * e)) // n * n)
+                g = (rows, cols)
+                out.append(Workload(f"t{n}_e{e}_w{w}", mesh, names, e, dist_type(g, [axes, []]), dist_type(g, [[], axes]),
+                                    "random_bits", 0, "row-sharded to column-sharded"))
+    for n, mesh in meshes.items():
+        if n == 64:
+            continue
+        axes = [0, 1, 2]
+        for w in (33, 65, 93, 129, 255, 401):
+            cols = n * w
+            g = (max(64, (200 << 20) // (cols * 4)), cols)
+            out.append(Workload(f"s{n}_w{w}", mesh, names, 4, dist_type(g, [[], []]), dist_type(g, [[], axes]),
+                                "random_bits", 0, "replicated to sliced along the last dimension"))
+            out.append(Workload(f"g{n}_w{w}", mesh, names, 4, dist_type(g, [[], axes]), dist_type(g, [[], []]),
+                                "random_bits", 0, "sliced along the last dimension to replicated"))
+    return out
+
+
 def evaluation_like_problems(n: int, seed: int = 2112010770) -> List[Workload]:
     """Random problems in the shape of the paper's evaluation sample (Section 8): three mesh axes,
     arrays of two to six dimensions holding 64 MB-800 MB of 4-byte elements, every axis either
