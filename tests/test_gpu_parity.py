@@ -716,6 +716,21 @@ def test_short_run_kernels_on_one_and_two_byte_units(mesh, gshape, a1, a2, e, un
     assert seen & {7, 8}, seen
 
 
+def test_structured_probes_at_reduced_size():
+    """Every mesh axis on one dimension over 8-64 devices, odd widths of 2- and 4-byte elements: the 92 shapes of
+    `bench.py --workload probes` with eight rows per device (the kernel choice depends on the widths, which stay)."""
+    seen = set()
+    for w in wl.structured_probes():
+        n = w.n_devices
+        rows = 8 * n if w.name.startswith("t") else 96
+        ws = w.scaled((rows, w.src.global_shape[1]))
+        src, dst, src_tiles, want = make_case(ws, seed=len(seen) + 7)
+        plan, got = run_gpu(ws.mesh_shape, src, dst, ws.elem_bytes, src_tiles)
+        assert_same(got, want, ws.name)
+        seen.update(plan.launch_info(q).variant for q in range(plan.num_launches))
+    assert seen >= {6, 7, 8}, seen
+
+
 @pytest.mark.parametrize("g,variant", [((32768, 32768), 4), ((44739243, 24), 7)])
 def test_four_gib_tiles_need_64_bit_offsets(g, variant):
     """u32 arrays of 4 GiB and a little more (value = global linear index) on two devices: replicated

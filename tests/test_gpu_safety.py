@@ -68,6 +68,7 @@ for case in T.INTERLEAVED:
     T.test_gather_walk_and_zip_kernels(*case)
 for case in T.SMALL_UNITS:
     T.test_short_run_kernels_on_one_and_two_byte_units(*case)
+T.test_structured_probes_at_reduced_size()
 for mesh, gshape, a1, a2, e, v in TP.KERNEL_CHOICE:
     if int(np.prod(gshape)) * e > (8 << 20):
         gshape = tuple(max(8, s // 8) if k else s for k, s in enumerate(gshape))
