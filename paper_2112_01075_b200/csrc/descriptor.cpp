@@ -350,8 +350,9 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
             // Two more cases go to the super-boxes, found by probing row-to-column transposes over 8-64 tiles:
             // zip launches that could use neither the periodic nor the by-range walk (tabulated or flat walk:
             // 0.88x of the super-boxes on 33 problems of the sweep, 2.8-3.0 against 4.1-5.2 TB/s on 2-byte units),
-            // and long source rows of runs up to 16 bytes unzipped into 32 or more tiles, where every store
-            // instruction of the zip walk scatters 16-byte pieces over as many tiles (2.3-2.8 against 4.5-5.8 TB/s).
+            // and long source rows of runs up to 16 bytes unzipped into 16 or more tiles, where every store
+            // instruction of the zip walk scatters 16-byte pieces over as many tiles (32 and 64 tiles: 2.3-2.8
+            // against 4.5-5.8 TB/s; 16 tiles: 4.3-4.6 against 5.6-6.1 on 12- and 14-byte runs, 4.8 against 4.4 on 6-byte runs).
             bool zip_slow = false;
             if (zip_n > 0) {
                 const bool ld = m2[kp] > 1;
@@ -364,7 +365,7 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
                 const bool periodic = (tune.zip_walks & 1) && lanes_needed <= kBlockThreads - 1 && rpb * L / 16 >= 2 * pc;
                 const bool by_range = (tune.zip_walks & 2) && run_bytes * 4 >= 32 * vec && vec < 16 &&
                                       rpb * (ld ? zm : 1) * ((run_bytes + 15) / 16) >= std::max<i64>(1, tune.zip_by_range_slots);
-                zip_slow = (!periodic && !by_range) || (!ld && run_bytes <= 16 && zm >= 32);
+                zip_slow = (!periodic && !by_range) || (!ld && run_bytes <= 16 && zm >= 16);
             }
             const bool wanted = tune.box >= 2 ||
                                 (zip_n > 0 ? (zip_range < 1536 && (zip_range < 768 || fan < 8)) || zip_n < 8 || zip_slow
