@@ -178,6 +178,8 @@ void redist_plan_cache_clear(void);
  *   "l2_hint"            0..4   bulk copies of the plain bulk-copy kernels that carry an L2 evict-first policy: none /
  *                               loads / stores / both / stores where every segment goes to four or more replicas
  *                               (default 4)
+ *   "piece"              0/1    1 (default): on units of 1 or 2 bytes and runs of 64 bytes and more the super-box
+ *                               kernels read a chunk that lies inside one run as one unaligned 16-byte piece; 0: unit by unit
  *   "pdl"                0/1    1: kernels use programmatic dependent launch (default); 0: plain stream order
  *   "nvtx"               0/1    1: redist_execute and redist_execute_static wrap every kernel launch in an NVTX
  *                               range named after the collective, for timeline profilers (default 0)

@@ -79,6 +79,7 @@ const TuningName kTuningNames[] = {
     {"zip_by_range_slots", &Tuning::zip_by_range_slots, 1, 1 << 20},
     {"item_kb", &Tuning::item_kb, 0, 1024},
     {"l2_hint", &Tuning::l2_hint, 0, 4},
+    {"piece", &Tuning::piece, 0, 1},
     {"pdl", &Tuning::pdl, 0, 1},
     {"nvtx", &Tuning::nvtx, 0, 1},
     {"step_latency", &Tuning::step_latency, 0, int64_t(1) << 50},

@@ -155,6 +155,7 @@ struct CopyGeometry {
     FastDiv bx_row_units_div;        // kModeBox: division by the units of one target row (zip_lut_units)
     uint32_t wait_polls;             // bulk-copy kernels: mbarrier polls before a block gives up (bounded wait)
     uint32_t l2_hint;                // plain bulk-copy kernels: 1 loads, 2 stores (3 both) carry an L2 evict-first policy
+    uint32_t one_piece;              // super-box kernels on units of 1 or 2 bytes: chunks inside one run are read in one piece
     uint32_t test_extra_tx;          // test only: bytes announced on the mbarrier beyond what the copies deliver, so
                                      // that every copy lands but the phase never completes (0 in every real plan)
     uint32_t n_src_tab, n_dst_tab;   // entries of the two pointer tables

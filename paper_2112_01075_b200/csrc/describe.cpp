@@ -109,7 +109,7 @@ void describe(Plan &p)
           << ",\"rows_per_item\":" << G.rows_per_item << ",\"items_per_box\":" << G.items_per_box.d << ",\"fast_boxes\":" << G.fast_boxes.d
           << ",\"n_items\":" << G.n_items << ",\"n_row_tab\":" << G.n_row_tab << ",\"tab_inner\":" << G.tab_inner.d << ",\"inner_n\":" << G.inner_n.d << ",\"inner_digit\":" << int(G.inner_digit) << ",\"inner_span\":" << G.inner_span << ",\"inner_mul\":" << G.inner_mul << ",\"gl_long_dst\":" << G.gl_long_dst << ",\"stage_pitch\":" << G.stage_pitch
           << ",\"units_per_run\":" << G.units_per_run.d << ",\"gl_levels\":" << G.gl_levels << ",\"gl_stretch\":" << G.gl_stretch
-          << ",\"gl_m\":" << G.gl_m.d << ",\"zip_seg_pitch\":" << G.zip_seg_pitch << ",\"zip_slots\":" << G.zip_slots.d << ",\"zip_cpr\":" << G.zip_cpr.d << ",\"zip_lut_units\":" << G.zip_lut_units << ",\"zip_period\":" << G.zip_period.d << ",\"zip_period_rows\":" << G.zip_period_rows << ",\"zip_width\":" << G.zip_width << ",\"l2_hint\":" << G.l2_hint << ",\"gl_n\":";
+          << ",\"gl_m\":" << G.gl_m.d << ",\"zip_seg_pitch\":" << G.zip_seg_pitch << ",\"zip_slots\":" << G.zip_slots.d << ",\"zip_cpr\":" << G.zip_cpr.d << ",\"zip_lut_units\":" << G.zip_lut_units << ",\"zip_period\":" << G.zip_period.d << ",\"zip_period_rows\":" << G.zip_period_rows << ",\"zip_width\":" << G.zip_width << ",\"l2_hint\":" << G.l2_hint << ",\"one_piece\":" << G.one_piece << ",\"gl_n\":";
         fd(o, G.gl_n, G.gl_levels);
         o << ",\"gl_b1\":";
         raw(o, G.gl_b1, G.gl_levels);

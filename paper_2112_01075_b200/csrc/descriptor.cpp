@@ -789,6 +789,10 @@ redist_status build_copy(const Plan &p, const Layout &a, const Layout &b, Launch
     // evict-first stores measured on the plain bulk-copy kernels by fan-out: 1: +0.1 %, 2: -0.4 %, 4: +0.5 %, 8 and
     // 16: +1.1 % (c3c 6.50 -> 6.55 TB/s); evict-first loads cost 0.6-1.7 % everywhere
     G.l2_hint = tune.l2_hint == 4 ? (fan >= 4 ? 2u : 0u) : uint32_t(tune.l2_hint);
+    // super-boxes of 1- and 2-byte units on runs of 64 bytes and more: most chunks lie inside one run, and the kernel
+    // that reads such a chunk as one unaligned 16-byte piece pays (1.2-1.3x on 1-byte units, 1.0-1.1x on 2-byte
+    // units; 0.85x on runs below 64 bytes; in the zip kernels 0.93-0.98x, not built)
+    G.one_piece = tune.piece != 0 && vec < 4 && run_bytes >= 64 && G.mode == kModeBox ? 1u : 0u;
     G.test_extra_tx = uint32_t(std::max<i64>(0, std::min<i64>(tune.test_extra_tx, 1 << 20)));
     G.n_src_tab = uint32_t(out.src_holder.size());
     G.n_dst_tab = uint32_t(out.dst_devs.size());

@@ -866,6 +866,22 @@ __device__ __forceinline__ uint4 lds_shifted(const unsigned char *tile, uint32_t
     return funnel_shift16(a, p[1], m);
 }
 
+// 16 bytes of shared memory from any byte address, as five aligned words funnel-shifted into four: no
+// branch on the misalignment, so the lanes of a warp may each have their own.  Reads the words that cover
+// [at, at + 16), i.e. up to 3 bytes before `at` and up to 4 bytes past at + 16.
+__device__ __forceinline__ uint4 lds_unaligned16(const unsigned char *tile, uint32_t at)
+{
+    const uint32_t bs = (at & 3u) * 8u;
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(tile + (at & ~3u));
+    const uint32_t w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3], w4 = w[4];
+    uint4 o;
+    o.x = __funnelshift_r(w0, w1, bs);
+    o.y = __funnelshift_r(w1, w2, bs);
+    o.z = __funnelshift_r(w2, w3, bs);
+    o.w = __funnelshift_r(w3, w4, bs);
+    return o;
+}
+
 template <int NT>
 __device__ __forceinline__ void ragged_bulk_body(const CopyParams<NT> &P)
 {
@@ -1388,7 +1404,11 @@ REDIST_DEFINE_ZIP_KERNEL(redist_fused_zip_kernel)
 // keeps (row, position in row) by adding a constant per step instead of dividing.  The host picks the
 // width: a warp or more per range as a rule, fewer lanes -- several ranges per warp -- where the units of
 // one range would all fall into a few shared-memory banks.
-template <typename T, int NT>
+// PIECE (units of 1 and 2 bytes on runs of 64 bytes and more, a kernel of its own): a chunk that lies inside
+// one run -- contiguous on both sides -- is read as one unaligned 16-byte piece instead of 8 or 16 units
+// (measured on the super-box launches of the 1-byte sweep 1.2-1.3x, of the 2-byte sweep 1.0-1.1x; the same in
+// the zip kernels measured 0.93-0.98x and is not built).
+template <typename T, int NT, bool PIECE>
 __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char *tile, uint32_t *base_of,
                                          uint32_t *tile_of, int64_t *row_d0, uint32_t mbar, unsigned int *wait_failed)
 {
@@ -1513,7 +1533,17 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
                 uint4 v;
                 T t[kPer];
             } u;
-            if (p + uint32_t(kPer) <= row_units) {
+            bool one_piece = false;
+            if constexpr (PIECE) {
+                const uint32_t in_run = p - fdiv(p, g.bx_trail) * g.bx_trail.d;
+                one_piece = in_run + uint32_t(kPer) <= g.bx_trail.d;
+                if (one_piece) {
+                    const uint32_t w = at + place[p];
+                    if (CHK_SMEM(w & ~3u, 20u)) u.v = lds_unaligned16(tile, w);
+                }
+            }
+            if (one_piece) {
+            } else if (p + uint32_t(kPer) <= row_units) {
 #pragma unroll
                 for (int i = 0; i < kPer; ++i) {
                     const uint32_t w = at + place[p + uint32_t(i)];
@@ -1575,7 +1605,7 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
 }
 
 #define REDIST_DEFINE_BOX_KERNEL(NAME)                                                               \
-    template <int NT, bool SMALL>                                                                    \
+    template <int NT, int SMALL>                                                                     \
     __global__ void __launch_bounds__(kBlockThreads) NAME(const __grid_constant__ CopyParams<NT> P)  \
     {                                                                                                \
         extern __shared__ __align__(128) unsigned char tile[];                                       \
@@ -1586,16 +1616,16 @@ __device__ __forceinline__ void box_body(const CopyParams<NT> &P, unsigned char 
         __shared__ unsigned int wait_failed;                                                         \
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");                              \
         const uint32_t mbar = smem_addr(&mbar_storage);                                              \
-        if constexpr (SMALL) {                                                                       \
+        if constexpr (SMALL != 0) {      /* 1: units of 1 and 2 bytes, 2: the same with chunks read in one piece */ \
             if (P.g.unit_bytes == 2)                                                                 \
-                box_body<uint16_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed);       \
+                box_body<uint16_t, NT, SMALL == 2>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); \
             else                                                                                     \
-                box_body<uint8_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed);        \
+                box_body<uint8_t, NT, SMALL == 2>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); \
         } else {                                                                                     \
             switch (P.g.unit_bytes) {                                                                \
-            case 16: box_body<uint4, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
-            case 8: box_body<uint2, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
-            default: box_body<uint32_t, NT>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            case 16: box_body<uint4, NT, false>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            case 8: box_body<uint2, NT, false>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
+            default: box_body<uint32_t, NT, false>(P, tile, base_of, tile_of, row_d0, mbar, &wait_failed); break; \
             }                                                                                        \
         }                                                                                            \
     }
@@ -1664,7 +1694,11 @@ const void *entry_for(int kernel, const CopyGeometry &geo)
     // instantiations, and of the time to compile them, for a rare case)
     if (part_of(geo) == 3) {
 #if REDIST_IN(3)
-        if (small) { fn = redist_fused_box_kernel<NT, true>; } else { REDIST_PICK(_box_kernel, NT, false) }
+        if (small) {
+            fn = geo.one_piece ? redist_fused_box_kernel<NT, 2> : redist_fused_box_kernel<NT, 1>;
+        } else {
+            REDIST_PICK(_box_kernel, NT, 0)
+        }
 #endif
     } else if (part_of(geo) == 2) {
 #if REDIST_IN(2)

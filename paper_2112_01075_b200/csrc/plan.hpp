@@ -62,6 +62,7 @@ struct Tuning {
     int64_t zip_walks = 7;            // chunk -> units maps the zip kernels may use: 1 periodic, 2 by range, 4 tabulated
     int64_t zip_by_range_slots = 256; // fewest chunk slots of a range for the by-range walk
     int64_t item_kb = 0;              // KiB read per work item (0: 32 / 16 / 8 by fan-out, bulk copies 20 / 12 / 6)
+    int64_t piece = 1;                // 0: the small-unit super-box kernels never read a chunk in one piece
     int64_t l2_hint = 4;              // plain bulk-copy kernels, L2 evict-first policy on: 0 nothing, 1 loads, 2 stores, 3 both, 4 stores from fan-out 4
     int64_t pdl = 1;                  // 0: plain stream order instead of programmatic dependent launch
     int64_t nvtx = 0;                 // 1: redist_execute wraps every kernel launch in an NVTX range named after the step
@@ -72,7 +73,7 @@ struct Tuning {
     bool operator==(const Tuning &o) const
     {
         return bulk == o.bulk && gather == o.gather && zip == o.zip && box == o.box && box_width == o.box_width && zip_walks == o.zip_walks &&
-               zip_by_range_slots == o.zip_by_range_slots && item_kb == o.item_kb && l2_hint == o.l2_hint && pdl == o.pdl && nvtx == o.nvtx &&
+               zip_by_range_slots == o.zip_by_range_slots && item_kb == o.item_kb && l2_hint == o.l2_hint && piece == o.piece && pdl == o.pdl && nvtx == o.nvtx &&
                step_latency == o.step_latency && wait_polls == o.wait_polls && test_extra_tx == o.test_extra_tx &&
                test_shrink_tiles == o.test_shrink_tiles;
     }

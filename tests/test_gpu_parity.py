@@ -694,6 +694,11 @@ SMALL_UNITS = [   # mesh, global shape, source axes, target axes, element bytes,
     ((4, 4, 4), (8, 12, 2, 28, 20, 12), ((), (1,), (), (2,), (), ()), ((2,), (), (), (), (0,), (1,)), 1, 1),  # 3-byte runs
     ((4, 2, 2), (2, 17, 16, 28, 9, 8), ((1,), (), (2, 0), (), (), ()), ((), (), (), (1,), (), (0, 2)), 2, 2),  # single elements 16 bytes apart
     ((2, 2, 2), (6, 6, 6, 48, 10, 26), ((), (2,), (), (0,), (), ()), ((), (), (1,), (), (2,), (0,)), 1, 1),  # 13-byte runs
+    # runs of 64 bytes and more: chunks inside one run are read in one piece
+    ((8,), (33, 520), ((), (0,)), ((), ()), 2, 2),                                                          # 130-byte runs
+    ((2, 4), (6, 10, 300), ((), (), (1,)), ((), (), ()), 1, 1),                                            # 75-byte runs
+    ((2, 2, 2), (6, 6, 6, 48, 10, 74), ((), (2,), (), (0,), (), ()), ((), (), (1,), (), (2,), (0,)), 2, 2),  # 74-byte runs, super-boxes
+    ((2, 2, 2), (4, 6, 6, 48, 10, 150), ((), (2,), (), (0,), (), ()), ((), (), (1,), (), (2,), (0,)), 1, 1), # 75-byte runs, super-boxes
 ]
 
 
@@ -706,7 +711,8 @@ def test_short_run_kernels_on_one_and_two_byte_units(mesh, gshape, a1, a2, e, un
     seen = set()
     for src, dst in (((gshape, a1), (gshape, a2)), ((gshape, a2), (gshape, a1))):
         src_tiles, want = oracle.reslice(mesh, src, G), oracle.reslice(mesh, dst, G)
-        for values in ({}, {"box": 2}, {"box": 0}, {"gather": 2, "zip": 0, "box": 0}):
+        for values in ({}, {"box": 2}, {"box": 0}, {"gather": 2, "zip": 0, "box": 0}, {"piece": 0}, {"piece": 0, "box": 2},
+                       {"box": 0, "zip_walks": 0}, {"box": 0, "zip_walks": 2, "zip_by_range_slots": 1}, {"box": 0, "zip_walks": 4}):
             with api.tuning(**values):
                 plan, got = run_gpu(mesh, src, dst, e, src_tiles)
             assert_same(got, want, f"small units {mesh} {src} -> {dst} {values}")

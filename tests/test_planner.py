@@ -452,7 +452,7 @@ def test_tuning_values_are_validated_and_copied_into_new_plans_only():
 
 TUNING_VALUES = {   # name: (default, lowest, highest) as the header states them
     "bulk": (1, 0, 1), "gather": (1, 0, 2), "zip": (2, 0, 2), "box": (1, 0, 2), "box_width": (0, 0, 256),
-    "zip_walks": (7, 0, 7), "zip_by_range_slots": (256, 1, 1 << 20), "item_kb": (0, 0, 1024), "l2_hint": (4, 0, 4),
+    "zip_walks": (7, 0, 7), "zip_by_range_slots": (256, 1, 1 << 20), "item_kb": (0, 0, 1024), "l2_hint": (4, 0, 4), "piece": (1, 0, 1),
     "pdl": (1, 0, 1), "nvtx": (0, 0, 1), "step_latency": (0, 0, 1 << 50), "wait_polls": (1 << 18, 1, 1 << 30),
     "test_extra_tx": (0, 0, 1 << 20), "test_shrink_tiles": (0, 0, 1 << 20),
 }
